@@ -1,0 +1,182 @@
+/*
+ * iodf.h -- C ABI of the B200 (sm_100a) integer-only discrete flow (IODF) inference library.
+ *
+ * The library runs the invertible integer flow of "Fast Lossless Neural Compression with
+ * Integer-Only Discrete Flows" (arXiv 2206.08869) in both directions on one GPU:
+ *
+ *   encode  x (uint8 image batch)  ->  z (int32 latents) + prior parameters (mu, log-scale index)
+ *   decode  z                      ->  x
+ *
+ * Every step is integer arithmetic, so both directions are exact and decode(encode(x)) == x
+ * bit for bit (Sec. 3: the change of variables p_X(x) = p_Z(f(x)) needs f to be a bijection on
+ * Z^d).
+ *
+ * Conventions
+ *   - Every function returns IODF_OK (0) or a negative iodf_status; none aborts or throws.
+ *   - "HOST" / "DEV" in a comment says where a pointer must live. The caller owns every buffer it
+ *     passes; the library owns the model object and its device workspace.
+ *   - iodf_forward / iodf_inverse enqueue work on the given CUDA stream (a cudaStream_t passed as
+ *     void*; NULL = the default stream) and return without synchronising. They allocate nothing.
+ *     At most one call per model may be in flight at a time (the model's workspace is shared).
+ *   - All validation happens on the host before anything is launched.
+ *
+ * Requantisation. rq(a; M0, s) = floor((a * M0 + 2^(30+s)) / 2^(31+s)) computed exactly in 64-bit
+ * integers: the fixed-point form, rounded half up, of the rescale factor s_W s_x / s_y of
+ * Eq. "quant_conv" (Sec. 4.1), with M0 in [2^30, 2^31) and s in [0, 31].
+ */
+#ifndef IODF_H_
+#define IODF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define IODF_ABI_VERSION 1u
+
+typedef enum {
+  IODF_OK = 0,
+  IODF_EINVAL = -1,       /* null/misaligned pointer, batch out of range, malformed descriptor      */
+  IODF_ENOMEM = -2,       /* host or device allocation failed in iodf_create                         */
+  IODF_ECUDA = -3,        /* a CUDA call failed; see iodf_last_cuda_error                            */
+  IODF_EVERSION = -4,     /* abi_version mismatch                                                    */
+  IODF_ETIMEOUT = -5,     /* a bounded device-side wait gave up (reported by iodf_check)             */
+  IODF_EUNSUPPORTED = -6, /* a valid model whose shape this build cannot run (see iodf_create)       */
+  IODF_EOVERFLOW = -7     /* a worst-case accumulator |sum| + |bias| would leave the int32 range     */
+} iodf_status;
+
+/*
+ * One integer convolution layer (Eq. 5 and Eq. "quant_conv", Sec. 4.1): stride 1, zero padding
+ * (k-1)/2, int8 weights and activations, int32 accumulator, int32 bias added to the accumulator,
+ * then rq() per OUTPUT channel, then max(0, .) if relu, then clip to [clamp_lo, clamp_hi] if
+ * has_clamp (Sec. 4.1 "Integer-Only ReLU"). Channel counts are the kept (pruned, Sec. 4.4) widths
+ * and may be odd.
+ */
+typedef struct {
+  uint32_t k;             /* kernel size: 1 or 3                                                     */
+  uint32_t c_in, c_out;
+  uint32_t relu;          /* 0 / 1                                                                   */
+  uint32_t has_clamp;     /* 0 / 1                                                                   */
+  int32_t clamp_lo, clamp_hi;
+  uint64_t weight_off;    /* element offset into `weights`: int8 [c_out][k][k][c_in]                 */
+  uint64_t requant_off;   /* element offset into `requant`: bias[c_out], M0[c_out], s[c_out]         */
+} iodf_layer_desc;
+
+/*
+ * One additive coupling (Eq. 2, Sec. 3). Before the coupling the C channels are permuted,
+ * y[k] = x[perm[k]]; x_a = y[0 : C/2] feeds the network, x_b = y[C/2 : C] is updated:
+ *   a0 = clip(rq(x_a; in_m0, in_s), -128, 127);  t = layers(a0);  z_b = x_b + t  (mod 2^32).
+ * The last layer must have relu = 0 and has_clamp = 0 (its rq output is the integer translation).
+ */
+typedef struct {
+  const int32_t* perm;            /* HOST, C entries, a permutation of 0..C-1                        */
+  int32_t in_m0, in_s;
+  uint32_t n_layers;
+  const iodf_layer_desc* layers;  /* HOST                                                            */
+} iodf_coupling_desc;
+
+/*
+ * One flow level (Sec. 5 / App. B.1): a 2x2 space-to-depth (out channel c*4 + dy*2 + dx takes
+ * in[c][2i+dy][2j+dx]), n_couplings couplings, then, if split, the second half of the channels is
+ * factored out into z and the first half goes on. With has_prior the prior head runs on the kept
+ * half: a0 = clip(rq(keep; prior_in_m0, prior_in_s), -128, 127); prior_layer maps C/2 -> 2*(C/2)
+ * channels, the first half being mu (int32, unclipped) and the second the log-scale index clipped
+ * to [ls_lo, ls_hi], one pair per factored-out element (Sec. 3, discretised logistic prior).
+ */
+typedef struct {
+  uint32_t n_couplings;
+  const iodf_coupling_desc* couplings; /* HOST                                                       */
+  uint32_t split;
+  uint32_t has_prior;                  /* requires split                                             */
+  int32_t prior_in_m0, prior_in_s;
+  iodf_layer_desc prior_layer;
+  int32_t ls_lo, ls_hi;
+} iodf_level_desc;
+
+typedef struct {
+  uint32_t abi_version;                /* IODF_ABI_VERSION                                           */
+  uint32_t in_c, in_h, in_w;           /* image shape; in_h, in_w divisible by 2^n_levels            */
+  uint32_t n_levels;
+  uint32_t max_batch;                  /* workspace is sized for this batch at create                */
+  const iodf_level_desc* levels;       /* HOST                                                       */
+} iodf_model_desc;
+
+#define IODF_MAX_LEVELS 8
+
+/* Shape of the latent. Per image, z is the concatenation, level 0 first, of every factored-out
+ * block in [channel][row][col] order, followed by the last level's remaining channels. The prior
+ * buffer holds, per image, d_fact values of mu followed by d_fact values of the log-scale index,
+ * in the order of the factored-out blocks that have a prior head. */
+typedef struct {
+  uint64_t d;                              /* latent elements per image = in_c*in_h*in_w            */
+  uint64_t d_fact;                         /* elements per image that have prior parameters         */
+  uint32_t n_levels;
+  uint32_t level_c[IODF_MAX_LEVELS], level_h[IODF_MAX_LEVELS], level_w[IODF_MAX_LEVELS];
+  uint64_t z_off[IODF_MAX_LEVELS];         /* offset of the level's factored-out block in z         */
+  uint64_t prior_off[IODF_MAX_LEVELS];     /* offset of the level's block in mu (and in ls)         */
+  uint64_t z_final_off;                    /* offset of the final block                             */
+  uint64_t macs_per_image;                 /* multiply-accumulates over the kept channels           */
+} iodf_layout;
+
+typedef struct iodf_model iodf_model;
+
+/*
+ * Validate `desc`, copy and repack weights and requant parameters to the device, size the
+ * workspace for desc->max_batch. `weights`/`requant` are HOST arrays that may be freed afterwards.
+ * `device` is a CUDA device ordinal; it is made current for the duration of the call.
+ * Errors: EINVAL (null pointer; odd channel count; perm not a permutation; M0 outside
+ * [2^30, 2^31); s outside [0, 31]; offsets beyond the blobs; layer shapes that do not chain),
+ * EOVERFLOW, EVERSION, ENOMEM, ECUDA, EUNSUPPORTED. This build runs couplings of the form
+ * conv3x3+ReLU+clip -> conv1x1+ReLU+clip -> conv3x3 with hidden activations inside the signed
+ * 8-bit range and hidden widths up to 256 kept channels, and 3x3 prior heads.
+ */
+int iodf_create(const iodf_model_desc* desc, const int8_t* weights, size_t weights_count,
+                const int32_t* requant, size_t requant_count, int device, iodf_model** out);
+
+void iodf_destroy(iodf_model* m);
+
+int iodf_get_layout(const iodf_model* m, iodf_layout* out);
+
+/*
+ * Encode: x_u8 DEV uint8 [B][in_c][in_h][in_w]  ->  z DEV int32 [B][d] and, if `prior` is not
+ * NULL, prior DEV int32 [B][2][d_fact]. 1 <= B <= max_batch. Pointers must be 16-byte aligned.
+ */
+int iodf_forward(iodf_model* m, const uint8_t* x_u8, int B, int32_t* z, int32_t* prior, void* cuda_stream);
+
+/*
+ * Decode: z DEV int32 [B][d] -> x_u8 DEV uint8 [B][in_c][in_h][in_w] (the low 8 bits of each
+ * recovered value). If `prior` is not NULL the same prior parameters as iodf_forward are written.
+ * If `out_of_range_count` (DEV uint32) is not NULL, the number of recovered values outside 0..255
+ * is ADDED to it (the caller zeroes it); this can only be non-zero for a z that no image encodes to.
+ */
+int iodf_inverse(iodf_model* m, const int32_t* z, int B, uint8_t* x_u8, int32_t* prior,
+                 uint32_t* out_of_range_count, void* cuda_stream);
+
+/*
+ * The same two operations for HOST buffers (pinned memory recommended): inputs are copied to a
+ * device staging area owned by the model, the flow runs, and the results are copied back, all
+ * enqueued on `cuda_stream`; the host buffers are valid once the stream has been synchronised.
+ */
+int iodf_forward_host(iodf_model* m, const uint8_t* x_u8_host, int B, int32_t* z_host, int32_t* prior_host,
+                      void* cuda_stream);
+int iodf_inverse_host(iodf_model* m, const int32_t* z_host, int B, uint8_t* x_u8_host, void* cuda_stream);
+
+/*
+ * Synchronise `cuda_stream` and report the device status word: IODF_OK, IODF_ETIMEOUT if a
+ * bounded wait inside a kernel gave up (the outputs of that call are then undefined), or
+ * IODF_ECUDA. Clears the status word.
+ */
+int iodf_check(iodf_model* m, void* cuda_stream);
+
+/* Number of kernel launches one iodf_forward / iodf_inverse call enqueues. */
+int iodf_launches_per_call(const iodf_model* m, int inverse);
+
+const char* iodf_strerror(int status);
+int iodf_last_cuda_error(const iodf_model* m); /* the cudaError_t behind the last IODF_ECUDA          */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IODF_H_ */

@@ -1,0 +1,245 @@
+"""ctypes binding of include/iodf.h. Argument marshalling only: model dicts (numpy arrays) become
+the C descriptor structs, torch tensors become device pointers, the current torch stream becomes
+the cudaStream_t. The function names are those of the C ABI."""
+import ctypes as C
+import os
+
+import numpy as np
+
+from . import build as _build
+
+IODF_ABI_VERSION = 1
+IODF_MAX_LEVELS = 8
+
+DECLARED_SYMBOLS = ["iodf_create", "iodf_destroy", "iodf_get_layout", "iodf_forward", "iodf_inverse",
+                    "iodf_forward_host", "iodf_inverse_host", "iodf_check", "iodf_launches_per_call",
+                    "iodf_strerror", "iodf_last_cuda_error"]
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("k", C.c_uint32), ("c_in", C.c_uint32), ("c_out", C.c_uint32), ("relu", C.c_uint32),
+                ("has_clamp", C.c_uint32), ("clamp_lo", C.c_int32), ("clamp_hi", C.c_int32),
+                ("weight_off", C.c_uint64), ("requant_off", C.c_uint64)]
+
+
+class CouplingDesc(C.Structure):
+    _fields_ = [("perm", C.POINTER(C.c_int32)), ("in_m0", C.c_int32), ("in_s", C.c_int32),
+                ("n_layers", C.c_uint32), ("layers", C.POINTER(LayerDesc))]
+
+
+class LevelDesc(C.Structure):
+    _fields_ = [("n_couplings", C.c_uint32), ("couplings", C.POINTER(CouplingDesc)), ("split", C.c_uint32),
+                ("has_prior", C.c_uint32), ("prior_in_m0", C.c_int32), ("prior_in_s", C.c_int32),
+                ("prior_layer", LayerDesc), ("ls_lo", C.c_int32), ("ls_hi", C.c_int32)]
+
+
+class ModelDesc(C.Structure):
+    _fields_ = [("abi_version", C.c_uint32), ("in_c", C.c_uint32), ("in_h", C.c_uint32), ("in_w", C.c_uint32),
+                ("n_levels", C.c_uint32), ("max_batch", C.c_uint32), ("levels", C.POINTER(LevelDesc))]
+
+
+class Layout(C.Structure):
+    _fields_ = [("d", C.c_uint64), ("d_fact", C.c_uint64), ("n_levels", C.c_uint32),
+                ("level_c", C.c_uint32 * IODF_MAX_LEVELS), ("level_h", C.c_uint32 * IODF_MAX_LEVELS),
+                ("level_w", C.c_uint32 * IODF_MAX_LEVELS), ("z_off", C.c_uint64 * IODF_MAX_LEVELS),
+                ("prior_off", C.c_uint64 * IODF_MAX_LEVELS), ("z_final_off", C.c_uint64),
+                ("macs_per_image", C.c_uint64)]
+
+
+class IodfError(RuntimeError):
+    def __init__(self, status, what):
+        super().__init__("%s failed: %s (status %d)" % (what, iodf_strerror(status), status))
+        self.status = status
+
+
+_lib = None
+
+
+def load_library(path=None):
+    """Load libiodf_b200.so (building it with nvcc if it is missing or stale). Raises if that is
+    impossible: there is no fallback implementation."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    lib_path = path or _build.build()
+    if not os.path.exists(lib_path):
+        raise RuntimeError("libiodf_b200.so is missing: run paper_2206_08869_b200.build.build()")
+    L = C.CDLL(lib_path)
+    vp = C.c_void_p
+    L.iodf_create.restype = C.c_int
+    L.iodf_create.argtypes = [C.POINTER(ModelDesc), vp, C.c_size_t, vp, C.c_size_t, C.c_int, C.POINTER(vp)]
+    L.iodf_destroy.restype = None
+    L.iodf_destroy.argtypes = [vp]
+    L.iodf_get_layout.restype = C.c_int
+    L.iodf_get_layout.argtypes = [vp, C.POINTER(Layout)]
+    L.iodf_forward.restype = C.c_int
+    L.iodf_forward.argtypes = [vp, vp, C.c_int, vp, vp, vp]
+    L.iodf_inverse.restype = C.c_int
+    L.iodf_inverse.argtypes = [vp, vp, C.c_int, vp, vp, vp, vp]
+    L.iodf_forward_host.restype = C.c_int
+    L.iodf_forward_host.argtypes = [vp, vp, C.c_int, vp, vp, vp]
+    L.iodf_inverse_host.restype = C.c_int
+    L.iodf_inverse_host.argtypes = [vp, vp, C.c_int, vp, vp]
+    L.iodf_check.restype = C.c_int
+    L.iodf_check.argtypes = [vp, vp]
+    L.iodf_launches_per_call.restype = C.c_int
+    L.iodf_launches_per_call.argtypes = [vp, C.c_int]
+    L.iodf_strerror.restype = C.c_char_p
+    L.iodf_strerror.argtypes = [C.c_int]
+    L.iodf_last_cuda_error.restype = C.c_int
+    L.iodf_last_cuda_error.argtypes = [vp]
+    if path is None:
+        _lib = L
+    return L
+
+
+def iodf_strerror(status):
+    return load_library().iodf_strerror(int(status)).decode()
+
+
+class _Marshalled:
+    """C descriptor structs for a model dict, with every referenced array kept alive."""
+
+    def __init__(self, model, max_batch):
+        self.keep = []
+        wts, par = [], []
+        self.woff = self.poff = 0
+
+        def layer(ly):
+            w = np.ascontiguousarray(ly["w"], dtype=np.int8)
+            cl = ly["clamp"]
+            if ly.get("gate") is not None:
+                raise ValueError("gated (masked-dense) layers must be compacted before deployment")
+            d = LayerDesc(ly["k"], ly["c_in"], ly["c_out"], int(ly["relu"]), int(cl is not None),
+                          cl[0] if cl else 0, cl[1] if cl else 0, self.woff, self.poff)
+            wts.append(w.reshape(-1))
+            self.woff += w.size
+            for a in (ly["bias"], ly["m0"], ly["s"]):
+                par.append(np.asarray(a, dtype=np.int32).reshape(-1))
+                self.poff += ly["c_out"]
+            return d
+
+        levels = (LevelDesc * len(model["levels"]))()
+        for li, lv in enumerate(model["levels"]):
+            cps = (CouplingDesc * max(1, len(lv["couplings"])))()
+            for ki, cp in enumerate(lv["couplings"]):
+                perm = np.ascontiguousarray(cp["perm"], dtype=np.int32)
+                lays = (LayerDesc * len(cp["layers"]))(*[layer(ly) for ly in cp["layers"]])
+                self.keep += [perm, lays]
+                cps[ki] = CouplingDesc(perm.ctypes.data_as(C.POINTER(C.c_int32)), cp["in_m0"], cp["in_s"],
+                                       len(cp["layers"]), lays)
+            self.keep.append(cps)
+            levels[li].n_couplings = len(lv["couplings"])
+            levels[li].couplings = cps
+            levels[li].split = int(lv["split"])
+            levels[li].has_prior = int(lv["prior"] is not None)
+            if lv["prior"] is not None:
+                hd = lv["prior"]
+                levels[li].prior_in_m0, levels[li].prior_in_s = hd["in_m0"], hd["in_s"]
+                levels[li].prior_layer = layer(hd["layer"])
+                levels[li].ls_lo, levels[li].ls_hi = hd["ls_lo"], hd["ls_hi"]
+        self.levels = levels
+        self.desc = ModelDesc(IODF_ABI_VERSION, model["in_c"], model["in_h"], model["in_w"], len(model["levels"]),
+                              int(max_batch), levels)
+        self.wts = np.concatenate(wts) if wts else np.zeros(1, np.int8)
+        self.par = np.concatenate(par) if par else np.zeros(1, np.int32)
+
+
+class Model:
+    """Handle of an iodf_model; destroyed when garbage collected."""
+
+    def __init__(self, handle, layout, in_shape, max_batch):
+        self.handle, self.layout, self.in_shape, self.max_batch = handle, layout, in_shape, max_batch
+        self.d, self.d_fact = int(layout.d), int(layout.d_fact)
+
+    def __del__(self):
+        h, self.handle = getattr(self, "handle", None), None
+        if h and _lib is not None:
+            _lib.iodf_destroy(h)
+
+
+def iodf_create(model, max_batch, device=0, marshalled=None):
+    L = load_library()
+    m = marshalled or _Marshalled(model, max_batch)
+    out = C.c_void_p()
+    rc = L.iodf_create(C.byref(m.desc), m.wts.ctypes.data, m.wts.size, m.par.ctypes.data, m.par.size, int(device),
+                       C.byref(out))
+    if rc != 0:
+        raise IodfError(rc, "iodf_create")
+    lay = Layout()
+    L.iodf_get_layout(out, C.byref(lay))
+    return Model(out, lay, (model["in_c"], model["in_h"], model["in_w"]), int(max_batch))
+
+
+def iodf_destroy(model):
+    h, model.handle = model.handle, None
+    if h:
+        load_library().iodf_destroy(h)
+
+
+def iodf_get_layout(model):
+    return model.layout
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    return C.c_void_p(int(stream))
+
+
+def _ptr(t):
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+def iodf_forward(model, x_u8, z=None, prior=None, stream=None, want_prior=True):
+    """x_u8: cuda uint8 [B,C,H,W]. Returns (z int32 [B,d], prior int32 [B,2,d_fact] | None)."""
+    import torch
+    B = x_u8.shape[0]
+    assert x_u8.is_cuda and x_u8.dtype == torch.uint8 and x_u8.is_contiguous()
+    if z is None:
+        z = torch.empty((B, model.d), dtype=torch.int32, device=x_u8.device)
+    if prior is None and want_prior and model.d_fact:
+        prior = torch.empty((B, 2, model.d_fact), dtype=torch.int32, device=x_u8.device)
+    rc = load_library().iodf_forward(model.handle, _ptr(x_u8), B, _ptr(z), _ptr(prior), _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_forward")
+    return z, prior
+
+
+def iodf_inverse(model, z, x_u8=None, prior=None, out_of_range=None, stream=None):
+    """z: cuda int32 [B,d]. Returns x_u8 uint8 [B,C,H,W]."""
+    import torch
+    B = z.shape[0]
+    assert z.is_cuda and z.dtype == torch.int32 and z.is_contiguous()
+    if x_u8 is None:
+        x_u8 = torch.empty((B,) + tuple(model.in_shape), dtype=torch.uint8, device=z.device)
+    rc = load_library().iodf_inverse(model.handle, _ptr(z), B, _ptr(x_u8), _ptr(prior), _ptr(out_of_range),
+                                     _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_inverse")
+    return x_u8
+
+
+def iodf_forward_host(model, x_u8, z, prior=None, stream=None):
+    """Host (ideally pinned) torch tensors in and out; results valid after the stream is synchronised."""
+    rc = load_library().iodf_forward_host(model.handle, _ptr(x_u8), x_u8.shape[0], _ptr(z), _ptr(prior),
+                                          _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_forward_host")
+
+
+def iodf_inverse_host(model, z, x_u8, stream=None):
+    rc = load_library().iodf_inverse_host(model.handle, _ptr(z), z.shape[0], _ptr(x_u8), _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_inverse_host")
+
+
+def iodf_check(model, stream=None):
+    rc = load_library().iodf_check(model.handle, _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_check")
+
+
+def iodf_launches_per_call(model, inverse=False):
+    return load_library().iodf_launches_per_call(model.handle, int(inverse))

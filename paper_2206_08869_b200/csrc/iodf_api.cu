@@ -1,0 +1,611 @@
+// Host side of the IODF library: descriptor validation, weight repacking into the tensor-core
+// operand layout, shared-memory planning per level, and the C entry points declared in iodf.h.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/iodf.h"
+#include "iodf_dev.h"
+#include "level_kernel.h"
+
+using namespace iodf;
+
+namespace {
+
+constexpr uint32_t kAlign = 128;
+
+inline uint32_t up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
+
+struct HostLevel {
+  LevelPlan plan;
+  std::vector<uint8_t> blob;
+  int grid_group = 1;
+};
+
+}  // namespace
+
+struct iodf_model {
+  int device = 0;
+  int last_cuda = 0;
+  uint32_t max_batch = 0;
+  uint32_t in_c = 0, in_h = 0, in_w = 0;
+  iodf_layout layout{};
+  std::vector<HostLevel> levels;
+  std::vector<LevelPlan*> d_plan;
+  std::vector<uint8_t*> d_blob;
+  std::vector<int32_t*> d_keep;     // kept channels between level l and l+1
+  uint32_t* d_status = nullptr;
+  // staging for the host-buffer entry points
+  uint8_t* d_x = nullptr;
+  int32_t* d_z = nullptr;
+  int32_t* d_prior = nullptr;
+};
+
+namespace {
+
+struct Blobs {
+  const int8_t* w;
+  size_t w_count;
+  const int32_t* r;
+  size_t r_count;
+};
+
+int check_layer(const iodf_layer_desc& L, const Blobs& B) {
+  if ((L.k != 1 && L.k != 3) || L.c_in < 1 || L.c_out < 1) return IODF_EINVAL;
+  const uint64_t wn = (uint64_t)L.c_out * L.k * L.k * L.c_in;
+  if (L.weight_off > B.w_count || wn > B.w_count - L.weight_off) return IODF_EINVAL;
+  if (L.requant_off > B.r_count || 3ull * L.c_out > B.r_count - L.requant_off) return IODF_EINVAL;
+  const int32_t* m0 = B.r + L.requant_off + L.c_out;
+  const int32_t* s = m0 + L.c_out;
+  for (uint32_t i = 0; i < L.c_out; ++i)
+    if (m0[i] < (1 << 30) || s[i] < 0 || s[i] > 31) return IODF_EINVAL;
+  if (L.has_clamp && L.clamp_lo > L.clamp_hi) return IODF_EINVAL;
+  return IODF_OK;
+}
+
+// Worst case |accumulator + bias| for inputs bounded by amax must fit int32.
+int check_overflow(const iodf_layer_desc& L, const Blobs& B, int64_t amax) {
+  const int8_t* w = B.w + L.weight_off;
+  const int32_t* bias = B.r + L.requant_off;
+  const size_t fan = (size_t)L.k * L.k * L.c_in;
+  for (uint32_t o = 0; o < L.c_out; ++o) {
+    int64_t sum = 0;
+    for (size_t i = 0; i < fan; ++i) sum += std::abs((int)w[o * fan + i]);
+    const int64_t worst = sum * amax + std::llabs((long long)bias[o]);
+    if (worst > 0x7FFFFFFFll) return IODF_EOVERFLOW;
+  }
+  return IODF_OK;
+}
+
+struct Act { int lo, hi; };
+
+// Effective range of a hidden layer's output; must be inside the signed 8-bit range.
+int hidden_range(const iodf_layer_desc& L, Act* out) {
+  if (!L.has_clamp) return IODF_EUNSUPPORTED;
+  int lo = L.clamp_lo, hi = L.clamp_hi;
+  if (L.relu) lo = std::max(lo, 0);
+  if (lo > hi) { lo = hi; }
+  if (lo < -128 || hi > 127) return IODF_EUNSUPPORTED;
+  out->lo = lo;
+  out->hi = hi;
+  return IODF_OK;
+}
+
+void put_hidden_rq(HiddenRq* dst, const iodf_layer_desc& L, const Blobs& B, int n_pad, int* fast) {
+  const int32_t* bias = B.r + L.requant_off;
+  const int32_t* m0 = bias + L.c_out;
+  const int32_t* s = m0 + L.c_out;
+  *fast = 1;
+  for (int i = 0; i < n_pad; ++i) {
+    HiddenRq h;
+    if (i < (int)L.c_out) {
+      const long long c64 = (long long)bias[i] * (long long)m0[i] + (1ll << (30 + s[i]));
+      h.m0 = m0[i];
+      h.sh = s[i] - 1;
+      h.c_lo = (uint32_t)((unsigned long long)c64 & 0xFFFFFFFFull);
+      h.c_hi = (uint32_t)((unsigned long long)c64 >> 32);
+      if (s[i] < 1) *fast = 0;
+    } else {  // padding channel: acc = 0 -> 0
+      h.m0 = 1 << 30;
+      h.sh = 0;
+      h.c_lo = 0x80000000u;
+      h.c_hi = 0;
+    }
+    dst[i] = h;
+  }
+}
+
+void put_out_rq(OutRq* dst, const iodf_layer_desc& L, const Blobs& B) {
+  const int32_t* bias = B.r + L.requant_off;
+  const int32_t* m0 = bias + L.c_out;
+  const int32_t* s = m0 + L.c_out;
+  for (uint32_t i = 0; i < L.c_out; ++i) dst[i] = OutRq{bias[i], m0[i], s[i], 0};
+}
+
+// Weight matrix [n_pad rows][kd bytes], K-major, no swizzle: byte (n, k) at (k/16)*n_pad*16 + n*16 + k%16.
+inline size_t wpos(int n_pad, int n, int k) { return (size_t)(k >> 4) * n_pad * 16 + (size_t)n * 16 + (k & 15); }
+
+struct PackedBlock {
+  std::vector<uint8_t> meta, w[3];
+};
+
+void append_block(std::vector<uint8_t>& blob, const PackedBlock& pb, BlockRef* ref) {
+  auto add = [&](const std::vector<uint8_t>& part, uint32_t* off, uint32_t* bytes) {
+    blob.resize(up((uint32_t)blob.size(), kAlign), 0);
+    *off = (uint32_t)blob.size();
+    *bytes = (uint32_t)part.size();
+    blob.insert(blob.end(), part.begin(), part.end());
+  };
+  add(pb.meta, &ref->meta_off, &ref->meta_bytes);
+  for (int i = 0; i < 3; ++i) add(pb.w[i], &ref->w_off[i], &ref->w_bytes[i]);
+  blob.resize(up((uint32_t)blob.size(), kAlign), 0);
+}
+
+struct Dims { int n1, n2, n3, kd1, kd2, kd3; };
+
+PackedBlock pack_coupling(const iodf_coupling_desc& cp, const Blobs& B, int ca, int cb, const int* colA,
+                          const int* colB, Act a1, Act a2, Dims* dims) {
+  const iodf_layer_desc& L1 = cp.layers[0];
+  const iodf_layer_desc& L2 = cp.layers[1];
+  const iodf_layer_desc& L3 = cp.layers[2];
+  const int k1 = (int)L1.c_out, k2 = (int)L2.c_out;
+  Dims d;
+  d.n1 = (int)up(k1, 16); d.n2 = (int)up(k2, 16); d.n3 = (int)up(9 * cb, 16);
+  d.kd1 = (int)up(9 * ca, 32); d.kd2 = (int)up(k1, 32); d.kd3 = (int)up(k2, 32);
+  *dims = d;
+  PackedBlock pb;
+  CouplingMeta M{};
+  M.in_m0 = cp.in_m0; M.in_s = cp.in_s;
+  M.n1 = d.n1; M.n2 = d.n2; M.kd1 = d.kd1; M.kd2 = d.kd2; M.kd3 = d.kd3; M.n3 = d.n3;
+  M.lo1 = a1.lo; M.hi1 = a1.hi; M.lo2 = a2.lo; M.hi2 = a2.hi;
+  uint32_t off = sizeof(CouplingMeta);
+  M.off_colA = (int)off; off += up(4 * ca, 16);
+  M.off_colB = (int)off; off += up(4 * cb, 16);
+  M.off_out = (int)off;  off += (uint32_t)sizeof(OutRq) * cb;
+  M.off_h1 = (int)off;   off += (uint32_t)sizeof(HiddenRq) * d.n1;
+  M.off_h2 = (int)off;   off += (uint32_t)sizeof(HiddenRq) * d.n2;
+  pb.meta.assign(off, 0);
+  std::memcpy(pb.meta.data() + M.off_colA, colA, 4 * ca);
+  std::memcpy(pb.meta.data() + M.off_colB, colB, 4 * cb);
+  put_out_rq(reinterpret_cast<OutRq*>(pb.meta.data() + M.off_out), L3, B);
+  put_hidden_rq(reinterpret_cast<HiddenRq*>(pb.meta.data() + M.off_h1), L1, B, d.n1, &M.fast1);
+  put_hidden_rq(reinterpret_cast<HiddenRq*>(pb.meta.data() + M.off_h2), L2, B, d.n2, &M.fast2);
+  std::memcpy(pb.meta.data(), &M, sizeof(M));
+
+  // W1: row = hidden channel, K index = tap*ca + c (the OHWI inner order)
+  pb.w[0].assign((size_t)d.n1 * d.kd1, 0);
+  const int8_t* w1 = B.w + L1.weight_off;
+  for (int n = 0; n < k1; ++n)
+    for (int k = 0; k < 9 * ca; ++k) pb.w[0][wpos(d.n1, n, k)] = (uint8_t)w1[(size_t)n * 9 * ca + k];
+  // W2: 1x1
+  pb.w[1].assign((size_t)d.n2 * d.kd2, 0);
+  const int8_t* w2 = B.w + L2.weight_off;
+  for (int n = 0; n < k2; ++n)
+    for (int k = 0; k < k1; ++k) pb.w[1][wpos(d.n2, n, k)] = (uint8_t)w2[(size_t)n * k1 + k];
+  // W3': row = tap*cb + c, K index = hidden channel
+  pb.w[2].assign((size_t)d.n3 * d.kd3, 0);
+  const int8_t* w3 = B.w + L3.weight_off;
+  for (int c = 0; c < cb; ++c)
+    for (int tap = 0; tap < 9; ++tap)
+      for (int k = 0; k < k2; ++k)
+        pb.w[2][wpos(d.n3, tap * cb + c, k)] = (uint8_t)w3[((size_t)c * 9 + tap) * k2 + k];
+  return pb;
+}
+
+PackedBlock pack_prior(const iodf_level_desc& lv, const Blobs& B, int ca, int cb, int* n_out, int* kd_out) {
+  const iodf_layer_desc& L = lv.prior_layer;
+  PackedBlock pb;
+  PriorMeta M{};
+  M.in_m0 = lv.prior_in_m0; M.in_s = lv.prior_in_s;
+  M.n = (int)up(2 * cb, 16);
+  M.kd = (int)up(9 * ca, 32);
+  M.ls_lo = lv.ls_lo; M.ls_hi = lv.ls_hi;
+  M.off_out = (int)sizeof(PriorMeta);
+  pb.meta.assign(sizeof(PriorMeta) + sizeof(OutRq) * 2 * cb, 0);
+  put_out_rq(reinterpret_cast<OutRq*>(pb.meta.data() + M.off_out), L, B);
+  std::memcpy(pb.meta.data(), &M, sizeof(M));
+  pb.w[0].assign((size_t)M.n * M.kd, 0);
+  const int8_t* w = B.w + L.weight_off;
+  for (int o = 0; o < 2 * cb; ++o)
+    for (int k = 0; k < 9 * ca; ++k) pb.w[0][wpos(M.n, o, k)] = (uint8_t)w[(size_t)o * 9 * ca + k];
+  *n_out = M.n;
+  *kd_out = M.kd;
+  return pb;
+}
+
+uint32_t pow2_cols(uint32_t need) {
+  uint32_t c = 32;
+  while (c < need) c <<= 1;
+  return c;
+}
+
+// Choose images per CTA and the shared-memory layout. Returns false if nothing fits.
+bool plan_smem(LevelPlan& P, uint32_t a13_bytes, uint32_t a2_bytes, uint32_t meta_bytes, const uint32_t wmax[3],
+               uint32_t limit, uint32_t max_batch) {
+  int group = P.px >= kTileM ? 1 : kTileM / P.px;
+  group = std::max(1, std::min<int>(group, (int)max_batch));
+  for (; group >= 1; group = (group > 1 ? group / 2 : 0)) {
+    for (int mode = 0; mode < 3; ++mode) {   // 0: nothing shared, 1: W1/W3 share, 2: also A2 inside A1/A3
+      const uint32_t pg = up((uint32_t)group * P.px, 32);
+      uint32_t off = 0;
+      auto take = [&](uint32_t bytes) { uint32_t o = off; off = up(off + bytes, kAlign); return o; };
+      P.s_v = take((uint32_t)P.c * pg * 4);
+      P.s_xa = take((uint32_t)P.ca * pg);
+      P.s_acc = take((uint32_t)P.cb * pg * 4);
+      const uint32_t a_all = std::max(a13_bytes, a2_bytes);
+      P.s_a13 = take(mode == 2 ? a_all : a13_bytes);
+      P.s_a2 = mode == 2 ? P.s_a13 : take(a2_bytes);
+      P.s_meta = take(meta_bytes);
+      P.s_w[0] = take(mode >= 1 ? std::max(wmax[0], wmax[2]) : wmax[0]);
+      P.s_w[1] = take(wmax[1]);
+      P.s_w[2] = mode >= 1 ? P.s_w[0] : take(wmax[2]);
+      P.s_total = off;
+      P.w13_alias = mode >= 1;
+      P.group = group;
+      P.pg = (int)pg;
+      P.tiles = (int)((group * P.px + kTileM - 1) / kTileM);
+      if (off <= limit) return true;
+    }
+    if (group == 1) break;
+  }
+  return false;
+}
+
+int cuda_fail(iodf_model* m, cudaError_t e) {
+  if (m) m->last_cuda = (int)e;
+  return e == cudaErrorMemoryAllocation ? IODF_ENOMEM : IODF_ECUDA;
+}
+
+#define CU(m, x)                                   \
+  do {                                             \
+    cudaError_t e__ = (x);                         \
+    if (e__ != cudaSuccess) return cuda_fail(m, e__); \
+  } while (0)
+
+int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_model* m) {
+  if (desc->abi_version != IODF_ABI_VERSION) return IODF_EVERSION;
+  if (!desc->levels || desc->n_levels < 1 || desc->n_levels > IODF_MAX_LEVELS || desc->max_batch < 1 ||
+      desc->in_c < 1 || desc->in_h < 1 || desc->in_w < 1)
+    return IODF_EINVAL;
+  if ((desc->in_h % (1u << desc->n_levels)) || (desc->in_w % (1u << desc->n_levels))) return IODF_EINVAL;
+  m->device = device;
+  m->max_batch = desc->max_batch;
+  m->in_c = desc->in_c; m->in_h = desc->in_h; m->in_w = desc->in_w;
+
+  int smem_limit = 0;
+  CU(m, cudaSetDevice(device));
+  CU(m, cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
+  smem_limit -= 1024;   // static control block and alignment slack
+
+  iodf_layout& lay = m->layout;
+  lay = iodf_layout{};
+  lay.n_levels = desc->n_levels;
+  lay.d = (uint64_t)desc->in_c * desc->in_h * desc->in_w;
+
+  // pass 1: shapes, validation, latent layout
+  uint32_t c = desc->in_c, h = desc->in_h, w = desc->in_w;
+  uint64_t zo = 0, po = 0;
+  for (uint32_t li = 0; li < desc->n_levels; ++li) {
+    const iodf_level_desc& lv = desc->levels[li];
+    c *= 4; h /= 2; w /= 2;
+    if (c % 2 || c > (uint32_t)kMaxC) return c % 2 ? IODF_EINVAL : IODF_EUNSUPPORTED;
+    if (lv.n_couplings > (uint32_t)kMaxCouplings) return IODF_EUNSUPPORTED;
+    if (lv.n_couplings && !lv.couplings) return IODF_EINVAL;
+    if (lv.has_prior && !lv.split) return IODF_EINVAL;
+    lay.level_c[li] = c; lay.level_h[li] = h; lay.level_w[li] = w;
+    lay.z_off[li] = zo; lay.prior_off[li] = po;
+    const uint32_t ca = c / 2, cb = c - ca, px = h * w;
+    for (uint32_t ki = 0; ki < lv.n_couplings; ++ki) {
+      const iodf_coupling_desc& cp = lv.couplings[ki];
+      if (!cp.perm || !cp.layers) return IODF_EINVAL;
+      std::vector<char> seen(c, 0);
+      for (uint32_t k = 0; k < c; ++k) {
+        if (cp.perm[k] < 0 || cp.perm[k] >= (int32_t)c || seen[cp.perm[k]]) return IODF_EINVAL;
+        seen[cp.perm[k]] = 1;
+      }
+      if (cp.in_m0 < (1 << 30) || cp.in_s < 0 || cp.in_s > 31) return IODF_EINVAL;
+      if (cp.n_layers < 1) return IODF_EINVAL;
+      uint32_t cin = ca;
+      for (uint32_t q = 0; q < cp.n_layers; ++q) {
+        int rc = check_layer(cp.layers[q], B);
+        if (rc) return rc;
+        if (cp.layers[q].c_in != cin) return IODF_EINVAL;
+        cin = cp.layers[q].c_out;
+      }
+      if (cin != cb) return IODF_EINVAL;
+      const iodf_layer_desc& last = cp.layers[cp.n_layers - 1];
+      if (last.relu || last.has_clamp) return IODF_EINVAL;
+      // the shape this build runs
+      if (cp.n_layers != 3 || cp.layers[0].k != 3 || cp.layers[1].k != 1 || cp.layers[2].k != 3)
+        return IODF_EUNSUPPORTED;
+      if (cp.layers[0].c_out > (uint32_t)kMaxHidden || cp.layers[1].c_out > (uint32_t)kMaxHidden)
+        return IODF_EUNSUPPORTED;
+      Act a1, a2;
+      int rc = hidden_range(cp.layers[0], &a1);
+      if (rc) return rc;
+      rc = hidden_range(cp.layers[1], &a2);
+      if (rc) return rc;
+      if ((rc = check_overflow(cp.layers[0], B, 128))) return rc;
+      if ((rc = check_overflow(cp.layers[1], B, std::max(std::abs(a1.lo), std::abs(a1.hi))))) return rc;
+      if ((rc = check_overflow(cp.layers[2], B, std::max(std::abs(a2.lo), std::abs(a2.hi))))) return rc;
+      for (uint32_t q = 0; q < cp.n_layers; ++q)
+        lay.macs_per_image += (uint64_t)px * cp.layers[q].k * cp.layers[q].k * cp.layers[q].c_in * cp.layers[q].c_out;
+    }
+    if (lv.has_prior) {
+      const iodf_layer_desc& L = lv.prior_layer;
+      int rc = check_layer(L, B);
+      if (rc) return rc;
+      if (L.c_in != ca || L.c_out != 2 * cb) return IODF_EINVAL;
+      if (lv.prior_in_m0 < (1 << 30) || lv.prior_in_s < 0 || lv.prior_in_s > 31 || lv.ls_lo > lv.ls_hi)
+        return IODF_EINVAL;
+      if (L.k != 3 || L.relu || L.has_clamp) return IODF_EUNSUPPORTED;
+      if ((rc = check_overflow(L, B, 128))) return rc;
+      lay.macs_per_image += (uint64_t)px * 9 * L.c_in * L.c_out;
+    }
+    if (lv.split) {
+      zo += (uint64_t)cb * px;
+      if (lv.has_prior) po += (uint64_t)cb * px;
+      c = ca;
+    }
+  }
+  lay.z_final_off = zo;
+  lay.d_fact = po;
+  if (zo + (uint64_t)c * h * w != lay.d) return IODF_EINVAL;
+
+  // pass 2: pack and plan
+  m->levels.resize(desc->n_levels);
+  c = desc->in_c; h = desc->in_h; w = desc->in_w;
+  uint32_t max_smem = 0;
+  for (uint32_t li = 0; li < desc->n_levels; ++li) {
+    const iodf_level_desc& lv = desc->levels[li];
+    HostLevel& hl = m->levels[li];
+    LevelPlan& P = hl.plan;
+    std::memset(&P, 0, sizeof(P));
+    c *= 4; h /= 2; w /= 2;
+    const int ca = (int)c / 2, cb = (int)c - ca;
+    P.c = (int)c; P.h = (int)h; P.w = (int)w; P.px = (int)(h * w); P.ca = ca; P.cb = cb;
+    P.n_couplings = (int)lv.n_couplings;
+    P.split = lv.split ? 1 : 0; P.has_prior = lv.has_prior ? 1 : 0;
+    P.is_first = li == 0; P.is_last = li + 1 == desc->n_levels;
+    P.keep_c = lv.split ? ca : (int)c;
+    P.z_off = lay.z_off[li]; P.prior_off = lay.prior_off[li]; P.z_final_off = lay.z_final_off;
+    P.d = lay.d; P.d_fact = lay.d_fact;
+
+    std::vector<int> pi(c);
+    for (uint32_t k = 0; k < c; ++k) pi[k] = (int)k;
+    uint32_t a13 = 0, a2 = 0, meta = 0, wmax[3] = {0, 0, 0};
+    uint32_t n1max = 0, need_cols = 32;
+    std::vector<Dims> dims(lv.n_couplings);
+    std::vector<PackedBlock> blocks;
+    for (uint32_t ki = 0; ki < lv.n_couplings; ++ki) {
+      const iodf_coupling_desc& cp = lv.couplings[ki];
+      std::vector<int> nxt(c);
+      for (uint32_t k = 0; k < c; ++k) nxt[k] = pi[cp.perm[k]];
+      pi.swap(nxt);
+      Act a1, a2r;
+      hidden_range(cp.layers[0], &a1);
+      hidden_range(cp.layers[1], &a2r);
+      blocks.push_back(pack_coupling(cp, B, ca, cb, pi.data(), pi.data() + ca, a1, a2r, &dims[ki]));
+      const Dims& d = dims[ki];
+      a13 = std::max<uint32_t>(a13, kTileM * std::max(d.kd1, d.kd3));
+      a2 = std::max<uint32_t>(a2, kTileM * d.kd2);
+      n1max = std::max<uint32_t>(n1max, d.n1);
+    }
+    P.d2_col = (int)up(n1max, 32);
+    for (uint32_t ki = 0; ki < lv.n_couplings; ++ki) {
+      const Dims& d = dims[ki];
+      need_cols = std::max<uint32_t>(need_cols, std::max<uint32_t>(P.d2_col + d.n2, d.n3));
+    }
+    for (int k = 0; k < (int)c; ++k) P.col_out[k] = pi[k];
+    PackedBlock prior_block;
+    if (lv.has_prior) {
+      int n, kd;
+      prior_block = pack_prior(lv, B, ca, cb, &n, &kd);
+      a13 = std::max<uint32_t>(a13, kTileM * kd);
+      need_cols = std::max<uint32_t>(need_cols, n);
+    }
+    if (need_cols > 512) return IODF_EUNSUPPORTED;
+    P.tmem_cols = (int)pow2_cols(need_cols);
+    for (uint32_t ki = 0; ki < lv.n_couplings; ++ki) {
+      append_block(hl.blob, blocks[ki], &P.coupling[ki]);
+      meta = std::max(meta, P.coupling[ki].meta_bytes);
+      for (int i = 0; i < 3; ++i) wmax[i] = std::max(wmax[i], P.coupling[ki].w_bytes[i]);
+    }
+    if (lv.has_prior) {
+      append_block(hl.blob, prior_block, &P.prior);
+      meta = std::max(meta, P.prior.meta_bytes);
+      wmax[0] = std::max(wmax[0], P.prior.w_bytes[0]);
+    }
+    if (hl.blob.empty()) hl.blob.resize(kAlign, 0);
+    if (!plan_smem(P, std::max(a13, 16u), std::max(a2, 16u), std::max(meta, 16u), wmax, (uint32_t)smem_limit,
+                   desc->max_batch))
+      return IODF_EUNSUPPORTED;
+    max_smem = std::max(max_smem, P.s_total);
+    if (lv.split) c = (uint32_t)ca;
+  }
+
+  // device objects
+  CU(m, configure_level_kernels(max_smem));
+  const size_t L = desc->n_levels;
+  m->d_plan.assign(L, nullptr); m->d_blob.assign(L, nullptr); m->d_keep.assign(L, nullptr);
+  for (size_t li = 0; li < L; ++li) {
+    HostLevel& hl = m->levels[li];
+    CU(m, cudaMalloc(&m->d_plan[li], sizeof(LevelPlan)));
+    CU(m, cudaMemcpy(m->d_plan[li], &hl.plan, sizeof(LevelPlan), cudaMemcpyHostToDevice));
+    CU(m, cudaMalloc(&m->d_blob[li], hl.blob.size()));
+    CU(m, cudaMemcpy(m->d_blob[li], hl.blob.data(), hl.blob.size(), cudaMemcpyHostToDevice));
+    if (li + 1 < L)
+      CU(m, cudaMalloc(&m->d_keep[li], (size_t)desc->max_batch * hl.plan.keep_c * hl.plan.px * sizeof(int32_t)));
+  }
+  CU(m, cudaMalloc(&m->d_status, sizeof(uint32_t)));
+  CU(m, cudaMemset(m->d_status, 0, sizeof(uint32_t)));
+  CU(m, cudaMalloc(&m->d_x, (size_t)desc->max_batch * lay.d));
+  CU(m, cudaMalloc(&m->d_z, (size_t)desc->max_batch * lay.d * sizeof(int32_t)));
+  if (lay.d_fact) CU(m, cudaMalloc(&m->d_prior, (size_t)desc->max_batch * 2 * lay.d_fact * sizeof(int32_t)));
+  CU(m, cudaDeviceSynchronize());
+  return IODF_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int run_forward(iodf_model* m, const uint8_t* x, int B, int32_t* z, int32_t* prior, cudaStream_t st) {
+  const size_t L = m->levels.size();
+  for (size_t li = 0; li < L; ++li) {
+    const LevelPlan& P = m->levels[li].plan;
+    LevelArgs a{};
+    a.plan = m->d_plan[li];
+    a.blob = m->d_blob[li];
+    a.in = li == 0 ? (const void*)x : (const void*)m->d_keep[li - 1];
+    a.in_stride = 0;
+    a.z = z;
+    a.prior = prior;
+    a.out = m->d_keep[li];
+    a.oor = nullptr;
+    a.status = m->d_status;
+    a.batch = B;
+    CU(m, launch_level(a, false, (B + P.group - 1) / P.group, P.s_total, st));
+  }
+  return IODF_OK;
+}
+
+int run_inverse(iodf_model* m, const int32_t* z, int B, uint8_t* x, int32_t* prior, uint32_t* oor, cudaStream_t st) {
+  const int L = (int)m->levels.size();
+  for (int li = L - 1; li >= 0; --li) {
+    const LevelPlan& P = m->levels[li].plan;
+    LevelArgs a{};
+    a.plan = m->d_plan[li];
+    a.blob = m->d_blob[li];
+    if (li == L - 1) { a.in = z + m->layout.z_final_off; a.in_stride = (long long)m->layout.d; }
+    else { a.in = m->d_keep[li]; a.in_stride = (long long)P.keep_c * P.px; }
+    a.z = const_cast<int32_t*>(z);
+    a.prior = prior;
+    a.out = li == 0 ? (void*)x : (void*)m->d_keep[li - 1];
+    a.oor = oor;
+    a.status = m->d_status;
+    a.batch = B;
+    CU(m, launch_level(a, true, (B + P.group - 1) / P.group, P.s_total, st));
+  }
+  return IODF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int iodf_create(const iodf_model_desc* desc, const int8_t* weights, size_t weights_count, const int32_t* requant,
+                size_t requant_count, int device, iodf_model** out) {
+  if (!desc || !weights || !requant || !out) return IODF_EINVAL;
+  *out = nullptr;
+  iodf_model* m = new (std::nothrow) iodf_model();
+  if (!m) return IODF_ENOMEM;
+  int rc;
+  try {
+    Blobs B{weights, weights_count, requant, requant_count};
+    rc = build_model(desc, B, device, m);
+  } catch (const std::bad_alloc&) {
+    rc = IODF_ENOMEM;
+  }
+  if (rc != IODF_OK) {
+    iodf_destroy(m);
+    return rc;
+  }
+  *out = m;
+  return IODF_OK;
+}
+
+void iodf_destroy(iodf_model* m) {
+  if (!m) return;
+  cudaSetDevice(m->device);
+  for (auto p : m->d_plan) if (p) cudaFree(p);
+  for (auto p : m->d_blob) if (p) cudaFree(p);
+  for (auto p : m->d_keep) if (p) cudaFree(p);
+  if (m->d_status) cudaFree(m->d_status);
+  if (m->d_x) cudaFree(m->d_x);
+  if (m->d_z) cudaFree(m->d_z);
+  if (m->d_prior) cudaFree(m->d_prior);
+  delete m;
+}
+
+int iodf_get_layout(const iodf_model* m, iodf_layout* out) {
+  if (!m || !out) return IODF_EINVAL;
+  *out = m->layout;
+  return IODF_OK;
+}
+
+int iodf_forward(iodf_model* m, const uint8_t* x_u8, int B, int32_t* z, int32_t* prior, void* cuda_stream) {
+  if (!m || !x_u8 || !z || B < 1 || (uint32_t)B > m->max_batch) return IODF_EINVAL;
+  if (!aligned16(x_u8) || !aligned16(z) || !aligned16(prior)) return IODF_EINVAL;
+  return run_forward(m, x_u8, B, z, m->layout.d_fact ? prior : nullptr, (cudaStream_t)cuda_stream);
+}
+
+int iodf_inverse(iodf_model* m, const int32_t* z, int B, uint8_t* x_u8, int32_t* prior, uint32_t* out_of_range_count,
+                 void* cuda_stream) {
+  if (!m || !x_u8 || !z || B < 1 || (uint32_t)B > m->max_batch) return IODF_EINVAL;
+  if (!aligned16(x_u8) || !aligned16(z) || !aligned16(prior)) return IODF_EINVAL;
+  return run_inverse(m, z, B, x_u8, m->layout.d_fact ? prior : nullptr, out_of_range_count,
+                     (cudaStream_t)cuda_stream);
+}
+
+int iodf_forward_host(iodf_model* m, const uint8_t* x_u8_host, int B, int32_t* z_host, int32_t* prior_host,
+                      void* cuda_stream) {
+  if (!m || !x_u8_host || !z_host || B < 1 || (uint32_t)B > m->max_batch) return IODF_EINVAL;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t d = m->layout.d, df = m->layout.d_fact;
+  int32_t* prior = (prior_host && df) ? m->d_prior : nullptr;
+  CU(m, cudaMemcpyAsync(m->d_x, x_u8_host, (size_t)B * d, cudaMemcpyHostToDevice, st));
+  int rc = run_forward(m, m->d_x, B, m->d_z, prior, st);
+  if (rc) return rc;
+  CU(m, cudaMemcpyAsync(z_host, m->d_z, (size_t)B * d * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  if (prior) CU(m, cudaMemcpyAsync(prior_host, prior, (size_t)B * 2 * df * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  return IODF_OK;
+}
+
+int iodf_inverse_host(iodf_model* m, const int32_t* z_host, int B, uint8_t* x_u8_host, void* cuda_stream) {
+  if (!m || !x_u8_host || !z_host || B < 1 || (uint32_t)B > m->max_batch) return IODF_EINVAL;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t d = m->layout.d;
+  CU(m, cudaMemcpyAsync(m->d_z, z_host, (size_t)B * d * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  int rc = run_inverse(m, m->d_z, B, m->d_x, nullptr, nullptr, st);
+  if (rc) return rc;
+  CU(m, cudaMemcpyAsync(x_u8_host, m->d_x, (size_t)B * d, cudaMemcpyDeviceToHost, st));
+  return IODF_OK;
+}
+
+int iodf_check(iodf_model* m, void* cuda_stream) {
+  if (!m) return IODF_EINVAL;
+  uint32_t st = 0;
+  CU(m, cudaStreamSynchronize((cudaStream_t)cuda_stream));
+  CU(m, cudaMemcpy(&st, m->d_status, sizeof(st), cudaMemcpyDeviceToHost));
+  if (st) {
+    CU(m, cudaMemset(m->d_status, 0, sizeof(uint32_t)));
+    return IODF_ETIMEOUT;
+  }
+  return IODF_OK;
+}
+
+int iodf_launches_per_call(const iodf_model* m, int inverse) {
+  (void)inverse;
+  return m ? (int)m->levels.size() : 0;
+}
+
+const char* iodf_strerror(int status) {
+  switch (status) {
+    case IODF_OK: return "ok";
+    case IODF_EINVAL: return "invalid argument or malformed model descriptor";
+    case IODF_ENOMEM: return "out of memory";
+    case IODF_ECUDA: return "CUDA call failed";
+    case IODF_EVERSION: return "ABI version mismatch";
+    case IODF_ETIMEOUT: return "a bounded device-side wait gave up";
+    case IODF_EUNSUPPORTED: return "model shape not supported by this build";
+    case IODF_EOVERFLOW: return "worst-case accumulator leaves the int32 range";
+    default: return "unknown status";
+  }
+}
+
+int iodf_last_cuda_error(const iodf_model* m) { return m ? m->last_cuda : 0; }
+
+}  // extern "C"
