@@ -1,0 +1,247 @@
+#!/usr/bin/env python
+"""Throughput benchmark of the integer-flow encoder on B200.
+
+One step = one encode (all levels: squeeze, couplings, split, prior heads) of one batch of the
+ImageNet64-shaped pruned flow (batch 128 of uint8 3x64x64 synthetic smooth-field images, 4 levels
+x 8 couplings, hidden 256 with 30-60 % of the filters pruned). Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--config 2] [--batch B]
+
+With N > 1 (launched by torch.distributed.run) every rank encodes its own batch (weak scaling,
+no collective on the data path); the time is the maximum over ranks.
+`--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+import iodf_synth as S
+
+METRIC = "flow_encode_images_per_sec"
+UNIT = "images/s"
+N_SETS = 8   # rotating input/output sets: 8 x 19.7 MB > the 126 MB L2
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return d["hbm_gbs"], d["bf16_tflops"], "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.stop_flag, self.sm, self.reasons, self.max_sm = index, False, [], set(), None
+
+    def run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_sm = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                     nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                     nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                     nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap"}
+            while not self.stop_flag:
+                self.sm.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for bit, nm in names.items():
+                    if r & bit:
+                        self.reasons.add(nm)
+                time.sleep(0.01)
+        except Exception as e:  # NVML unavailable: report that instead of clocks
+            self.reasons.add("nvml_error:%s" % type(e).__name__)
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.max_sm,
+                "reasons": sorted(self.reasons), "samples": len(self.sm)}
+
+
+def oracle_rate(model, cfg, batch, cores):
+    """images/s of the CPU oracle on a bounded sample of the workload."""
+    import oracle as O
+    pk = O.Packed(model)
+    n = max(cores, 16)
+    x = S.config_images(cfg, batch=n)
+    t0 = time.perf_counter()
+    O.forward(pk, x, threads=cores)
+    dt = time.perf_counter() - t0
+    return n / dt, n, dt
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    cores = os.cpu_count() or 1
+    model = S.config_model(args.config)
+    rates = []
+    for i in range(args.warmup + args.steps):
+        r, n, dt = oracle_rate(model, args.config, args.batch, cores)
+        if i >= args.warmup:
+            rates.append((r, dt))
+    value = float(np.mean([r for r, _ in rates]))
+    sample = "%d images of the workload per step, oracle forward, %d threads" % (n, cores)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean([d for _, d in rates])),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": workload(args),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def workload(args):
+    c = S.CONFIGS[args.config]
+    return {"workload": "config %s: ImageNet%d-shaped pruned IODF encode, batch %d of uint8 3x%dx%d, %d levels x %d "
+                        "couplings, hidden %d" % (args.config, c["hw"], args.batch, c["hw"], c["hw"],
+                                                   len(c["splits"]), c["n_couplings"], c["hidden"]),
+            "batch_per_gpu": args.batch, "l2_policy": "rotating %d input/output sets (> L2)" % N_SETS,
+            "parallelism": "independent batches per GPU, no collective"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="b200")
+    ap.add_argument("--config", default="2")
+    ap.add_argument("--batch", type=int, default=None)
+    args = ap.parse_args()
+    args.config = int(args.config) if args.config.isdigit() else args.config
+    args.batch = args.batch or S.CONFIGS[args.config]["batch"]
+    args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2206_08869_b200 as G
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg, B = args.config, args.batch
+    model = S.config_model(cfg)
+    m = G.iodf_create(model, B, device=local_rank)
+    lay = m.layout
+    macs = int(lay.macs_per_image)
+
+    xs = [torch.from_numpy(S.config_images(cfg, batch=B, seed_offset=100 * rank + i)).to(dev) for i in range(N_SETS)]
+    zs = [torch.empty((B, m.d), dtype=torch.int32, device=dev) for _ in range(N_SETS)]
+    ps = [torch.empty((B, 2, m.d_fact), dtype=torch.int32, device=dev) for _ in range(N_SETS)]
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident throughput ----------------------------------------------------------
+    for i in range(args.warmup):
+        G.iodf_forward(m, xs[i % N_SETS], zs[i % N_SETS], ps[i % N_SETS])
+    G.iodf_check(m)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        G.iodf_forward(m, xs[i % N_SETS], zs[i % N_SETS], ps[i % N_SETS])
+    e1.record(stream)
+    barrier()
+    total_ms = e0.elapsed_time(e1)
+    sampler.stop_flag = True
+    sampler.join()
+    G.iodf_check(m)
+
+    # ---- dominant kernel, timed alone per launch with events on the same stream --------------
+    lvl = np.zeros(int(lay.n_levels))
+    reps = 50
+    for i in range(reps):
+        lvl += np.array(G.iodf_forward_timed(m, xs[i % N_SETS], zs[i % N_SETS], ps[i % N_SETS]))
+    lvl /= reps
+    top = int(np.argmax(lvl))
+    lv = model["levels"][top]
+    px = lv["h"] * lv["w"]
+    top_macs = sum(px * ly["k"] ** 2 * ly["c_in"] * ly["c_out"] for cp in lv["couplings"] for ly in cp["layers"])
+    if lv["prior"] is not None:
+        ly = lv["prior"]["layer"]
+        top_macs += px * 9 * ly["c_in"] * ly["c_out"]
+    hbm, bf16, which = peaks()
+    peak_int8 = 2.0 * bf16                      # dense int8 : bf16 = 2 : 1 nominal
+    achieved = 2.0 * top_macs * B / (lvl[top] * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "level_kernel<encode> level %d" % top, "achieved": achieved,
+                "peak": peak_int8, "unit": "TOP/s (int8)", "frac": achieved / peak_int8, "traffic": None,
+                "peak_source": "2 x %s burst bf16 %.1f TFLOP/s" % (which, bf16),
+                "level_ms": [float(v) for v in lvl],
+                "whole_step_frac": (2.0 * macs * B / (total_ms / args.steps * 1e-3) / 1e12) / peak_int8}
+
+    # ---- end to end through the host-buffer entry point --------------------------------------
+    hx = [torch.from_numpy(S.config_images(cfg, batch=B, seed_offset=100 * rank + i)).pin_memory() for i in range(2)]
+    hz = [torch.empty((B, m.d), dtype=torch.int32).pin_memory() for _ in range(2)]
+    hp = [torch.empty((B, 2, m.d_fact), dtype=torch.int32).pin_memory() for _ in range(2)]
+    e2e_steps = max(10, min(args.steps, 100))
+    for i in range(3):
+        G.iodf_forward_host(m, hx[i % 2], hz[i % 2], hp[i % 2])
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        G.iodf_forward_host(m, hx[i % 2], hz[i % 2], hp[i % 2])
+        stream.synchronize()      # the result is read on the host every step
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    G.iodf_check(m)
+
+    t = torch.tensor([total_ms, e2e_s], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_s = float(t[0]), float(t[1])
+
+    if rank == 0:
+        cores = os.cpu_count() or 1
+        out = {
+            "metric": METRIC, "value": B * world * args.steps / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+            "ms_per_sample": total_ms / args.steps / B,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": workload(args), "clocks": sampler.summary(), "roofline": roofline,
+            "e2e": {"value": B * world * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": B * m.d,
+                    "d2h_bytes_per_step": B * m.d * 4 + B * 2 * m.d_fact * 4, "steps": e2e_steps},
+            "gpu_launches": G.iodf_launches_per_call(m) * args.steps,
+            "gops_per_image": 2.0 * macs / 1e9,
+        }
+        if world == 1:
+            r, n, dt = oracle_rate(model, cfg, B, cores)
+            out["cpu_baseline"] = {"value": r, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                   "sample": "%d images of the same workload, oracle forward, %.1f s" % (n, dt)}
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -170,6 +170,17 @@ int iodf_inverse_host(iodf_model* m, const int32_t* z_host, int B, uint8_t* x_u8
  */
 int iodf_check(iodf_model* m, void* cuda_stream);
 
+/*
+ * Profiling variants: the same work as iodf_forward / iodf_inverse with a CUDA event recorded on
+ * `cuda_stream` before and after each level's kernel. They synchronise the stream before returning
+ * and write the device time of each level's kernel, in milliseconds, to level_ms[0 .. n_levels)
+ * (HOST; level 0 is the finest level in both directions).
+ */
+int iodf_forward_timed(iodf_model* m, const uint8_t* x_u8, int B, int32_t* z, int32_t* prior, void* cuda_stream,
+                       float* level_ms);
+int iodf_inverse_timed(iodf_model* m, const int32_t* z, int B, uint8_t* x_u8, int32_t* prior,
+                       uint32_t* out_of_range_count, void* cuda_stream, float* level_ms);
+
 /* Number of kernel launches one iodf_forward / iodf_inverse call enqueues. */
 int iodf_launches_per_call(const iodf_model* m, int inverse);
 

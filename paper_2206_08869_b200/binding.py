@@ -12,7 +12,7 @@ IODF_ABI_VERSION = 1
 IODF_MAX_LEVELS = 8
 
 DECLARED_SYMBOLS = ["iodf_create", "iodf_destroy", "iodf_get_layout", "iodf_forward", "iodf_inverse",
-                    "iodf_forward_host", "iodf_inverse_host", "iodf_check", "iodf_launches_per_call",
+                    "iodf_forward_host", "iodf_inverse_host", "iodf_forward_timed", "iodf_inverse_timed", "iodf_check", "iodf_launches_per_call",
                     "iodf_strerror", "iodf_last_cuda_error"]
 
 
@@ -80,6 +80,10 @@ def load_library(path=None):
     L.iodf_forward_host.argtypes = [vp, vp, C.c_int, vp, vp, vp]
     L.iodf_inverse_host.restype = C.c_int
     L.iodf_inverse_host.argtypes = [vp, vp, C.c_int, vp, vp]
+    L.iodf_forward_timed.restype = C.c_int
+    L.iodf_forward_timed.argtypes = [vp, vp, C.c_int, vp, vp, vp, C.POINTER(C.c_float)]
+    L.iodf_inverse_timed.restype = C.c_int
+    L.iodf_inverse_timed.argtypes = [vp, vp, C.c_int, vp, vp, vp, vp, C.POINTER(C.c_float)]
     L.iodf_check.restype = C.c_int
     L.iodf_check.argtypes = [vp, vp]
     L.iodf_launches_per_call.restype = C.c_int
@@ -233,6 +237,27 @@ def iodf_inverse_host(model, z, x_u8, stream=None):
     rc = load_library().iodf_inverse_host(model.handle, _ptr(z), z.shape[0], _ptr(x_u8), _stream(stream))
     if rc != 0:
         raise IodfError(rc, "iodf_inverse_host")
+
+
+def iodf_forward_timed(model, x_u8, z, prior=None, stream=None):
+    """Encode with per-level event timing; returns the list of per-level kernel times in ms."""
+    n = int(model.layout.n_levels)
+    ms = (C.c_float * n)()
+    rc = load_library().iodf_forward_timed(model.handle, _ptr(x_u8), x_u8.shape[0], _ptr(z), _ptr(prior),
+                                           _stream(stream), ms)
+    if rc != 0:
+        raise IodfError(rc, "iodf_forward_timed")
+    return list(ms)
+
+
+def iodf_inverse_timed(model, z, x_u8, prior=None, out_of_range=None, stream=None):
+    n = int(model.layout.n_levels)
+    ms = (C.c_float * n)()
+    rc = load_library().iodf_inverse_timed(model.handle, _ptr(z), z.shape[0], _ptr(x_u8), _ptr(prior),
+                                           _ptr(out_of_range), _stream(stream), ms)
+    if rc != 0:
+        raise IodfError(rc, "iodf_inverse_timed")
+    return list(ms)
 
 
 def iodf_check(model, stream=None):

@@ -39,6 +39,7 @@ struct iodf_model {
   std::vector<uint8_t*> d_blob;
   std::vector<int32_t*> d_keep;     // kept channels between level l and l+1
   uint32_t* d_status = nullptr;
+  std::vector<cudaEvent_t> ev;      // n_levels + 1 events for the timed entry points
   // staging for the host-buffer entry points
   uint8_t* d_x = nullptr;
   int32_t* d_z = nullptr;
@@ -276,11 +277,6 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
   m->max_batch = desc->max_batch;
   m->in_c = desc->in_c; m->in_h = desc->in_h; m->in_w = desc->in_w;
 
-  int smem_limit = 0;
-  CU(m, cudaSetDevice(device));
-  CU(m, cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
-  smem_limit -= 1024;   // static control block and alignment slack
-
   iodf_layout& lay = m->layout;
   lay = iodf_layout{};
   lay.n_levels = desc->n_levels;
@@ -355,6 +351,12 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
   lay.z_final_off = zo;
   lay.d_fact = po;
   if (zo + (uint64_t)c * h * w != lay.d) return IODF_EINVAL;
+
+  // Everything above is host-only, so a malformed descriptor is reported even without a device.
+  int smem_limit = 0;
+  CU(m, cudaSetDevice(device));
+  CU(m, cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
+  smem_limit -= 1024;   // static control block and alignment slack
 
   // pass 2: pack and plan
   m->levels.resize(desc->n_levels);
@@ -441,6 +443,8 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
     if (li + 1 < L)
       CU(m, cudaMalloc(&m->d_keep[li], (size_t)desc->max_batch * hl.plan.keep_c * hl.plan.px * sizeof(int32_t)));
   }
+  m->ev.assign(L + 1, nullptr);
+  for (size_t i = 0; i <= L; ++i) CU(m, cudaEventCreate(&m->ev[i]));
   CU(m, cudaMalloc(&m->d_status, sizeof(uint32_t)));
   CU(m, cudaMemset(m->d_status, 0, sizeof(uint32_t)));
   CU(m, cudaMalloc(&m->d_x, (size_t)desc->max_batch * lay.d));
@@ -452,8 +456,10 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int run_forward(iodf_model* m, const uint8_t* x, int B, int32_t* z, int32_t* prior, cudaStream_t st) {
+int run_forward(iodf_model* m, const uint8_t* x, int B, int32_t* z, int32_t* prior, cudaStream_t st,
+                bool timed = false) {
   const size_t L = m->levels.size();
+  if (timed) CU(m, cudaEventRecord(m->ev[0], st));
   for (size_t li = 0; li < L; ++li) {
     const LevelPlan& P = m->levels[li].plan;
     LevelArgs a{};
@@ -468,12 +474,15 @@ int run_forward(iodf_model* m, const uint8_t* x, int B, int32_t* z, int32_t* pri
     a.status = m->d_status;
     a.batch = B;
     CU(m, launch_level(a, false, (B + P.group - 1) / P.group, P.s_total, st));
+    if (timed) CU(m, cudaEventRecord(m->ev[li + 1], st));
   }
   return IODF_OK;
 }
 
-int run_inverse(iodf_model* m, const int32_t* z, int B, uint8_t* x, int32_t* prior, uint32_t* oor, cudaStream_t st) {
+int run_inverse(iodf_model* m, const int32_t* z, int B, uint8_t* x, int32_t* prior, uint32_t* oor, cudaStream_t st,
+                bool timed = false) {
   const int L = (int)m->levels.size();
+  if (timed) CU(m, cudaEventRecord(m->ev[L], st));
   for (int li = L - 1; li >= 0; --li) {
     const LevelPlan& P = m->levels[li].plan;
     LevelArgs a{};
@@ -488,6 +497,18 @@ int run_inverse(iodf_model* m, const int32_t* z, int B, uint8_t* x, int32_t* pri
     a.status = m->d_status;
     a.batch = B;
     CU(m, launch_level(a, true, (B + P.group - 1) / P.group, P.s_total, st));
+    if (timed) CU(m, cudaEventRecord(m->ev[li], st));
+  }
+  return IODF_OK;
+}
+
+// Level li ran between events li and li+1 (encode) or li+1 and li (decode).
+int read_level_times(iodf_model* m, cudaStream_t st, bool inverse, float* level_ms) {
+  CU(m, cudaStreamSynchronize(st));
+  const size_t L = m->levels.size();
+  for (size_t li = 0; li < L; ++li) {
+    if (inverse) CU(m, cudaEventElapsedTime(&level_ms[li], m->ev[li + 1], m->ev[li]));
+    else CU(m, cudaEventElapsedTime(&level_ms[li], m->ev[li], m->ev[li + 1]));
   }
   return IODF_OK;
 }
@@ -523,6 +544,7 @@ void iodf_destroy(iodf_model* m) {
   for (auto p : m->d_plan) if (p) cudaFree(p);
   for (auto p : m->d_blob) if (p) cudaFree(p);
   for (auto p : m->d_keep) if (p) cudaFree(p);
+  for (auto e : m->ev) if (e) cudaEventDestroy(e);
   if (m->d_status) cudaFree(m->d_status);
   if (m->d_x) cudaFree(m->d_x);
   if (m->d_z) cudaFree(m->d_z);
@@ -548,6 +570,25 @@ int iodf_inverse(iodf_model* m, const int32_t* z, int B, uint8_t* x_u8, int32_t*
   if (!aligned16(x_u8) || !aligned16(z) || !aligned16(prior)) return IODF_EINVAL;
   return run_inverse(m, z, B, x_u8, m->layout.d_fact ? prior : nullptr, out_of_range_count,
                      (cudaStream_t)cuda_stream);
+}
+
+int iodf_forward_timed(iodf_model* m, const uint8_t* x_u8, int B, int32_t* z, int32_t* prior, void* cuda_stream,
+                       float* level_ms) {
+  if (!m || !x_u8 || !z || !level_ms || B < 1 || (uint32_t)B > m->max_batch) return IODF_EINVAL;
+  if (!aligned16(x_u8) || !aligned16(z) || !aligned16(prior)) return IODF_EINVAL;
+  int rc = run_forward(m, x_u8, B, z, m->layout.d_fact ? prior : nullptr, (cudaStream_t)cuda_stream, true);
+  if (rc) return rc;
+  return read_level_times(m, (cudaStream_t)cuda_stream, false, level_ms);
+}
+
+int iodf_inverse_timed(iodf_model* m, const int32_t* z, int B, uint8_t* x_u8, int32_t* prior,
+                       uint32_t* out_of_range_count, void* cuda_stream, float* level_ms) {
+  if (!m || !x_u8 || !z || !level_ms || B < 1 || (uint32_t)B > m->max_batch) return IODF_EINVAL;
+  if (!aligned16(x_u8) || !aligned16(z) || !aligned16(prior)) return IODF_EINVAL;
+  int rc = run_inverse(m, z, B, x_u8, m->layout.d_fact ? prior : nullptr, out_of_range_count,
+                       (cudaStream_t)cuda_stream, true);
+  if (rc) return rc;
+  return read_level_times(m, (cudaStream_t)cuda_stream, true, level_ms);
 }
 
 int iodf_forward_host(iodf_model* m, const uint8_t* x_u8_host, int B, int32_t* z_host, int32_t* prior_host,

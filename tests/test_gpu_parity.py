@@ -1,0 +1,198 @@
+"""CUDA path vs CPU oracle, element by element, through the C ABI. Everything is integer, so the
+bar is bit-exact equality of z, the prior parameters and the reconstructed x."""
+import numpy as np
+import pytest
+
+import iodf_synth as S
+import oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def G():
+    import paper_2206_08869_b200 as g
+    g.load_library()
+    return g
+
+
+def _t(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _check_both_ways(G, model, x, max_batch=None, sample=None):
+    """Encode x on the GPU and compare with the oracle (all images, or the `sample` indices);
+    decode the oracle's z on the GPU and compare with x."""
+    import torch
+    B = x.shape[0]
+    pk = O.Packed(model)
+    idx = np.arange(B) if sample is None else np.asarray(sample)
+    z_ref, p_ref = O.forward(pk, x[idx])
+    m = G.iodf_create(model, max_batch or B)
+    z, p = G.iodf_forward(m, _t(x))
+    G.iodf_check(m)
+    zc = z.cpu().numpy()
+    np.testing.assert_array_equal(zc[idx], z_ref)
+    if p_ref is not None:
+        np.testing.assert_array_equal(p.cpu().numpy()[idx], p_ref)
+    # decode what the GPU encoded (full batch): exact round trip, and the same prior parameters
+    oor = torch.zeros(1, dtype=torch.int32, device="cuda")
+    p2 = torch.empty_like(p) if p is not None else None
+    xr = G.iodf_inverse(m, z, prior=p2, out_of_range=oor)
+    G.iodf_check(m)
+    np.testing.assert_array_equal(xr.cpu().numpy(), x)
+    assert int(oor.item()) == 0
+    if p is not None:
+        assert torch.equal(p, p2)
+    return m, zc
+
+
+# ---- small shapes: several tiles, ragged tails, odd widths ---------------------------------------
+@pytest.mark.parametrize("hw,splits,hidden,prune,batch", [
+    (8, [False], 16, None, 3),                   # 16 px per image: several images share one tile
+    (8, [True, True], 24, (0.4, 0.7), 5),        # ragged last group (5 images, 8 and 32 per CTA)
+    (16, [True, True, True], 40, (0.4, 0.7), 9), # three levels, odd kept widths
+    (12, [True, False], 20, (0.4, 0.7), 7),      # 36-px and 9-px levels: tiles straddle images
+    (4, [True], 8, None, 70),                    # 4-px level: 32 images per CTA, three CTAs
+    (32, [True, True], 64, (0.4, 0.7), 3),       # 256-px level: two tiles per image
+])
+def test_small_models_bit_exact(G, hw, splits, hidden, prune, batch):
+    model = S.make_model(100 + hw, 3, hw, hw, splits, 3, hidden, prune=prune)
+    x = S.smooth_field_images(200 + hw, batch, hw, hw, 1.5)
+    _check_both_ways(G, model, x)
+
+
+def test_adversarial_inputs_and_wraparound(G):
+    import torch
+    model = S.make_model(7, 3, 16, 16, [True, True], 4, 32, prune=(0.4, 0.7))
+    x = np.concatenate([np.zeros((1, 3, 16, 16), np.uint8), np.full((1, 3, 16, 16), 255, np.uint8),
+                        S.Stream(8, "u8").integers(0, 256, 2 * 3 * 256).astype(np.uint8).reshape(2, 3, 16, 16)])
+    m, _ = _check_both_ways(G, model, x)
+    # any int32 vector is a latent: decode must agree with the oracle, including values far outside 0..255
+    pk = O.Packed(model)
+    zr = S.Stream(9, "z").integers(-(1 << 31), 1 << 31, 4 * pk.d).astype(np.int32).reshape(4, pk.d)
+    xu_ref, xi_ref, p_ref, oor_ref = O.inverse(pk, zr)
+    oor = torch.zeros(1, dtype=torch.int32, device="cuda")
+    p = torch.empty((4, 2, pk.d_fact), dtype=torch.int32, device="cuda")
+    xu = G.iodf_inverse(m, _t(zr), prior=p, out_of_range=oor)
+    G.iodf_check(m)
+    np.testing.assert_array_equal(xu.cpu().numpy(), xu_ref)
+    np.testing.assert_array_equal(p.cpu().numpy(), p_ref)
+    assert int(oor.item()) == oor_ref and oor_ref > 0
+
+
+def test_zero_shift_layers_take_the_exact_path(G):
+    """s = 0 in a hidden layer (multiplier in [1/2, 1)) must match as well."""
+    model = S.make_model(17, 3, 8, 8, [True], 2, 12, prune=None)
+    for cp in model["levels"][0]["couplings"]:
+        cp["layers"][0]["s"][:] = 0
+        cp["layers"][1]["s"][::2] = 0
+        cp["in_s"] = 0
+    x = S.smooth_field_images(18, 4, 8, 8, 1.0)
+    _check_both_ways(G, model, x)
+
+
+def test_zero_bias_and_no_prior(G):
+    model = S.make_model(19, 3, 16, 16, [True, False], 2, 16, prune=None, prior=False, with_bias=False)
+    _check_both_ways(G, model, S.smooth_field_images(20, 4, 16, 16, 1.5))
+
+
+def test_batch_limits_and_argument_errors(G):
+    import torch
+    model = S.make_model(21, 3, 8, 8, [True], 1, 8, prune=None)
+    m = G.iodf_create(model, 4)
+    x = _t(S.smooth_field_images(22, 5, 8, 8, 1.0))
+    with pytest.raises(G.IodfError) as e:
+        G.iodf_forward(m, x)                     # batch 5 > max_batch 4
+    assert e.value.status == -1
+    z = torch.empty((4, m.d + 1), dtype=torch.int32, device="cuda").reshape(-1)[1:1 + 4 * m.d].reshape(4, m.d)
+    with pytest.raises(G.IodfError) as e:
+        G.iodf_forward(m, x[:4].contiguous(), z=z)   # z not 16-byte aligned
+    assert e.value.status == -1
+    z1, _ = G.iodf_forward(m, x[:1].contiguous())    # batch 1
+    z4, _ = G.iodf_forward(m, x[:4].contiguous())
+    G.iodf_check(m)
+    assert torch.equal(z1[0], z4[0])
+
+
+def test_repeat_runs_are_identical(G):
+    import torch
+    model = S.config_model(0)
+    m = G.iodf_create(model, 16)
+    x = _t(S.config_images(0))
+    z1, _ = G.iodf_forward(m, x)
+    z2, _ = G.iodf_forward(m, x)
+    G.iodf_check(m)
+    assert torch.equal(z1, z2)
+
+
+def test_host_buffer_entry_points(G):
+    import torch
+    model = S.make_model(23, 3, 16, 16, [True, True], 2, 24, prune=(0.4, 0.7))
+    x = S.smooth_field_images(24, 6, 16, 16, 1.5)
+    z_ref, p_ref = O.forward(O.Packed(model), x)
+    m = G.iodf_create(model, 8)
+    hx = torch.from_numpy(x).pin_memory()
+    hz = torch.empty((6, m.d), dtype=torch.int32).pin_memory()
+    hp = torch.empty((6, 2, m.d_fact), dtype=torch.int32).pin_memory()
+    G.iodf_forward_host(m, hx, hz, hp)
+    G.iodf_check(m)
+    np.testing.assert_array_equal(hz.numpy(), z_ref)
+    np.testing.assert_array_equal(hp.numpy(), p_ref)
+    hx2 = torch.empty_like(hx)
+    G.iodf_inverse_host(m, hz, hx2)
+    G.iodf_check(m)
+    np.testing.assert_array_equal(hx2.numpy(), x)
+
+
+# ---- the five benchmark configurations ------------------------------------------------------------
+def test_config0_tiny_flow(G):
+    _check_both_ways(G, S.config_model(0), S.config_images(0))
+
+
+def test_config1_imagenet32_encode_full_batch(G):
+    _check_both_ways(G, S.config_model(1), S.config_images(1))
+
+
+def test_config2_imagenet64_encode(G):
+    """Full batch of 128 in the launch configuration the benchmark times; the oracle checks a
+    sample (first, last, group boundaries, seeded random picks); the remaining images are covered
+    by the exact round trip and by batch independence."""
+    import torch
+    x = S.config_images(2)
+    B = x.shape[0]
+    pick = sorted(set([0, 1, B // 2 - 1, B // 2, B - 2, B - 1] + S.Stream(5, "pick").integers(0, B, 10).tolist()))
+    m, z = _check_both_ways(G, S.config_model(2), x, sample=pick)
+    z8, _ = G.iodf_forward(m, _t(x[40:48]))
+    G.iodf_check(m)
+    np.testing.assert_array_equal(z8.cpu().numpy(), z[40:48])
+
+
+def test_config3_decode_of_config1(G):
+    import torch
+    model, x = S.config_model(3), S.config_images(3)
+    pk = O.Packed(model)
+    z_ref, p_ref = O.forward(pk, x)
+    m = G.iodf_create(model, x.shape[0])
+    p = torch.empty((x.shape[0], 2, pk.d_fact), dtype=torch.int32, device="cuda")
+    xr = G.iodf_inverse(m, _t(z_ref), prior=p)
+    G.iodf_check(m)
+    np.testing.assert_array_equal(xr.cpu().numpy(), x)
+    np.testing.assert_array_equal(p.cpu().numpy(), p_ref)
+
+
+@pytest.mark.parametrize("batch", [1, 8, 64, 512, 2048])
+def test_config4_batch_sweep_pruned(G, batch):
+    """Encode and decode at each batch size. The oracle checks up to 12 sampled images; beyond
+    batch 64 the GPU result must also equal the concatenation of batch-64 runs."""
+    import torch
+    model = S.config_model(4)
+    x = S.config_images(4, batch=batch)
+    pick = sorted(set([0, batch - 1] + S.Stream(batch, "pick").integers(0, batch, 10).tolist()))
+    m, z = _check_both_ways(G, model, x, sample=pick)
+    if batch > 64:
+        for b0 in range(0, batch, 64):
+            z64, _ = G.iodf_forward(m, _t(x[b0:b0 + 64]))
+            np.testing.assert_array_equal(z64.cpu().numpy(), z[b0:b0 + 64])
+        G.iodf_check(m)
