@@ -180,7 +180,7 @@ def main():
 
     # ---- dominant kernel, timed alone per launch with events on the same stream --------------
     lvl = np.zeros(int(lay.n_levels))
-    reps = 50
+    reps = min(50, max(5, args.steps))
     for i in range(reps):
         lvl += np.array(G.iodf_forward_timed(m, xs[i % N_SETS], zs[i % N_SETS], ps[i % N_SETS]))
     lvl /= reps

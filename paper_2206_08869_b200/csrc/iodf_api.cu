@@ -154,9 +154,10 @@ PackedBlock pack_coupling(const iodf_coupling_desc& cp, const Blobs& B, int ca, 
   const iodf_layer_desc& L2 = cp.layers[1];
   const iodf_layer_desc& L3 = cp.layers[2];
   const int k1 = (int)L1.c_out, k2 = (int)L2.c_out;
+  const int cpad = (int)up(ca, 8), cbp = (int)up(cb, 8);
   Dims d;
-  d.n1 = (int)up(k1, 16); d.n2 = (int)up(k2, 16); d.n3 = (int)up(9 * cb, 16);
-  d.kd1 = (int)up(9 * ca, 32); d.kd2 = (int)up(k1, 32); d.kd3 = (int)up(k2, 32);
+  d.n1 = (int)up(k1, 16); d.n2 = (int)up(k2, 16); d.n3 = (int)up(9 * cbp, 16);
+  d.kd1 = (int)up(9 * cpad, 32); d.kd2 = (int)up(k1, 32); d.kd3 = (int)up(k2, 32);
   *dims = d;
   PackedBlock pb;
   CouplingMeta M{};
@@ -177,33 +178,36 @@ PackedBlock pack_coupling(const iodf_coupling_desc& cp, const Blobs& B, int ca, 
   put_hidden_rq(reinterpret_cast<HiddenRq*>(pb.meta.data() + M.off_h2), L2, B, d.n2, &M.fast2);
   std::memcpy(pb.meta.data(), &M, sizeof(M));
 
-  // W1: row = hidden channel, K index = tap*ca + c (the OHWI inner order)
+  // W1: row = hidden channel, K index = tap*cpad + c
   pb.w[0].assign((size_t)d.n1 * d.kd1, 0);
   const int8_t* w1 = B.w + L1.weight_off;
   for (int n = 0; n < k1; ++n)
-    for (int k = 0; k < 9 * ca; ++k) pb.w[0][wpos(d.n1, n, k)] = (uint8_t)w1[(size_t)n * 9 * ca + k];
+    for (int tap = 0; tap < 9; ++tap)
+      for (int c = 0; c < ca; ++c)
+        pb.w[0][wpos(d.n1, n, tap * cpad + c)] = (uint8_t)w1[((size_t)n * 9 + tap) * ca + c];
   // W2: 1x1
   pb.w[1].assign((size_t)d.n2 * d.kd2, 0);
   const int8_t* w2 = B.w + L2.weight_off;
   for (int n = 0; n < k2; ++n)
     for (int k = 0; k < k1; ++k) pb.w[1][wpos(d.n2, n, k)] = (uint8_t)w2[(size_t)n * k1 + k];
-  // W3': row = tap*cb + c, K index = hidden channel
+  // W3': row = tap*cbp + c, K index = hidden channel
   pb.w[2].assign((size_t)d.n3 * d.kd3, 0);
   const int8_t* w3 = B.w + L3.weight_off;
   for (int c = 0; c < cb; ++c)
     for (int tap = 0; tap < 9; ++tap)
       for (int k = 0; k < k2; ++k)
-        pb.w[2][wpos(d.n3, tap * cb + c, k)] = (uint8_t)w3[((size_t)c * 9 + tap) * k2 + k];
+        pb.w[2][wpos(d.n3, tap * cbp + c, k)] = (uint8_t)w3[((size_t)c * 9 + tap) * k2 + k];
   return pb;
 }
 
 PackedBlock pack_prior(const iodf_level_desc& lv, const Blobs& B, int ca, int cb, int* n_out, int* kd_out) {
   const iodf_layer_desc& L = lv.prior_layer;
+  const int cpad = (int)up(ca, 8);
   PackedBlock pb;
   PriorMeta M{};
   M.in_m0 = lv.prior_in_m0; M.in_s = lv.prior_in_s;
   M.n = (int)up(2 * cb, 16);
-  M.kd = (int)up(9 * ca, 32);
+  M.kd = (int)up(9 * cpad, 32);
   M.ls_lo = lv.ls_lo; M.ls_hi = lv.ls_hi;
   M.off_out = (int)sizeof(PriorMeta);
   pb.meta.assign(sizeof(PriorMeta) + sizeof(OutRq) * 2 * cb, 0);
@@ -212,7 +216,9 @@ PackedBlock pack_prior(const iodf_level_desc& lv, const Blobs& B, int ca, int cb
   pb.w[0].assign((size_t)M.n * M.kd, 0);
   const int8_t* w = B.w + L.weight_off;
   for (int o = 0; o < 2 * cb; ++o)
-    for (int k = 0; k < 9 * ca; ++k) pb.w[0][wpos(M.n, o, k)] = (uint8_t)w[(size_t)o * 9 * ca + k];
+    for (int tap = 0; tap < 9; ++tap)
+      for (int c = 0; c < ca; ++c)
+        pb.w[0][wpos(M.n, o, tap * cpad + c)] = (uint8_t)w[((size_t)o * 9 + tap) * ca + c];
   *n_out = M.n;
   *kd_out = M.kd;
   return pb;
@@ -224,31 +230,38 @@ uint32_t pow2_cols(uint32_t need) {
   return c;
 }
 
-// Choose images per CTA and the shared-memory layout. Returns false if nothing fits.
-bool plan_smem(LevelPlan& P, uint32_t a13_bytes, uint32_t a2_bytes, uint32_t meta_bytes, const uint32_t wmax[3],
+// Choose images per CTA, tiles in flight and the shared-memory layout. Returns false if nothing fits.
+//   mode 0: two tile slots, every weight matrix resident      (needs all N <= 256 and >= 2 tiles)
+//   mode 1: one tile slot, every weight matrix resident
+//   mode 2: one tile slot, W1 and W3 share a slot and are re-fetched per tile
+bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32_t wmax[3], uint32_t n_max,
                uint32_t limit, uint32_t max_batch) {
   int group = P.px >= kTileM ? 1 : kTileM / P.px;
   group = std::max(1, std::min<int>(group, (int)max_batch));
   for (; group >= 1; group = (group > 1 ? group / 2 : 0)) {
-    for (int mode = 0; mode < 3; ++mode) {   // 0: nothing shared, 1: W1/W3 share, 2: also A2 inside A1/A3
+    const int tiles = (group * P.px + kTileM - 1) / kTileM;
+    for (int mode = 0; mode < 3; ++mode) {
+      if (mode == 0 && (tiles < 2 || n_max > (uint32_t)kSlotCols)) continue;
       const uint32_t pg = up((uint32_t)group * P.px, 32);
       uint32_t off = 0;
       auto take = [&](uint32_t bytes) { uint32_t o = off; off = up(off + bytes, kAlign); return o; };
       P.s_v = take((uint32_t)P.c * pg * 4);
-      P.s_xa = take((uint32_t)P.ca * pg);
+      P.s_xa = take(pg * (uint32_t)P.cpad);
       P.s_acc = take((uint32_t)P.cb * pg * 4);
-      const uint32_t a_all = std::max(a13_bytes, a2_bytes);
-      P.s_a13 = take(mode == 2 ? a_all : a13_bytes);
-      P.s_a2 = mode == 2 ? P.s_a13 : take(a2_bytes);
-      P.s_meta = take(meta_bytes);
-      P.s_w[0] = take(mode >= 1 ? std::max(wmax[0], wmax[2]) : wmax[0]);
+      P.s_a[0] = take(a_bytes);
+      P.s_a[1] = mode == 0 ? take(a_bytes) : P.s_a[0];
+      P.s_meta[0] = take(meta_bytes);
+      P.s_meta[1] = take(meta_bytes);
+      P.s_w[0] = take(mode == 2 ? std::max(wmax[0], wmax[2]) : wmax[0]);
       P.s_w[1] = take(wmax[1]);
-      P.s_w[2] = mode >= 1 ? P.s_w[0] : take(wmax[2]);
+      P.s_w[2] = mode == 2 ? P.s_w[0] : take(wmax[2]);
       P.s_total = off;
-      P.w13_alias = mode >= 1;
+      P.w13_alias = mode == 2;
+      P.nslots = mode == 0 ? 2 : 1;
+      P.tmem_cols = (int)(mode == 0 ? 2 * kSlotCols : pow2_cols(n_max));
       P.group = group;
       P.pg = (int)pg;
-      P.tiles = (int)((group * P.px + kTileM - 1) / kTileM);
+      P.tiles = tiles;
       if (off <= limit) return true;
     }
     if (group == 1) break;
@@ -377,11 +390,11 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
     P.z_off = lay.z_off[li]; P.prior_off = lay.prior_off[li]; P.z_final_off = lay.z_final_off;
     P.d = lay.d; P.d_fact = lay.d_fact;
 
+    P.cpad = (int)up(ca, 8); P.cbp = (int)up(cb, 8);
     std::vector<int> pi(c);
     for (uint32_t k = 0; k < c; ++k) pi[k] = (int)k;
-    uint32_t a13 = 0, a2 = 0, meta = 0, wmax[3] = {0, 0, 0};
-    uint32_t n1max = 0, need_cols = 32;
-    std::vector<Dims> dims(lv.n_couplings);
+    uint32_t a_bytes = 16, meta = 16, wmax[3] = {16, 16, 16};
+    uint32_t n_max = 32;
     std::vector<PackedBlock> blocks;
     for (uint32_t ki = 0; ki < lv.n_couplings; ++ki) {
       const iodf_coupling_desc& cp = lv.couplings[ki];
@@ -391,27 +404,20 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
       Act a1, a2r;
       hidden_range(cp.layers[0], &a1);
       hidden_range(cp.layers[1], &a2r);
-      blocks.push_back(pack_coupling(cp, B, ca, cb, pi.data(), pi.data() + ca, a1, a2r, &dims[ki]));
-      const Dims& d = dims[ki];
-      a13 = std::max<uint32_t>(a13, kTileM * std::max(d.kd1, d.kd3));
-      a2 = std::max<uint32_t>(a2, kTileM * d.kd2);
-      n1max = std::max<uint32_t>(n1max, d.n1);
-    }
-    P.d2_col = (int)up(n1max, 32);
-    for (uint32_t ki = 0; ki < lv.n_couplings; ++ki) {
-      const Dims& d = dims[ki];
-      need_cols = std::max<uint32_t>(need_cols, std::max<uint32_t>(P.d2_col + d.n2, d.n3));
+      Dims d;
+      blocks.push_back(pack_coupling(cp, B, ca, cb, pi.data(), pi.data() + ca, a1, a2r, &d));
+      a_bytes = std::max<uint32_t>(a_bytes, kTileM * std::max(d.kd1, std::max(d.kd2, d.kd3)));
+      n_max = std::max<uint32_t>(n_max, std::max(d.n1, std::max(d.n2, d.n3)));
     }
     for (int k = 0; k < (int)c; ++k) P.col_out[k] = pi[k];
     PackedBlock prior_block;
     if (lv.has_prior) {
       int n, kd;
       prior_block = pack_prior(lv, B, ca, cb, &n, &kd);
-      a13 = std::max<uint32_t>(a13, kTileM * kd);
-      need_cols = std::max<uint32_t>(need_cols, n);
+      a_bytes = std::max<uint32_t>(a_bytes, kTileM * kd);
+      n_max = std::max<uint32_t>(n_max, n);
     }
-    if (need_cols > 512) return IODF_EUNSUPPORTED;
-    P.tmem_cols = (int)pow2_cols(need_cols);
+    if (n_max > 512) return IODF_EUNSUPPORTED;
     for (uint32_t ki = 0; ki < lv.n_couplings; ++ki) {
       append_block(hl.blob, blocks[ki], &P.coupling[ki]);
       meta = std::max(meta, P.coupling[ki].meta_bytes);
@@ -423,8 +429,7 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
       wmax[0] = std::max(wmax[0], P.prior.w_bytes[0]);
     }
     if (hl.blob.empty()) hl.blob.resize(kAlign, 0);
-    if (!plan_smem(P, std::max(a13, 16u), std::max(a2, 16u), std::max(meta, 16u), wmax, (uint32_t)smem_limit,
-                   desc->max_batch))
+    if (!plan_smem(P, a_bytes, meta, wmax, n_max, (uint32_t)smem_limit, desc->max_batch))
       return IODF_EUNSUPPORTED;
     max_smem = std::max(max_smem, P.s_total);
     if (lv.split) c = (uint32_t)ca;

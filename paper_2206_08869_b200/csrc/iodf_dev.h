@@ -9,17 +9,24 @@
 //     bytes; consecutive 8-row groups are 128 bytes apart (stride-dimension offset) and
 //     consecutive 16-byte K chunks are N*16 bytes apart (leading-dimension offset).
 //   * Activation tiles (128 pixels x K bytes) use the same scheme: [K/16][128][16 bytes].
+//   * K of a 3x3 conv over the coupling input is ordered tap-major with the channel count padded
+//     to 8 (k = tap*cpad + c), so every im2col granule is an aligned 8-byte copy. N of the last
+//     3x3 conv is one row per (tap, out channel) with the channel count padded to 8
+//     (n = tap*cbp + c), so every 8-column accumulator granule belongs to one tap.
 #pragma once
 #include <stdint.h>
 
 namespace iodf {
 
 constexpr int kTileM = 128;          // pixels per MMA tile (UMMA M)
-constexpr int kThreads = 256;        // threads per CTA: 8 warps, two per TMEM lane quarter
+constexpr int kWorkerWarps = 16;     // four per TMEM lane quarter
+constexpr int kWorkers = kWorkerWarps * 32;
+constexpr int kThreads = kWorkers + 32;   // + one control warp (bulk copies and MMA issue)
 constexpr int kMaxCouplings = 32;    // per level
 constexpr int kMaxC = 256;           // flow channels per level
 constexpr int kMaxHidden = 256;      // kept hidden channels per layer (padded)
-constexpr uint32_t kSpinLimit = 20000000u;
+constexpr int kSlotCols = 256;       // TMEM columns per tile slot when two tiles are in flight
+constexpr uint32_t kSpinLimit = 4000000u;
 
 // Per-hidden-channel constants of the fast requantisation path (16 bytes).
 //   y = hi32(acc * m0 + c64) >> sh,  c64 = bias * m0 + 2^(30+s),  sh = s - 1   (needs s >= 1)
@@ -35,13 +42,13 @@ struct OutRq {
 };
 
 // Meta part of a coupling block, followed in memory by
-//   colA[ca] colB[cb] (int32 physical column of each logical channel), OutRq[n_out],
+//   colA[ca] colB[cb] (int32 physical column of each logical channel), OutRq[cb],
 //   HiddenRq[n1], HiddenRq[n2]; every array 16-byte aligned.
 struct CouplingMeta {
   int32_t in_m0, in_s;
   int32_t n1, n2;                // hidden widths padded to 16 (MMA N)
   int32_t kd1, kd2, kd3;         // K bytes of the three GEMMs, padded to 32
-  int32_t n3;                    // 9*cb padded to 16 (per-tap partial outputs of the last conv)
+  int32_t n3;                    // 9*cbp padded to 16 (per-tap partial outputs of the last conv)
   int32_t lo1, hi1, lo2, hi2;    // effective activation clips (ReLU folded in)
   int32_t fast1, fast2;          // 1: every s >= 1 in that layer (fast path exact)
   int32_t off_colA, off_colB, off_out, off_h1, off_h2;   // byte offsets from the meta start
@@ -49,11 +56,11 @@ struct CouplingMeta {
 };
 static_assert(sizeof(CouplingMeta) == 128, "meta header is 128 bytes");
 
-// Meta part of a prior-head block, followed by OutRq[n_out] (n_out = 2*cb real channels).
+// Meta part of a prior-head block, followed by OutRq[2*cb].
 struct PriorMeta {
   int32_t in_m0, in_s;
   int32_t n;                     // 2*cb padded to 16
-  int32_t kd;                    // 9*ca padded to 32
+  int32_t kd;                    // 9*cpad padded to 32
   int32_t ls_lo, ls_hi;
   int32_t off_out;
   int32_t pad[25];
@@ -65,20 +72,22 @@ struct BlockRef {                // where a block's parts sit in the level blob 
   uint32_t w_off[3], w_bytes[3];
 };
 
-// Everything a level kernel needs; lives in global memory, read through the constant cache.
+// Everything a level kernel needs; lives in global memory.
 struct LevelPlan {
   int32_t c, h, w, px;           // level shape after the squeeze
   int32_t ca, cb;
+  int32_t cpad, cbp;             // ca, cb rounded up to 8
   int32_t group;                 // images per CTA
   int32_t pg;                    // pixel slots per CTA = group*px rounded up to 32
   int32_t tiles;                 // ceil(group*px / 128)
   int32_t n_couplings;
   int32_t split, has_prior, is_first, is_last;
   int32_t keep_c;                // channels that go on to the next level (c/2 if split else c)
-  int32_t tmem_cols, d2_col;     // TMEM allocation and the column where the second GEMM lands
+  int32_t nslots;                // tiles in flight per CTA: 1 or 2
+  int32_t tmem_cols;
   int32_t w13_alias;             // 1: W1 and W3 share a slot and are re-fetched per tile
   // shared-memory byte offsets
-  uint32_t s_v, s_xa, s_acc, s_a13, s_a2, s_meta, s_w[3], s_total;
+  uint32_t s_v, s_xa, s_acc, s_a[2], s_meta[2], s_w[3], s_total;
   // global layout
   uint64_t z_off, prior_off, z_final_off, d, d_fact;
   int32_t col_out[kMaxC];        // physical column of logical channel k after the last coupling

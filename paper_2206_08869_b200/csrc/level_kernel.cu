@@ -4,10 +4,10 @@
 // all couplings of the level, so global memory is touched only for the level's input, its outputs
 // and the packed weights (which stay in L2). Per coupling (Eq. 2, Sec. 3):
 //
-//   x_a -> int8 (input requant)                                     all threads, exact 64-bit rq
+//   x_a -> int8 (input requant)                                     workers, exact 64-bit rq
 //   per 128-pixel tile:
-//     A1 = im2col(x_a)            [128 x 9*ca]                      threads -> shared memory
-//     D1 = A1 * W1^T              tcgen05.mma kind::i8, int32 in TMEM
+//     A1 = im2col(x_a)            [128 x 9*cpad]                    workers -> shared memory
+//     D1 = A1 * W1^T              tcgen05.mma kind::i8, int32 in TMEM (control thread issues)
 //     A2 = clip(ReLU(rq(D1)))     TMEM -> registers -> shared memory (int8, MMA operand layout)
 //     D2 = A2 * W2^T ; A3 = clip(ReLU(rq(D2)))                      (the 1x1 conv)
 //     D3 = A3 * W3'^T             W3' has one row per (tap, out channel): the nine per-tap partial
@@ -23,6 +23,12 @@
 // Squeeze, channel permutation and split are index maps: v is loaded in squeeze order, each
 // coupling addresses v through its table of physical columns (the composition of all permutations
 // so far), and the level's outputs are written through the final table.
+//
+// Execution structure: 16 worker warps and one control warp. The workers form one or two groups;
+// each group owns a tile slot (an A-operand buffer in shared memory and a range of TMEM columns)
+// and walks its tiles through build -> epilogue 1 -> epilogue 2 -> scatter, handing the slot to
+// the control thread between stages through mbarriers. The control thread issues the bulk copies
+// of weights and the MMAs, so while one group requantises, the tensor core works for the other.
 #include "iodf_dev.h"
 #include "level_kernel.h"
 #include "ptx.cuh"
@@ -32,9 +38,11 @@ namespace iodf {
 namespace {
 
 struct __align__(16) Ctl {
-  uint64_t bar_meta;
-  uint64_t bar_w[3];
-  uint64_t bar_mma;
+  uint64_t a_ready[2];    // workers -> control: the slot's A operand is written (count = group threads)
+  uint64_t d_ready[2];    // tensor core -> workers: the slot's accumulator is complete
+  uint64_t w_full[3];     // bulk copy -> control: weight slot filled
+  uint64_t w_free[3];     // tensor core -> control: last MMA reading the weight slot is complete
+  uint64_t meta_full[2];  // bulk copy -> everyone: meta block of step (i & 1) has landed
   uint32_t tmem_base;
   uint32_t abort;
 };
@@ -43,15 +51,17 @@ struct Ctx {
   uint8_t* smem;
   Ctl* ctl;
   uint32_t* status;
-  int tid, warp, lane, wq, wh, row;
-  uint32_t tmem;       // TMEM base address (lane 0, first allocated column)
-  uint32_t tmem_row;   // the same with this warp's lane quarter in the lane field
+  int tid, warp, lane;
+  int wq;                 // TMEM lane quarter of this warp
+  int group, cs, ncs;     // tile slot, column-split index and count inside the group
+  int row;                // tile row (= TMEM lane) of this thread
+  uint32_t tmem_slot;     // TMEM address of the slot's first column, this warp's lane quarter
 };
 
 // Bounded wait on an mbarrier phase. After one wait in the CTA has given up, every later wait
 // returns at once, so a stuck CTA drains in bounded time, frees its TMEM and exits.
-__device__ __noinline__ bool wait_bar(const Ctx& cx, uint64_t* bar, uint32_t parity) {
-  volatile uint32_t* ab = &cx.ctl->abort;
+__device__ __noinline__ bool wait_bar(Ctl* ctl, uint32_t* status, uint64_t* bar, uint32_t parity) {
+  volatile uint32_t* ab = &ctl->abort;
   if (*ab) return false;
   const uint32_t b = ptx::smem_u32(bar);
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
@@ -59,9 +69,11 @@ __device__ __noinline__ bool wait_bar(const Ctx& cx, uint64_t* bar, uint32_t par
     if ((it & 255u) == 255u && *ab) return false;
   }
   *ab = 1;
-  atomicExch(cx.status, 1u);
+  atomicExch(status, 1u);
   return false;
 }
+
+__device__ __forceinline__ void worker_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); }
 
 __device__ __forceinline__ int32_t rq_exact(int32_t a, int32_t m0, int32_t s) {
   const long long p = (long long)a * (long long)m0 + (1ll << (30 + s));
@@ -70,14 +82,26 @@ __device__ __forceinline__ int32_t rq_exact(int32_t a, int32_t m0, int32_t s) {
 
 __device__ __forceinline__ int clampi(int v, int lo, int hi) { return min(max(v, lo), hi); }
 
-template <bool kFast>
+__device__ __forceinline__ int min_relu(int v, int hi) {
+  int r;
+  asm("min.relu.s32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(hi));
+  return r;
+}
+
+template <bool kFast, bool kLo0>
 __device__ __forceinline__ int rq_hidden(int acc, const HiddenRq r, int lo, int hi) {
   const long long c64 = (long long)(((unsigned long long)r.c_hi << 32) | (unsigned long long)r.c_lo);
   const long long p = (long long)acc * (long long)r.m0 + c64;
   int y;
   if (kFast) y = ((int)(p >> 32)) >> r.sh;
   else y = (int)(p >> (32 + r.sh));
-  return clampi(y, lo, hi);
+  return kLo0 ? min_relu(y, hi) : clampi(y, lo, hi);
+}
+
+__device__ __forceinline__ uint32_t pack4(int y0, int y1, int y2, int y3) {
+  const uint32_t a = __byte_perm((uint32_t)y0, (uint32_t)y1, 0x0040);
+  const uint32_t b = __byte_perm((uint32_t)y2, (uint32_t)y3, 0x0040);
+  return __byte_perm(a, b, 0x5410);
 }
 
 // Pixel bookkeeping of one tile row.
@@ -110,30 +134,146 @@ __device__ __forceinline__ RowPos row_pos(int tile, int row, int pvalid, int px,
   return r;
 }
 
-// A[row][tap*ca + c] = xa[c][p + tap offset] (0 outside the image or beyond 9*ca), written as
-// 16-byte chunks into the MMA operand layout [K/16][128][16].
-__device__ void build_im2col(const Ctx& cx, uint8_t* sA, const int8_t* xa, int ca, int pg, int w, int kd,
-                             const RowPos rp) {
+__device__ __forceinline__ int tap_offset(int tap, int w) {
+  const int u = (tap * 11) >> 5;            // tap / 3 for 0..8
+  return (u - 1) * w + (tap - u * 3 - 1);
+}
+
+// A[row][tap*cpad + c] = xa[p + tap offset][c] (0 outside the image), as aligned 8-byte granules,
+// written in 16-byte chunks into the MMA operand layout [K/16][128][16].
+__device__ void build_im2col(const Ctx& cx, uint8_t* sA, const int8_t* xa, int cpad, int w, int kd, const RowPos rp) {
   const int nchunks = kd >> 4;
-  for (int jc = cx.wh; jc < nchunks; jc += kThreads / kTileM) {
-    int k = jc << 4;
-    int tap = k / ca;
-    int c = k - tap * ca;
-    uint32_t wd[4] = {0u, 0u, 0u, 0u};
+  const int gpt = cpad >> 3;                // granules per tap
+  const int ngran = 9 * gpt;
+  for (int jc = cx.cs; jc < nchunks; jc += cx.ncs) {
+    uint2 g2[2];
 #pragma unroll
-    for (int b = 0; b < 16; ++b) {
-      int val = 0;
-      if (tap < 9 && ((rp.gmask >> tap) & 1u)) {
-        const int du = tap / 3 - 1, dv = tap - (tap / 3) * 3 - 1;
-        val = xa[c * pg + rp.p + du * w + dv];
+    for (int half = 0; half < 2; ++half) {
+      const int g = 2 * jc + half;
+      g2[half] = make_uint2(0u, 0u);
+      if (g < ngran) {
+        const int tap = g / gpt, i = g - tap * gpt;
+        if ((rp.gmask >> tap) & 1u)
+          g2[half] = *reinterpret_cast<const uint2*>(xa + (size_t)(rp.p + tap_offset(tap, w)) * cpad + 8 * i);
       }
-      wd[b >> 2] |= (uint32_t)(val & 0xFF) << (8 * (b & 3));
-      if (++c == ca) { c = 0; ++tap; }
     }
-    *reinterpret_cast<uint4*>(sA + (size_t)jc * (kTileM * 16) + cx.row * 16) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+    *reinterpret_cast<uint4*>(sA + (size_t)jc * (kTileM * 16) + cx.row * 16) =
+        make_uint4(g2[0].x, g2[0].y, g2[1].x, g2[1].y);
   }
 }
 
+// 16 accumulator columns -> requantised bytes -> one 16-byte chunk of the next A operand.
+template <bool kFast, bool kLo0>
+__device__ __forceinline__ uint4 requant16(const uint32_t* r, const HiddenRq* rq, int lo, int hi) {
+  uint32_t wd[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int y0 = rq_hidden<kFast, kLo0>((int)r[4 * i + 0], rq[4 * i + 0], lo, hi);
+    const int y1 = rq_hidden<kFast, kLo0>((int)r[4 * i + 1], rq[4 * i + 1], lo, hi);
+    const int y2 = rq_hidden<kFast, kLo0>((int)r[4 * i + 2], rq[4 * i + 2], lo, hi);
+    const int y3 = rq_hidden<kFast, kLo0>((int)r[4 * i + 3], rq[4 * i + 3], lo, hi);
+    wd[i] = pack4(y0, y1, y2, y3);
+  }
+  return make_uint4(wd[0], wd[1], wd[2], wd[3]);
+}
+
+// TMEM accumulator -> requantised int8 activations in the next GEMM's A layout. n is a multiple
+// of 16; kd (the next GEMM's K) is n rounded up to 32, the extra chunk being zero.
+template <bool kFast, bool kLo0>
+__device__ void epilogue_hidden_t(const Ctx& cx, int n, int kd, const HiddenRq* rq, int lo, int hi, uint8_t* sOut) {
+  const int nblk = (n + 31) >> 5;
+  for (int b = cx.cs; b < nblk; b += cx.ncs) {
+    const int c0 = b << 5;
+    uint8_t* dst = sOut + (size_t)(2 * b) * (kTileM * 16) + cx.row * 16;
+    if (n - c0 >= 32) {
+      uint32_t r[32];
+      ptx::tmem_ld32(cx.tmem_slot + (uint32_t)c0, r);
+      ptx::tmem_ld_wait();
+      *reinterpret_cast<uint4*>(dst) = requant16<kFast, kLo0>(r, rq + c0, lo, hi);
+      *reinterpret_cast<uint4*>(dst + kTileM * 16) = requant16<kFast, kLo0>(r + 16, rq + c0 + 16, lo, hi);
+    } else {
+      uint32_t r[16];
+      ptx::tmem_ld16(cx.tmem_slot + (uint32_t)c0, r);
+      ptx::tmem_ld_wait();
+      *reinterpret_cast<uint4*>(dst) = requant16<kFast, kLo0>(r, rq + c0, lo, hi);
+      if (c0 + 16 < kd) *reinterpret_cast<uint4*>(dst + kTileM * 16) = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+}
+
+__device__ void epilogue_hidden(const Ctx& cx, int fast, int n, int kd, const HiddenRq* rq, int lo, int hi,
+                                uint8_t* sOut) {
+  if (fast) {
+    if (lo == 0) epilogue_hidden_t<true, true>(cx, n, kd, rq, lo, hi, sOut);
+    else epilogue_hidden_t<true, false>(cx, n, kd, rq, lo, hi, sOut);
+  } else {
+    epilogue_hidden_t<false, false>(cx, n, kd, rq, lo, hi, sOut);
+  }
+}
+
+// Per-tap partial products -> shifted sum into the translation accumulator. Column granule gi
+// (8 columns) belongs to tap gi / (cbp/8) and out channels (gi % (cbp/8))*8 .. +8.
+__device__ void epilogue_scatter(const Ctx& cx, int cb, int cbp, int32_t* acc, int pg, int w, const RowPos rp) {
+  const int gpt = cbp >> 3;
+  const int ngran = 9 * gpt;
+  for (int gi = cx.cs; gi < ngran; gi += cx.ncs) {
+    uint32_t r[8];
+    ptx::tmem_ld8(cx.tmem_slot + (uint32_t)(gi << 3), r);
+    ptx::tmem_ld_wait();
+    const int tap = gi / gpt;
+    const int c0 = (gi - tap * gpt) << 3;
+    if (rp.valid && ((rp.smask >> tap) & 1u)) {
+      int32_t* dst = acc + c0 * pg + rp.p - tap_offset(tap, w);
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (c0 + i < cb) atomicAdd(dst + i * pg, (int32_t)r[i]);
+    }
+  }
+}
+
+// Prior head accumulator -> (mu, log-scale index) in global memory.
+__device__ void epilogue_prior(const Ctx& cx, const LevelPlan& P, const LevelArgs& a, const PriorMeta& M,
+                               const OutRq* orq, int img0, const RowPos rp) {
+  const int cb = P.cb, px = P.px;
+  const int g = rp.valid ? rp.p / px : 0;
+  const int q = rp.p - g * px;
+  int32_t* mu = a.prior + (size_t)(img0 + g) * 2u * P.d_fact + P.prior_off + q;
+  int32_t* ls = mu + P.d_fact;
+  const int ngran = (2 * cb + 7) >> 3;
+  for (int gi = cx.cs; gi < ngran; gi += cx.ncs) {
+    uint32_t r[8];
+    ptx::tmem_ld8(cx.tmem_slot + (uint32_t)(gi << 3), r);
+    ptx::tmem_ld_wait();
+    if (rp.valid) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int col = (gi << 3) + i;
+        if (col < 2 * cb) {
+          const OutRq o = orq[col];
+          const int32_t y = rq_exact((int32_t)r[i] + o.bias, o.m0, o.s);
+          if (col < cb) mu[(size_t)col * px] = y;
+          else ls[(size_t)(col - cb) * px] = clampi(y, M.ls_lo, M.ls_hi);
+        }
+      }
+    }
+  }
+}
+
+// ---- step bookkeeping shared by workers and control -------------------------------------------
+struct Steps {
+  int n_couplings, nsteps;
+  bool do_prior, inverse;
+  __device__ bool is_prior(int i) const { return do_prior && (inverse ? i == 0 : i == nsteps - 1); }
+  __device__ int coupling_index(int i) const {
+    return inverse ? (n_couplings - 1 - (i - (do_prior ? 1 : 0))) : i;
+  }
+};
+
+__device__ __forceinline__ const BlockRef& step_ref(const LevelPlan& P, const Steps& st, int i) {
+  return st.is_prior(i) ? P.prior : P.coupling[st.coupling_index(i)];
+}
+
+// ---- control thread ---------------------------------------------------------------------------
 // D[128 x n] (+)= A[128 x kd] * B[n x kd]^T for B rows n0..n0+n of a matrix with n_total rows.
 __device__ void issue_gemm(uint32_t d_tmem, uint32_t sa, uint32_t sb, int n_total, int n0, int n, int kd) {
   const uint32_t idesc = ptx::umma_idesc_s8((uint32_t)n);
@@ -145,253 +285,279 @@ __device__ void issue_gemm(uint32_t d_tmem, uint32_t sa, uint32_t sb, int n_tota
   }
 }
 
-// TMEM accumulator -> requantised int8 activations in the next GEMM's A layout.
-template <bool kFast>
-__device__ void epilogue_hidden(const Ctx& cx, uint32_t taddr, int n, int kd, const HiddenRq* rq, int lo, int hi,
-                                uint8_t* sOut) {
-  const int nblk = (n + 31) >> 5;
-  for (int b = cx.wh; b < nblk; b += kThreads / kTileM) {
-    const int c0 = b << 5;
-    uint32_t r[32];
-    if (n - c0 >= 32) {
-      ptx::tmem_ld32(taddr + (uint32_t)c0, r);
-    } else {
-      uint32_t t[16];
-      ptx::tmem_ld16(taddr + (uint32_t)c0, t);
-#pragma unroll
-      for (int i = 0; i < 16; ++i) { r[i] = t[i]; r[16 + i] = 0u; }
-    }
-    ptx::tmem_ld_wait();
-    uint32_t wd[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) wd[i] = 0u;
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      int y = 0;
-      if (c0 + i < n) y = rq_hidden<kFast>((int)r[i], rq[c0 + i], lo, hi);
-      wd[i >> 2] |= (uint32_t)(y & 0xFF) << (8 * (i & 3));
-    }
-    uint8_t* dst = sOut + (size_t)(2 * b) * (kTileM * 16) + cx.row * 16;
-    *reinterpret_cast<uint4*>(dst) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
-    if (c0 + 16 < kd) *reinterpret_cast<uint4*>(dst + kTileM * 16) = make_uint4(wd[4], wd[5], wd[6], wd[7]);
-  }
-}
+struct WSlot {
+  uint32_t full_par, free_par;
+  int uses_left, cur_uses;
+  bool inflight, need_free, exhausted;
+  int g_step, g_sub;      // position of the load-sequence generator
+};
 
-// Per-tap partial products -> shifted sum into the translation accumulator.
-__device__ void epilogue_scatter(const Ctx& cx, uint32_t taddr, int n3, int cb, int32_t* acc, int pg, int w,
-                                 const RowPos rp) {
-  const int nblk = n3 >> 4;
-  for (int b = cx.wh; b < nblk; b += kThreads / kTileM) {
-    uint32_t r[16];
-    ptx::tmem_ld16(taddr + (uint32_t)(b << 4), r);
-    ptx::tmem_ld_wait();
-    if (rp.valid) {
-      int col = b << 4;
-      int tap = col / cb;
-      int c = col - tap * cb;
-#pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        if (tap < 9 && ((rp.smask >> tap) & 1u)) {
-          const int du = tap / 3 - 1, dv = tap - (tap / 3) * 3 - 1;
-          atomicAdd(&acc[c * pg + rp.p - du * w - dv], (int32_t)r[i]);
+struct Control {
+  const LevelPlan& P;
+  const LevelArgs& a;
+  uint8_t* smem;
+  Ctl* ctl;
+  Steps st;
+  int ntv;                // valid tiles of this CTA
+  bool alias;
+  WSlot ws[3];
+
+  __device__ bool wait(uint64_t* bar, uint32_t par) { return wait_bar(ctl, a.status, bar, par); }
+
+  __device__ void bulk(uint32_t off, uint32_t bytes, uint32_t s_dst, uint64_t* bar) {
+    const uint32_t b = ptx::smem_u32(bar);
+    ptx::mbar_expect_tx(b, bytes);
+    ptx::bulk_g2s(ptx::smem_u32(smem + s_dst), a.blob + off, bytes, b);
+  }
+
+  // Next matrix that weight slot s will hold, in the fixed order the MMAs consume them.
+  __device__ bool next_load(int s, uint32_t* off, uint32_t* bytes, int* uses) {
+    WSlot& w = ws[s];
+    for (;;) {
+      if (w.g_step >= st.nsteps) return false;
+      const BlockRef& br = step_ref(P, st, w.g_step);
+      if (st.is_prior(w.g_step)) {
+        if (s != 0 || w.g_sub > 0) { ++w.g_step; w.g_sub = 0; continue; }
+        *off = br.w_off[0]; *bytes = br.w_bytes[0]; *uses = ntv; w.g_sub = 1;
+        return true;
+      }
+      if (alias && s == 0) {                      // W1, W3, W1, W3, ... once per tile
+        if (w.g_sub >= 2 * ntv) { ++w.g_step; w.g_sub = 0; continue; }
+        const int which = (w.g_sub & 1) ? 2 : 0;
+        *off = br.w_off[which]; *bytes = br.w_bytes[which]; *uses = 1; ++w.g_sub;
+        return true;
+      }
+      if (alias && s == 2) return false;
+      if (w.g_sub > 0) { ++w.g_step; w.g_sub = 0; continue; }
+      *off = br.w_off[s]; *bytes = br.w_bytes[s]; *uses = ntv; w.g_sub = 1;
+      return true;
+    }
+  }
+
+  __device__ void issue_next(int s) {
+    uint32_t off, bytes;
+    int uses;
+    if (!next_load(s, &off, &bytes, &uses)) { ws[s].exhausted = true; return; }
+    bulk(off, bytes, P.s_w[s], &ctl->w_full[s]);
+    ws[s].inflight = true;
+    ws[s].cur_uses = uses;
+  }
+
+  __device__ void try_prefetch(int s) {
+    WSlot& w = ws[s];
+    if (w.uses_left != 0 || w.inflight || w.exhausted) return;
+    if (w.need_free) {
+      if (!ptx::mbar_try_wait(ptx::smem_u32(&ctl->w_free[s]), w.free_par)) return;
+      w.free_par ^= 1u;
+      w.need_free = false;
+    }
+    issue_next(s);
+  }
+
+  __device__ void acquire(int s) {
+    WSlot& w = ws[s];
+    if (w.uses_left != 0) return;
+    if (!w.inflight) {
+      if (w.need_free) { wait(&ctl->w_free[s], w.free_par); w.free_par ^= 1u; w.need_free = false; }
+      issue_next(s);
+    }
+    wait(&ctl->w_full[s], w.full_par);
+    w.full_par ^= 1u;
+    w.uses_left = w.cur_uses;
+    w.inflight = false;
+  }
+
+  __device__ void release(int s) {
+    WSlot& w = ws[s];
+    if (--w.uses_left == 0) {
+      ptx::umma_commit(ptx::smem_u32(&ctl->w_free[s]));
+      w.need_free = true;
+    }
+  }
+
+  __device__ void run(uint32_t tmem) {
+    for (int s = 0; s < 3; ++s) {
+      ws[s].full_par = ws[s].free_par = 0;
+      ws[s].uses_left = ws[s].cur_uses = 0;
+      ws[s].inflight = ws[s].need_free = ws[s].exhausted = false;
+      ws[s].g_step = ws[s].g_sub = 0;
+    }
+    for (int i = 0; i < st.nsteps && i < 2; ++i) {
+      const BlockRef& br = step_ref(P, st, i);
+      bulk(br.meta_off, br.meta_bytes, P.s_meta[i], &ctl->meta_full[i]);
+    }
+    for (int s = 0; s < 3; ++s) try_prefetch(s);
+
+    uint32_t apar[2] = {0u, 0u};
+    const int nslots = P.nslots;
+    for (int i = 0; i < st.nsteps; ++i) {
+      if (!wait(&ctl->meta_full[i & 1], (uint32_t)((i >> 1) & 1))) return;
+      const uint8_t* mb = smem + P.s_meta[i & 1];
+      const bool prior = st.is_prior(i);
+      int n[3], kd[3];
+      if (prior) {
+        const PriorMeta* M = reinterpret_cast<const PriorMeta*>(mb);
+        n[0] = M->n; kd[0] = M->kd;
+        n[1] = n[2] = kd[1] = kd[2] = 0;
+      } else {
+        const CouplingMeta* M = reinterpret_cast<const CouplingMeta*>(mb);
+        n[0] = M->n1; n[1] = M->n2; n[2] = M->n3;
+        kd[0] = M->kd1; kd[1] = M->kd2; kd[2] = M->kd3;
+      }
+      const int nstages = prior ? 1 : 3;
+      int tcur[2] = {0, 1}, stg[2] = {0, 0};
+      int remaining = ntv * nstages;
+      bool first = true;
+      uint32_t spin = 0;
+      while (remaining > 0) {
+        bool progress = false;
+        for (int s = 0; s < nslots; ++s) {
+          if (tcur[s] >= ntv) continue;
+          if (!ptx::mbar_try_wait(ptx::smem_u32(&ctl->a_ready[s]), apar[s])) continue;
+          apar[s] ^= 1u;
+          ptx::tc_fence_after();
+          if (first) {
+            // every worker has left step i-1, so its meta slot can take step i+1
+            first = false;
+            if (i >= 1 && i + 1 < st.nsteps) {
+              const BlockRef& br = step_ref(P, st, i + 1);
+              bulk(br.meta_off, br.meta_bytes, P.s_meta[(i + 1) & 1], &ctl->meta_full[(i + 1) & 1]);
+            }
+          }
+          const int stage = stg[s];
+          const int phys = prior ? 0 : ((stage == 2 && alias) ? 0 : stage);
+          acquire(phys);
+          const uint32_t d = tmem + (uint32_t)(s * kSlotCols);
+          const uint32_t sa = ptx::smem_u32(smem + P.s_a[s]);
+          const uint32_t sb = ptx::smem_u32(smem + P.s_w[phys]);
+          for (int n0 = 0; n0 < n[stage]; n0 += 256)
+            issue_gemm(d + (uint32_t)n0, sa, sb, n[stage], n0, min(256, n[stage] - n0), kd[stage]);
+          ptx::umma_commit(ptx::smem_u32(&ctl->d_ready[s]));
+          release(phys);
+          if (++stg[s] == nstages) { stg[s] = 0; tcur[s] += nslots; }
+          --remaining;
+          progress = true;
         }
-        if (++c == cb) { c = 0; ++tap; }
+        for (int s = 0; s < 3; ++s) try_prefetch(s);
+        if (progress) spin = 0;
+        else if (++spin > kSpinLimit || ctl->abort) {
+          if (!ctl->abort) { ctl->abort = 1; atomicExch(a.status, 1u); }
+          return;
+        }
       }
     }
   }
-}
-
-struct WeightState {   // thread 0 only
-  uint32_t ph[3];
 };
 
-__device__ __forceinline__ void load_part(const Ctx& cx, const uint8_t* blob, uint32_t off, uint32_t bytes,
-                                          uint32_t s_dst, uint64_t* bar) {
-  const uint32_t b = ptx::smem_u32(bar);
-  ptx::mbar_expect_tx(b, bytes);
-  ptx::bulk_g2s(ptx::smem_u32(cx.smem + s_dst), blob + off, bytes, b);
-}
-
-// One additive coupling over all tiles of the CTA. sign = +1 encodes, -1 decodes.
+// ---- workers ----------------------------------------------------------------------------------
 template <bool kInv>
-__device__ void run_coupling(const Ctx& cx, const LevelPlan& P, const LevelArgs& a, const BlockRef& br, int pvalid,
-                             uint32_t& ph_meta, uint32_t& ph_mma, WeightState& ws) {
+__device__ void run_workers(Ctx& cx, const LevelPlan& P, const LevelArgs& a, const Steps& st, int img0, int pvalid,
+                            int ntv) {
   uint8_t* smem = cx.smem;
+  Ctl* ctl = cx.ctl;
   int32_t* v = reinterpret_cast<int32_t*>(smem + P.s_v);
   int8_t* xa = reinterpret_cast<int8_t*>(smem + P.s_xa);
   int32_t* acc = reinterpret_cast<int32_t*>(smem + P.s_acc);
-  uint8_t* sA13 = smem + P.s_a13;
-  uint8_t* sA2 = smem + P.s_a2;
-  const int pg = P.pg, ca = P.ca, cb = P.cb, w = P.w, h = P.h, px = P.px;
-  const bool alias = P.w13_alias != 0;
+  uint8_t* sA = smem + P.s_a[cx.group];
+  const int pg = P.pg, ca = P.ca, cb = P.cb, w = P.w, h = P.h, px = P.px, cpad = P.cpad, cbp = P.cbp;
+  const int gthreads = (kWorkers / P.nslots);
+  uint64_t* a_ready = &ctl->a_ready[cx.group];
+  uint64_t* d_ready = &ctl->d_ready[cx.group];
+  uint32_t dpar = 0;
+  const CouplingMeta* prevM = nullptr;       // coupling whose translation is still to be applied
 
-  if (cx.tid == 0) {
-    load_part(cx, a.blob, br.meta_off, br.meta_bytes, P.s_meta, &cx.ctl->bar_meta);
-    load_part(cx, a.blob, br.w_off[0], br.w_bytes[0], P.s_w[0], &cx.ctl->bar_w[0]);
-    load_part(cx, a.blob, br.w_off[1], br.w_bytes[1], P.s_w[1], &cx.ctl->bar_w[1]);
-    if (!alias) load_part(cx, a.blob, br.w_off[2], br.w_bytes[2], P.s_w[2], &cx.ctl->bar_w[2]);
-  }
-  wait_bar(cx, &cx.ctl->bar_meta, ph_meta);
-  ph_meta ^= 1u;
-  const uint8_t* mb = smem + P.s_meta;
-  const CouplingMeta M = *reinterpret_cast<const CouplingMeta*>(mb);
-  const int32_t* colA = reinterpret_cast<const int32_t*>(mb + M.off_colA);
-  const int32_t* colB = reinterpret_cast<const int32_t*>(mb + M.off_colB);
-  const OutRq* orq = reinterpret_cast<const OutRq*>(mb + M.off_out);
-  const HiddenRq* h1 = reinterpret_cast<const HiddenRq*>(mb + M.off_h1);
-  const HiddenRq* h2 = reinterpret_cast<const HiddenRq*>(mb + M.off_h2);
-
-  // network input: x_a requantised to int8
-  for (int idx = cx.tid; idx < ca * pg; idx += kThreads) {
-    const int c = idx / pg, p = idx - c * pg;
-    int y = 0;
-    if (p < pvalid) y = clampi(rq_exact(v[colA[c] * pg + p], M.in_m0, M.in_s), -128, 127);
-    xa[idx] = (int8_t)y;
-  }
-  __syncthreads();
-
-  bool w_ready[3] = {false, false, false};
-  for (int tile = 0; tile < P.tiles; ++tile) {
-    if (tile * kTileM >= pvalid) break;
-    const RowPos rp = row_pos(tile, cx.row, pvalid, px, h, w);
-
-    // conv 3x3: ca -> n1
-    build_im2col(cx, sA13, xa, ca, pg, w, M.kd1, rp);
-    ptx::fence_async_smem();
-    __syncthreads();
-    if (cx.tid == 0) {
-      if (!w_ready[0] || alias) { wait_bar(cx, &cx.ctl->bar_w[0], ws.ph[0]); ws.ph[0] ^= 1u; w_ready[0] = true; }
-      ptx::tc_fence_after();
-      issue_gemm(cx.tmem, ptx::smem_u32(sA13), ptx::smem_u32(smem + P.s_w[0]), M.n1, 0, M.n1, M.kd1);
-      ptx::umma_commit(ptx::smem_u32(&cx.ctl->bar_mma));
-    }
-    wait_bar(cx, &cx.ctl->bar_mma, ph_mma);
-    ph_mma ^= 1u;
-    ptx::tc_fence_after();
-    if (alias && cx.tid == 0)
-      load_part(cx, a.blob, br.w_off[2], br.w_bytes[2], P.s_w[2], &cx.ctl->bar_w[2]);
-    if (M.fast1) epilogue_hidden<true>(cx, cx.tmem_row, M.n1, M.kd2, h1, M.lo1, M.hi1, sA2);
-    else epilogue_hidden<false>(cx, cx.tmem_row, M.n1, M.kd2, h1, M.lo1, M.hi1, sA2);
+  auto arrive_a = [&]() {
     ptx::tc_fence_before();
     ptx::fence_async_smem();
-    __syncthreads();
-
-    // conv 1x1: n1 -> n2
-    if (cx.tid == 0) {
-      if (!w_ready[1]) { wait_bar(cx, &cx.ctl->bar_w[1], ws.ph[1]); ws.ph[1] ^= 1u; w_ready[1] = true; }
-      ptx::tc_fence_after();
-      issue_gemm(cx.tmem + (uint32_t)P.d2_col, ptx::smem_u32(sA2), ptx::smem_u32(smem + P.s_w[1]), M.n2, 0, M.n2,
-                 M.kd2);
-      ptx::umma_commit(ptx::smem_u32(&cx.ctl->bar_mma));
-    }
-    wait_bar(cx, &cx.ctl->bar_mma, ph_mma);
-    ph_mma ^= 1u;
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ptx::smem_u32(a_ready)) : "memory");
+  };
+  auto wait_d = [&]() {
+    wait_bar(ctl, a.status, d_ready, dpar);
+    dpar ^= 1u;
     ptx::tc_fence_after();
-    if (M.fast2) epilogue_hidden<true>(cx, cx.tmem_row + (uint32_t)P.d2_col, M.n2, M.kd3, h2, M.lo2, M.hi2, sA13);
-    else epilogue_hidden<false>(cx, cx.tmem_row + (uint32_t)P.d2_col, M.n2, M.kd3, h2, M.lo2, M.hi2, sA13);
-    ptx::tc_fence_before();
-    ptx::fence_async_smem();
-    __syncthreads();
-
-    // conv 3x3: n2 -> cb, as nine per-tap partial products
-    if (cx.tid == 0) {
-      if (!w_ready[2] || alias) { wait_bar(cx, &cx.ctl->bar_w[2], ws.ph[2]); ws.ph[2] ^= 1u; w_ready[2] = true; }
-      ptx::tc_fence_after();
-      for (int n0 = 0; n0 < M.n3; n0 += 256)
-        issue_gemm(cx.tmem + (uint32_t)n0, ptx::smem_u32(sA13), ptx::smem_u32(smem + P.s_w[2]), M.n3, n0,
-                   min(256, M.n3 - n0), M.kd3);
-      ptx::umma_commit(ptx::smem_u32(&cx.ctl->bar_mma));
-    }
-    wait_bar(cx, &cx.ctl->bar_mma, ph_mma);
-    ph_mma ^= 1u;
-    ptx::tc_fence_after();
-    if (alias && cx.tid == 0 && (tile + 1) * kTileM < pvalid)
-      load_part(cx, a.blob, br.w_off[0], br.w_bytes[0], P.s_w[0], &cx.ctl->bar_w[0]);
-    epilogue_scatter(cx, cx.tmem_row, M.n3, cb, acc, pg, w, rp);
-    ptx::tc_fence_before();
-    __syncthreads();
-  }
-
-  // z_b = x_b + t (encode) or x_b = z_b - t (decode); clear the accumulator for the next coupling
-  for (int idx = cx.tid; idx < cb * pg; idx += kThreads) {
-    const int c = idx / pg, p = idx - c * pg;
-    if (p < pvalid) {
+  };
+  // x_b +/-= rq(acc + bias) of the previous coupling for pixel p
+  auto apply_translation = [&](int p) {
+    const uint8_t* pm = reinterpret_cast<const uint8_t*>(prevM);
+    const int32_t* colB = reinterpret_cast<const int32_t*>(pm + prevM->off_colB);
+    const OutRq* orq = reinterpret_cast<const OutRq*>(pm + prevM->off_out);
+    for (int c = 0; c < cb; ++c) {
       const OutRq o = orq[c];
-      const uint32_t t = (uint32_t)rq_exact(acc[idx] + o.bias, o.m0, o.s);
+      const uint32_t t = (uint32_t)rq_exact(acc[c * pg + p] + o.bias, o.m0, o.s);
+      acc[c * pg + p] = 0;
       uint32_t* vv = reinterpret_cast<uint32_t*>(&v[colB[c] * pg + p]);
       *vv = kInv ? (*vv - t) : (*vv + t);
     }
-    acc[idx] = 0;
-  }
-  __syncthreads();
-}
-
-// Prior head on the kept channels: (mu, log-scale index) for every factored-out element.
-__device__ void run_prior(const Ctx& cx, const LevelPlan& P, const LevelArgs& a, int img0, int pvalid,
-                          uint32_t& ph_meta, uint32_t& ph_mma, WeightState& ws) {
-  uint8_t* smem = cx.smem;
-  const int32_t* v = reinterpret_cast<const int32_t*>(smem + P.s_v);
-  int8_t* xa = reinterpret_cast<int8_t*>(smem + P.s_xa);
-  uint8_t* sA = smem + P.s_a13;
-  const int pg = P.pg, ca = P.ca, cb = P.cb, w = P.w, h = P.h, px = P.px;
-  const BlockRef& br = P.prior;
-  if (cx.tid == 0) {
-    load_part(cx, a.blob, br.meta_off, br.meta_bytes, P.s_meta, &cx.ctl->bar_meta);
-    load_part(cx, a.blob, br.w_off[0], br.w_bytes[0], P.s_w[0], &cx.ctl->bar_w[0]);
-  }
-  wait_bar(cx, &cx.ctl->bar_meta, ph_meta);
-  ph_meta ^= 1u;
-  const uint8_t* mb = smem + P.s_meta;
-  const PriorMeta M = *reinterpret_cast<const PriorMeta*>(mb);
-  const OutRq* orq = reinterpret_cast<const OutRq*>(mb + M.off_out);
-  for (int idx = cx.tid; idx < ca * pg; idx += kThreads) {
-    const int c = idx / pg, p = idx - c * pg;
-    int y = 0;
-    if (p < pvalid) y = clampi(rq_exact(v[P.col_out[c] * pg + p], M.in_m0, M.in_s), -128, 127);
-    xa[idx] = (int8_t)y;
-  }
-  __syncthreads();
-  bool w_ready = false;
-  for (int tile = 0; tile < P.tiles; ++tile) {
-    if (tile * kTileM >= pvalid) break;
-    const RowPos rp = row_pos(tile, cx.row, pvalid, px, h, w);
-    build_im2col(cx, sA, xa, ca, pg, w, M.kd, rp);
-    ptx::fence_async_smem();
-    __syncthreads();
-    if (cx.tid == 0) {
-      if (!w_ready) { wait_bar(cx, &cx.ctl->bar_w[0], ws.ph[0]); ws.ph[0] ^= 1u; w_ready = true; }
-      ptx::tc_fence_after();
-      issue_gemm(cx.tmem, ptx::smem_u32(sA), ptx::smem_u32(smem + P.s_w[0]), M.n, 0, M.n, M.kd);
-      ptx::umma_commit(ptx::smem_u32(&cx.ctl->bar_mma));
-    }
-    wait_bar(cx, &cx.ctl->bar_mma, ph_mma);
-    ph_mma ^= 1u;
-    ptx::tc_fence_after();
-    const int g = rp.valid ? rp.p / px : 0;
-    const int q = rp.p - g * px;
-    int32_t* mu = a.prior + (size_t)(img0 + g) * 2u * P.d_fact + P.prior_off + q;
-    int32_t* ls = mu + P.d_fact;
-    const int nblk = M.n >> 4;
-    for (int b = cx.wh; b < nblk; b += kThreads / kTileM) {
-      uint32_t r[16];
-      ptx::tmem_ld16(cx.tmem_row + (uint32_t)(b << 4), r);
-      ptx::tmem_ld_wait();
-      if (rp.valid) {
+  };
+  // network input of pixel p: ca channels requantised to int8, padded to cpad bytes
+  auto requant_input = [&](int p, const int32_t* cols, int32_t m0, int32_t s) {
+    for (int g0 = 0; g0 < cpad; g0 += 8) {
+      int y[8];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int col = (b << 4) + i;
-          if (col < 2 * cb) {
-            const OutRq o = orq[col];
-            const int32_t y = rq_exact((int32_t)r[i] + o.bias, o.m0, o.s);
-            if (col < cb) mu[(size_t)col * px] = y;
-            else ls[(size_t)(col - cb) * px] = clampi(y, M.ls_lo, M.ls_hi);
-          }
-        }
+      for (int i = 0; i < 8; ++i) {
+        y[i] = 0;
+        if (g0 + i < ca) y[i] = clampi(rq_exact(v[cols[g0 + i] * pg + p], m0, s), -128, 127);
       }
+      *reinterpret_cast<uint2*>(xa + (size_t)p * cpad + g0) =
+          make_uint2(pack4(y[0], y[1], y[2], y[3]), pack4(y[4], y[5], y[6], y[7]));
+    }
+  };
+
+  for (int i = 0; i < st.nsteps; ++i) {
+    wait_bar(ctl, a.status, &ctl->meta_full[i & 1], (uint32_t)((i >> 1) & 1));
+    const uint8_t* mb = smem + P.s_meta[i & 1];
+    const bool prior = st.is_prior(i);
+    if (prior) {
+      const PriorMeta M = *reinterpret_cast<const PriorMeta*>(mb);
+      const OutRq* orq = reinterpret_cast<const OutRq*>(mb + M.off_out);
+      for (int p = cx.tid; p < pvalid; p += kWorkers) {
+        if (prevM) apply_translation(p);
+        requant_input(p, P.col_out, M.in_m0, M.in_s);
+      }
+      prevM = nullptr;
+      worker_barrier();
+      for (int t = cx.group; t < ntv; t += P.nslots) {
+        const RowPos rp = row_pos(t, cx.row, pvalid, px, h, w);
+        build_im2col(cx, sA, xa, cpad, w, M.kd, rp);
+        arrive_a();
+        wait_d();
+        epilogue_prior(cx, P, a, M, orq, img0, rp);
+      }
+      worker_barrier();
+      continue;
+    }
+    const CouplingMeta* Mp = reinterpret_cast<const CouplingMeta*>(mb);
+    const CouplingMeta M = *Mp;
+    const int32_t* colA = reinterpret_cast<const int32_t*>(mb + M.off_colA);
+    const HiddenRq* h1 = reinterpret_cast<const HiddenRq*>(mb + M.off_h1);
+    const HiddenRq* h2 = reinterpret_cast<const HiddenRq*>(mb + M.off_h2);
+    for (int p = cx.tid; p < pvalid; p += kWorkers) {
+      if (prevM) apply_translation(p);
+      requant_input(p, colA, M.in_m0, M.in_s);
+    }
+    prevM = Mp;
+    worker_barrier();
+    for (int t = cx.group; t < ntv; t += P.nslots) {
+      const RowPos rp = row_pos(t, cx.row, pvalid, px, h, w);
+      build_im2col(cx, sA, xa, cpad, w, M.kd1, rp);
+      arrive_a();
+      wait_d();
+      epilogue_hidden(cx, M.fast1, M.n1, M.kd2, h1, M.lo1, M.hi1, sA);
+      arrive_a();
+      wait_d();
+      epilogue_hidden(cx, M.fast2, M.n2, M.kd3, h2, M.lo2, M.hi2, sA);
+      arrive_a();
+      wait_d();
+      epilogue_scatter(cx, cb, cbp, acc, pg, w, rp);
     }
     ptx::tc_fence_before();
-    __syncthreads();
+    worker_barrier();
   }
+  if (prevM) {
+    for (int p = cx.tid; p < pvalid; p += kWorkers) apply_translation(p);
+    worker_barrier();
+  }
+  (void)gthreads;
 }
 
 template <bool kInv>
@@ -399,117 +565,133 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
   extern __shared__ __align__(1024) uint8_t smem[];
   __shared__ Ctl ctl;
   const LevelPlan& P = *a.plan;
-  Ctx cx;
-  cx.smem = smem;
-  cx.ctl = &ctl;
-  cx.status = a.status;
-  cx.tid = threadIdx.x;
-  cx.warp = cx.tid >> 5;
-  cx.lane = cx.tid & 31;
-  cx.wq = cx.warp & 3;
-  cx.wh = cx.warp >> 2;
-  cx.row = cx.wq * 32 + cx.lane;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool is_worker = warp < kWorkerWarps;
+  const int wpg = kWorkerWarps / P.nslots;       // warps per group
 
-  if (cx.tid == 0) {
-    ptx::mbar_init(ptx::smem_u32(&ctl.bar_meta), 1);
-    for (int i = 0; i < 3; ++i) ptx::mbar_init(ptx::smem_u32(&ctl.bar_w[i]), 1);
-    ptx::mbar_init(ptx::smem_u32(&ctl.bar_mma), 1);
+  if (tid == 0) {
+    for (int s = 0; s < 2; ++s) {
+      ptx::mbar_init(ptx::smem_u32(&ctl.a_ready[s]), (uint32_t)(wpg * 32));
+      ptx::mbar_init(ptx::smem_u32(&ctl.d_ready[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl.meta_full[s]), 1);
+    }
+    for (int s = 0; s < 3; ++s) {
+      ptx::mbar_init(ptx::smem_u32(&ctl.w_full[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl.w_free[s]), 1);
+    }
     ptx::mbar_init_fence();
     ctl.abort = 0;
   }
-  if (cx.warp == 0) ptx::tmem_alloc(ptx::smem_u32(&ctl.tmem_base), (uint32_t)P.tmem_cols);
+  if (warp == 0) ptx::tmem_alloc(ptx::smem_u32(&ctl.tmem_base), (uint32_t)P.tmem_cols);
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
-  cx.tmem = ctl.tmem_base;
-  cx.tmem_row = cx.tmem + ((uint32_t)(cx.wq * 32) << 16);
+  const uint32_t tmem = ctl.tmem_base;
 
   const int c = P.c, px = P.px, pg = P.pg, w = P.w;
   const int img0 = blockIdx.x * P.group;
   const int nimg = min(P.group, a.batch - img0);
   const int pvalid = nimg * px;
+  const int ntv = (pvalid + kTileM - 1) / kTileM;
   const int per_img = c * px;                    // elements per image at this level
   int32_t* v = reinterpret_cast<int32_t*>(smem + P.s_v);
-  int32_t* acc = reinterpret_cast<int32_t*>(smem + P.s_acc);
-  for (int idx = cx.tid; idx < P.cb * pg; idx += kThreads) acc[idx] = 0;
 
-  if (!kInv) {
-    // space-to-depth on load: plane c*4 + dy*2 + dx, pixel (i, j) <- in[c][2i+dy][2j+dx]
-    const int w2 = 2 * w;
-    for (int e = cx.tid; e < nimg * per_img; e += kThreads) {
-      const int g = e / per_img, r = e - g * per_img;
-      const int ci = r / (4 * px), r2 = r - ci * 4 * px;
-      const int y = r2 / w2, x = r2 - y * w2;
-      const size_t src = (size_t)(img0 + g) * per_img + r;
-      const int32_t val = P.is_first ? (int32_t) reinterpret_cast<const uint8_t*>(a.in)[src]
-                                     : reinterpret_cast<const int32_t*>(a.in)[src];
-      v[(ci * 4 + (y & 1) * 2 + (x & 1)) * pg + g * px + (y >> 1) * w + (x >> 1)] = val;
+  Steps st;
+  st.n_couplings = P.n_couplings;
+  st.do_prior = P.has_prior && a.prior != nullptr;
+  st.nsteps = P.n_couplings + (st.do_prior ? 1 : 0);
+  st.inverse = kInv;
+
+  if (!is_worker) {
+    if (lane == 0) {
+      Control ctrl{P, a, smem, &ctl, st, ntv, P.w13_alias != 0};
+      ctrl.run(tmem);
     }
   } else {
-    // merge: logical channel k < keep_c from the deeper level, the rest from z's block of this level
-    for (int e = cx.tid; e < nimg * per_img; e += kThreads) {
-      const int g = e / per_img, r = e - g * per_img;
-      const int k = r / px, q = r - k * px;
-      const size_t b = (size_t)(img0 + g);
-      const int32_t val = (k < P.keep_c)
-                              ? reinterpret_cast<const int32_t*>(a.in)[b * (size_t)a.in_stride + (size_t)k * px + q]
-                              : a.z[b * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q];
-      v[P.col_out[k] * pg + g * px + q] = val;
-    }
-  }
-  __syncthreads();
+    Ctx cx;
+    cx.smem = smem;
+    cx.ctl = &ctl;
+    cx.status = a.status;
+    cx.tid = tid;
+    cx.warp = warp;
+    cx.lane = lane;
+    cx.wq = warp & 3;
+    cx.group = warp / wpg;
+    cx.cs = (warp % wpg) >> 2;
+    cx.ncs = wpg >> 2;
+    cx.row = cx.wq * 32 + lane;
+    cx.tmem_slot = tmem + ((uint32_t)(cx.wq * 32) << 16) + (uint32_t)(cx.group * kSlotCols);
 
-  uint32_t ph_meta = 0, ph_mma = 0;
-  WeightState ws;
-  ws.ph[0] = ws.ph[1] = ws.ph[2] = 0;
-
-  if (kInv && P.has_prior && a.prior != nullptr) run_prior(cx, P, a, img0, pvalid, ph_meta, ph_mma, ws);
-
-  for (int jj = 0; jj < P.n_couplings; ++jj) {
-    const int j = kInv ? (P.n_couplings - 1 - jj) : jj;
-    run_coupling<kInv>(cx, P, a, P.coupling[j], pvalid, ph_meta, ph_mma, ws);
-  }
-
-  if (!kInv) {
-    // split on store: factored-out half -> z block of this level; kept half -> next level (or the
-    // final z block)
-    int32_t* keep_out = reinterpret_cast<int32_t*>(a.out);
-    for (int e = cx.tid; e < nimg * per_img; e += kThreads) {
-      const int g = e / per_img, r = e - g * per_img;
-      const int k = r / px, q = r - k * px;
-      const size_t b = (size_t)(img0 + g);
-      const int32_t val = v[P.col_out[k] * pg + g * px + q];
-      if (k >= P.keep_c) a.z[b * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q] = val;
-      else if (P.is_last) a.z[b * P.d + P.z_final_off + (size_t)k * px + q] = val;
-      else keep_out[(b * P.keep_c + k) * (size_t)px + q] = val;
-    }
-    if (P.has_prior && a.prior != nullptr) run_prior(cx, P, a, img0, pvalid, ph_meta, ph_mma, ws);
-  } else {
-    // depth-to-space on store
-    const int w2 = 2 * w;
-    uint32_t bad = 0;
-    for (int e = cx.tid; e < nimg * per_img; e += kThreads) {
-      const int g = e / per_img, r = e - g * per_img;
-      const int ci = r / (4 * px), r2 = r - ci * 4 * px;
-      const int y = r2 / w2, x = r2 - y * w2;
-      const int32_t val = v[(ci * 4 + (y & 1) * 2 + (x & 1)) * pg + g * px + (y >> 1) * w + (x >> 1)];
-      const size_t dst = (size_t)(img0 + g) * per_img + r;
-      if (P.is_first) {
-        reinterpret_cast<uint8_t*>(a.out)[dst] = (uint8_t)((uint32_t)val & 0xFFu);
-        bad += (val < 0 || val > 255) ? 1u : 0u;
-      } else {
-        reinterpret_cast<int32_t*>(a.out)[dst] = val;
+    int32_t* acc = reinterpret_cast<int32_t*>(smem + P.s_acc);
+    for (int idx = tid; idx < P.cb * pg; idx += kWorkers) acc[idx] = 0;
+    if (!kInv) {
+      // space-to-depth on load: plane c*4 + dy*2 + dx, pixel (i, j) <- in[c][2i+dy][2j+dx]
+      const int w2 = 2 * w;
+      for (int e = tid; e < nimg * per_img; e += kWorkers) {
+        const int g = e / per_img, r = e - g * per_img;
+        const int ci = r / (4 * px), r2 = r - ci * 4 * px;
+        const int y = r2 / w2, x = r2 - y * w2;
+        const size_t src = (size_t)(img0 + g) * per_img + r;
+        const int32_t val = P.is_first ? (int32_t) reinterpret_cast<const uint8_t*>(a.in)[src]
+                                       : reinterpret_cast<const int32_t*>(a.in)[src];
+        v[(ci * 4 + (y & 1) * 2 + (x & 1)) * pg + g * px + (y >> 1) * w + (x >> 1)] = val;
+      }
+    } else {
+      // merge: logical channel k < keep_c from the deeper level, the rest from z's block of this level
+      for (int e = tid; e < nimg * per_img; e += kWorkers) {
+        const int g = e / per_img, r = e - g * per_img;
+        const int k = r / px, q = r - k * px;
+        const size_t b = (size_t)(img0 + g);
+        const int32_t val =
+            (k < P.keep_c) ? reinterpret_cast<const int32_t*>(a.in)[b * (size_t)a.in_stride + (size_t)k * px + q]
+                           : a.z[b * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q];
+        v[P.col_out[k] * pg + g * px + q] = val;
       }
     }
-    if (P.is_first && a.oor != nullptr) {
-      bad = __reduce_add_sync(0xFFFFFFFFu, bad);
-      if (cx.lane == 0 && bad) atomicAdd(a.oor, bad);
+    worker_barrier();
+
+    run_workers<kInv>(cx, P, a, st, img0, pvalid, ntv);
+
+    if (!kInv) {
+      // split on store: factored-out half -> z block of this level; kept half -> next level (or
+      // the final z block)
+      int32_t* keep_out = reinterpret_cast<int32_t*>(a.out);
+      for (int e = tid; e < nimg * per_img; e += kWorkers) {
+        const int g = e / per_img, r = e - g * per_img;
+        const int k = r / px, q = r - k * px;
+        const size_t b = (size_t)(img0 + g);
+        const int32_t val = v[P.col_out[k] * pg + g * px + q];
+        if (k >= P.keep_c) a.z[b * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q] = val;
+        else if (P.is_last) a.z[b * P.d + P.z_final_off + (size_t)k * px + q] = val;
+        else keep_out[(b * P.keep_c + k) * (size_t)px + q] = val;
+      }
+    } else {
+      // depth-to-space on store
+      const int w2 = 2 * w;
+      uint32_t bad = 0;
+      for (int e = tid; e < nimg * per_img; e += kWorkers) {
+        const int g = e / per_img, r = e - g * per_img;
+        const int ci = r / (4 * px), r2 = r - ci * 4 * px;
+        const int y = r2 / w2, x = r2 - y * w2;
+        const int32_t val = v[(ci * 4 + (y & 1) * 2 + (x & 1)) * pg + g * px + (y >> 1) * w + (x >> 1)];
+        const size_t dst = (size_t)(img0 + g) * per_img + r;
+        if (P.is_first) {
+          reinterpret_cast<uint8_t*>(a.out)[dst] = (uint8_t)((uint32_t)val & 0xFFu);
+          bad += (val < 0 || val > 255) ? 1u : 0u;
+        } else {
+          reinterpret_cast<int32_t*>(a.out)[dst] = val;
+        }
+      }
+      if (P.is_first && a.oor != nullptr) {
+        bad = __reduce_add_sync(0xFFFFFFFFu, bad);
+        if (lane == 0 && bad) atomicAdd(a.oor, bad);
+      }
     }
   }
 
   ptx::tc_fence_before();
   __syncthreads();
-  if (cx.warp == 0) ptx::tmem_dealloc(cx.tmem, (uint32_t)P.tmem_cols);
+  if (warp == 0) ptx::tmem_dealloc(tmem, (uint32_t)P.tmem_cols);
 }
 
 }  // namespace
