@@ -96,11 +96,13 @@ int hidden_range(const iodf_layer_desc& L, Act* out) {
   return IODF_OK;
 }
 
-void put_hidden_rq(HiddenRq* dst, const iodf_layer_desc& L, const Blobs& B, int n_pad, int* fast) {
+// Fills both constant tables of a hidden layer and picks its requantisation flavour.
+void put_hidden_rq(HiddenRq* dst, int32_t* mb, const iodf_layer_desc& L, const Blobs& B, int n_pad, int* mode,
+                   int* uniform_s) {
   const int32_t* bias = B.r + L.requant_off;
   const int32_t* m0 = bias + L.c_out;
   const int32_t* s = m0 + L.c_out;
-  *fast = 1;
+  bool fast = true, uniform = true;
   for (int i = 0; i < n_pad; ++i) {
     HiddenRq h;
     if (i < (int)L.c_out) {
@@ -109,15 +111,22 @@ void put_hidden_rq(HiddenRq* dst, const iodf_layer_desc& L, const Blobs& B, int 
       h.sh = s[i] - 1;
       h.c_lo = (uint32_t)((unsigned long long)c64 & 0xFFFFFFFFull);
       h.c_hi = (uint32_t)((unsigned long long)c64 >> 32);
-      if (s[i] < 1) *fast = 0;
-    } else {  // padding channel: acc = 0 -> 0
+      if (s[i] < 1) fast = false;
+      if (s[i] != s[0] || s[i] < 1) uniform = false;
+      mb[2 * i] = m0[i];
+      mb[2 * i + 1] = bias[i];
+    } else {  // padding channel: acc = 0 -> 0 (its weights in the next layer are zero anyway)
       h.m0 = 1 << 30;
       h.sh = 0;
       h.c_lo = 0x80000000u;
       h.c_hi = 0;
+      mb[2 * i] = 1 << 30;
+      mb[2 * i + 1] = 0;
     }
     dst[i] = h;
   }
+  *mode = uniform ? 2 : (fast ? 1 : 0);
+  *uniform_s = uniform ? s[0] : 0;
 }
 
 void put_out_rq(OutRq* dst, const iodf_layer_desc& L, const Blobs& B) {
@@ -170,12 +179,16 @@ PackedBlock pack_coupling(const iodf_coupling_desc& cp, const Blobs& B, int ca, 
   M.off_out = (int)off;  off += (uint32_t)sizeof(OutRq) * cb;
   M.off_h1 = (int)off;   off += (uint32_t)sizeof(HiddenRq) * d.n1;
   M.off_h2 = (int)off;   off += (uint32_t)sizeof(HiddenRq) * d.n2;
+  M.off_u1 = (int)off;   off += 8u * d.n1;
+  M.off_u2 = (int)off;   off += 8u * d.n2;
   pb.meta.assign(off, 0);
   std::memcpy(pb.meta.data() + M.off_colA, colA, 4 * ca);
   std::memcpy(pb.meta.data() + M.off_colB, colB, 4 * cb);
   put_out_rq(reinterpret_cast<OutRq*>(pb.meta.data() + M.off_out), L3, B);
-  put_hidden_rq(reinterpret_cast<HiddenRq*>(pb.meta.data() + M.off_h1), L1, B, d.n1, &M.fast1);
-  put_hidden_rq(reinterpret_cast<HiddenRq*>(pb.meta.data() + M.off_h2), L2, B, d.n2, &M.fast2);
+  put_hidden_rq(reinterpret_cast<HiddenRq*>(pb.meta.data() + M.off_h1),
+                reinterpret_cast<int32_t*>(pb.meta.data() + M.off_u1), L1, B, d.n1, &M.mode1, &M.us1);
+  put_hidden_rq(reinterpret_cast<HiddenRq*>(pb.meta.data() + M.off_h2),
+                reinterpret_cast<int32_t*>(pb.meta.data() + M.off_u2), L2, B, d.n2, &M.mode2, &M.us2);
   std::memcpy(pb.meta.data(), &M, sizeof(M));
 
   // W1: row = hidden channel, K index = tap*cpad + c
@@ -248,6 +261,7 @@ bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32
       P.s_v = take((uint32_t)P.c * pg * 4);
       P.s_xa = take(pg * (uint32_t)P.cpad);
       P.s_acc = take((uint32_t)P.cb * pg * 4);
+      P.s_rowinfo = take((uint32_t)tiles * kTileM * 4);
       P.s_a[0] = take(a_bytes);
       P.s_a[1] = mode == 0 ? take(a_bytes) : P.s_a[0];
       P.s_meta[0] = take(meta_bytes);
@@ -391,6 +405,8 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
     P.d = lay.d; P.d_fact = lay.d_fact;
 
     P.cpad = (int)up(ca, 8); P.cbp = (int)up(cb, 8);
+    P.recip_gpa = 65536u / (uint32_t)(P.cpad / 8) + 1u;
+    P.recip_gpb = 65536u / (uint32_t)(P.cbp / 8) + 1u;
     std::vector<int> pi(c);
     for (uint32_t k = 0; k < c; ++k) pi[k] = (int)k;
     uint32_t a_bytes = 16, meta = 16, wmax[3] = {16, 16, 16};

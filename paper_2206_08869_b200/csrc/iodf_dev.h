@@ -21,7 +21,7 @@ namespace iodf {
 constexpr int kTileM = 128;          // pixels per MMA tile (UMMA M)
 constexpr int kWorkerWarps = 16;     // four per TMEM lane quarter
 constexpr int kWorkers = kWorkerWarps * 32;
-constexpr int kThreads = kWorkers + 32;   // + one control warp (bulk copies and MMA issue)
+constexpr int kThreads = kWorkers;
 constexpr int kMaxCouplings = 32;    // per level
 constexpr int kMaxC = 256;           // flow channels per level
 constexpr int kMaxHidden = 256;      // kept hidden channels per layer (padded)
@@ -43,16 +43,21 @@ struct OutRq {
 
 // Meta part of a coupling block, followed in memory by
 //   colA[ca] colB[cb] (int32 physical column of each logical channel), OutRq[cb],
-//   HiddenRq[n1], HiddenRq[n2]; every array 16-byte aligned.
+//   HiddenRq[n1], HiddenRq[n2], {m0, bias}[n1], {m0, bias}[n2]; every array 16-byte aligned.
 struct CouplingMeta {
   int32_t in_m0, in_s;
   int32_t n1, n2;                // hidden widths padded to 16 (MMA N)
   int32_t kd1, kd2, kd3;         // K bytes of the three GEMMs, padded to 32
   int32_t n3;                    // 9*cbp padded to 16 (per-tap partial outputs of the last conv)
   int32_t lo1, hi1, lo2, hi2;    // effective activation clips (ReLU folded in)
-  int32_t fast1, fast2;          // 1: every s >= 1 in that layer (fast path exact)
+  int32_t mode1, mode2;          // requantisation flavour of the two hidden layers:
+                                 //   2: one shift s >= 1 for the whole layer ({m0, bias} table)
+                                 //   1: per-channel shifts, all >= 1 (HiddenRq table, high-word path)
+                                 //   0: any shift (HiddenRq table, full 64-bit shift)
+  int32_t us1, us2;              // the uniform shift (mode 2)
   int32_t off_colA, off_colB, off_out, off_h1, off_h2;   // byte offsets from the meta start
-  int32_t pad[13];
+  int32_t off_u1, off_u2;        // {m0, bias} tables (int2 per channel)
+  int32_t pad[9];
 };
 static_assert(sizeof(CouplingMeta) == 128, "meta header is 128 bytes");
 
@@ -87,7 +92,8 @@ struct LevelPlan {
   int32_t tmem_cols;
   int32_t w13_alias;             // 1: W1 and W3 share a slot and are re-fetched per tile
   // shared-memory byte offsets
-  uint32_t s_v, s_xa, s_acc, s_a[2], s_meta[2], s_w[3], s_total;
+  uint32_t s_v, s_xa, s_acc, s_rowinfo, s_a[2], s_meta[2], s_w[3], s_total;
+  uint32_t recip_gpa, recip_gpb; // floor(g / (cpad/8)) = (g * recip_gpa) >> 16 for g < 4096; same for cbp/8
   // global layout
   uint64_t z_off, prior_off, z_final_off, d, d_fact;
   int32_t col_out[kMaxC];        // physical column of logical channel k after the last coupling

@@ -24,11 +24,12 @@
 // coupling addresses v through its table of physical columns (the composition of all permutations
 // so far), and the level's outputs are written through the final table.
 //
-// Execution structure: 16 worker warps and one control warp. The workers form one or two groups;
-// each group owns a tile slot (an A-operand buffer in shared memory and a range of TMEM columns)
-// and walks its tiles through build -> epilogue 1 -> epilogue 2 -> scatter, handing the slot to
-// the control thread between stages through mbarriers. The control thread issues the bulk copies
-// of weights and the MMAs, so while one group requantises, the tensor core works for the other.
+// Execution structure: 16 warps form one or two groups; each group owns a tile slot (an A-operand
+// buffer in shared memory and a range of TMEM columns) and walks its tiles through build ->
+// epilogue 1 -> epilogue 2 -> scatter. Between stages the group meets at a named barrier, one
+// elected thread issues the stage's MMAs and commits them to the slot's mbarrier, and the group
+// waits on it; so while one group requantises, the tensor core works for the other. One thread
+// of the CTA also issues the bulk copies that bring the next coupling's weights in.
 #include "iodf_dev.h"
 #include "level_kernel.h"
 #include "ptx.cuh"
@@ -38,10 +39,8 @@ namespace iodf {
 namespace {
 
 struct __align__(16) Ctl {
-  uint64_t a_ready[2];    // workers -> control: the slot's A operand is written (count = group threads)
-  uint64_t d_ready[2];    // tensor core -> workers: the slot's accumulator is complete
-  uint64_t w_full[3];     // bulk copy -> control: weight slot filled
-  uint64_t w_free[3];     // tensor core -> control: last MMA reading the weight slot is complete
+  uint64_t d_ready[2];    // tensor core -> group: the slot's accumulator is complete
+  uint64_t w_full[3];     // bulk copy -> elected threads: weight slot filled
   uint64_t meta_full[2];  // bulk copy -> everyone: meta block of step (i & 1) has landed
   uint32_t tmem_base;
   uint32_t abort;
@@ -54,8 +53,12 @@ struct Ctx {
   int tid, warp, lane;
   int wq;                 // TMEM lane quarter of this warp
   int group, cs, ncs;     // tile slot, column-split index and count inside the group
+  int gthreads;           // threads per group
   int row;                // tile row (= TMEM lane) of this thread
+  bool elected;           // issues this group's MMAs
+  bool loader;            // issues the CTA's bulk copies (the elected thread of group 0)
   uint32_t tmem_slot;     // TMEM address of the slot's first column, this warp's lane quarter
+  uint32_t tmem_slot0;    // the same with lane field 0 (MMA destination)
 };
 
 // Bounded wait on an mbarrier phase. After one wait in the CTA has given up, every later wait
@@ -73,11 +76,15 @@ __device__ __noinline__ bool wait_bar(Ctl* ctl, uint32_t* status, uint64_t* bar,
   return false;
 }
 
-__device__ __forceinline__ void worker_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); }
+__device__ __forceinline__ void worker_barrier() { __syncthreads(); }
+__device__ __forceinline__ void group_barrier(int group, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(group + 1), "r"(nthreads) : "memory");
+}
 
 __device__ __forceinline__ int32_t rq_exact(int32_t a, int32_t m0, int32_t s) {
   const long long p = (long long)a * (long long)m0 + (1ll << (30 + s));
-  return (int32_t)(p >> (31 + s));
+  if (s >= 1) return ((int32_t)(p >> 32)) >> (s - 1);   // same value, one 32-bit shift
+  return (int32_t)(p >> 31);
 }
 
 __device__ __forceinline__ int clampi(int v, int lo, int hi) { return min(max(v, lo), hi); }
@@ -86,16 +93,6 @@ __device__ __forceinline__ int min_relu(int v, int hi) {
   int r;
   asm("min.relu.s32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(hi));
   return r;
-}
-
-template <bool kFast, bool kLo0>
-__device__ __forceinline__ int rq_hidden(int acc, const HiddenRq r, int lo, int hi) {
-  const long long c64 = (long long)(((unsigned long long)r.c_hi << 32) | (unsigned long long)r.c_lo);
-  const long long p = (long long)acc * (long long)r.m0 + c64;
-  int y;
-  if (kFast) y = ((int)(p >> 32)) >> r.sh;
-  else y = (int)(p >> (32 + r.sh));
-  return kLo0 ? min_relu(y, hi) : clampi(y, lo, hi);
 }
 
 __device__ __forceinline__ uint32_t pack4(int y0, int y1, int y2, int y3) {
@@ -112,25 +109,31 @@ struct RowPos {
   uint32_t smask;   // bit t: output pixel (i-u+1, j-v+1) is inside the image           (scatter)
 };
 
-__device__ __forceinline__ RowPos row_pos(int tile, int row, int pvalid, int px, int h, int w) {
+// Packed row record: bit 0 valid, bits 1..9 gather mask, bits 10..18 scatter mask.
+__device__ __forceinline__ uint32_t row_record(int p, int pvalid, int px, int h, int w) {
+  if (p >= pvalid) return 0u;
+  uint32_t r = 1u;
+  const int q = p % px;
+  const int i = q / w, j = q - i * w;
+#pragma unroll
+  for (int u = 0; u < 3; ++u)
+#pragma unroll
+    for (int v = 0; v < 3; ++v) {
+      const bool gi = (i + u - 1 >= 0) && (i + u - 1 < h) && (j + v - 1 >= 0) && (j + v - 1 < w);
+      const bool si = (i - u + 1 >= 0) && (i - u + 1 < h) && (j - v + 1 >= 0) && (j - v + 1 < w);
+      r |= (gi ? 1u : 0u) << (1 + u * 3 + v);
+      r |= (si ? 1u : 0u) << (10 + u * 3 + v);
+    }
+  return r;
+}
+
+__device__ __forceinline__ RowPos row_pos(const uint32_t* rowinfo, int tile, int row) {
   RowPos r;
   r.p = tile * kTileM + row;
-  r.valid = r.p < pvalid;
-  r.gmask = 0;
-  r.smask = 0;
-  if (r.valid) {
-    const int q = r.p % px;
-    const int i = q / w, j = q - i * w;
-#pragma unroll
-    for (int u = 0; u < 3; ++u)
-#pragma unroll
-      for (int v = 0; v < 3; ++v) {
-        const bool gi = (i + u - 1 >= 0) && (i + u - 1 < h) && (j + v - 1 >= 0) && (j + v - 1 < w);
-        const bool si = (i - u + 1 >= 0) && (i - u + 1 < h) && (j - v + 1 >= 0) && (j - v + 1 < w);
-        r.gmask |= (gi ? 1u : 0u) << (u * 3 + v);
-        r.smask |= (si ? 1u : 0u) << (u * 3 + v);
-      }
-  }
+  const uint32_t rec = rowinfo[r.p];
+  r.valid = (rec & 1u) != 0;
+  r.gmask = (rec >> 1) & 0x1FFu;
+  r.smask = (rec >> 10) & 0x1FFu;
   return r;
 }
 
@@ -141,10 +144,12 @@ __device__ __forceinline__ int tap_offset(int tap, int w) {
 
 // A[row][tap*cpad + c] = xa[p + tap offset][c] (0 outside the image), as aligned 8-byte granules,
 // written in 16-byte chunks into the MMA operand layout [K/16][128][16].
-__device__ void build_im2col(const Ctx& cx, uint8_t* sA, const int8_t* xa, int cpad, int w, int kd, const RowPos rp) {
+__device__ void build_im2col(const Ctx& cx, uint8_t* __restrict__ sA, const int8_t* __restrict__ xa, int cpad, int w,
+                             int kd, uint32_t recip_gpt, const RowPos rp) {
   const int nchunks = kd >> 4;
   const int gpt = cpad >> 3;                // granules per tap
   const int ngran = 9 * gpt;
+  const int8_t* base = xa + (size_t)rp.p * cpad;
   for (int jc = cx.cs; jc < nchunks; jc += cx.ncs) {
     uint2 g2[2];
 #pragma unroll
@@ -152,9 +157,9 @@ __device__ void build_im2col(const Ctx& cx, uint8_t* sA, const int8_t* xa, int c
       const int g = 2 * jc + half;
       g2[half] = make_uint2(0u, 0u);
       if (g < ngran) {
-        const int tap = g / gpt, i = g - tap * gpt;
+        const int tap = (int)(((uint32_t)g * recip_gpt) >> 16), i = g - tap * gpt;
         if ((rp.gmask >> tap) & 1u)
-          g2[half] = *reinterpret_cast<const uint2*>(xa + (size_t)(rp.p + tap_offset(tap, w)) * cpad + 8 * i);
+          g2[half] = *reinterpret_cast<const uint2*>(base + tap_offset(tap, w) * cpad + 8 * i);
       }
     }
     *reinterpret_cast<uint4*>(sA + (size_t)jc * (kTileM * 16) + cx.row * 16) =
@@ -162,25 +167,66 @@ __device__ void build_im2col(const Ctx& cx, uint8_t* sA, const int8_t* xa, int c
   }
 }
 
-// 16 accumulator columns -> requantised bytes -> one 16-byte chunk of the next A operand.
-template <bool kFast, bool kLo0>
-__device__ __forceinline__ uint4 requant16(const uint32_t* r, const HiddenRq* rq, int lo, int hi) {
-  uint32_t wd[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int y0 = rq_hidden<kFast, kLo0>((int)r[4 * i + 0], rq[4 * i + 0], lo, hi);
-    const int y1 = rq_hidden<kFast, kLo0>((int)r[4 * i + 1], rq[4 * i + 1], lo, hi);
-    const int y2 = rq_hidden<kFast, kLo0>((int)r[4 * i + 2], rq[4 * i + 2], lo, hi);
-    const int y3 = rq_hidden<kFast, kLo0>((int)r[4 * i + 3], rq[4 * i + 3], lo, hi);
-    wd[i] = pack4(y0, y1, y2, y3);
-  }
-  return make_uint4(wd[0], wd[1], wd[2], wd[3]);
+// Requantisation flavours of a hidden layer (chosen per layer when the model is packed):
+//   kModeUniform  every channel has the same shift s >= 1: constants {m0, bias} per channel,
+//                 y = hi32((acc + bias) * m0 + 2^(30+s)) >> (s-1)
+//   kModeFast     per-channel shifts, all s >= 1: y = hi32(acc * m0 + c64) >> (s-1)
+//   kModeExact    any s: y = (acc * m0 + c64) >> (31 + s) in 64 bits
+// All three are exact: for s >= 1, floor(x / 2^(31+s)) = floor(floor(x / 2^32) / 2^(s-1)).
+constexpr int kModeUniform = 2, kModeFast = 1, kModeExact = 0;
+
+// Clip flavours: kClipS8Relu is the common ReLU + clip to [0, 127]: max(y, 0) followed by the
+// saturating 32->8 bit pack (which clips at 127); kClipAny is max/min with the layer's bounds.
+constexpr int kClipS8Relu = 1, kClipAny = 0;
+
+// d = {sat8(y3), sat8(y2), sat8(y1), sat8(y0)} (y0 in the lowest byte)
+__device__ __forceinline__ uint32_t pack4_sat(int y0, int y1, int y2, int y3) {
+  uint32_t t, w;
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(y3), "r"(y2), "r"(0));
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(y1), "r"(y0), "r"(t));
+  return w;
 }
+
+template <int kMode, int kClip>
+struct Requant {
+  const HiddenRq* __restrict__ rq;     // kModeFast / kModeExact
+  const int2* __restrict__ mb;         // kModeUniform: {m0, bias}
+  int lo, hi, sh;
+  long long rnd64;
+
+  __device__ __forceinline__ int one(int acc, int ch) const {
+    int y;
+    if (kMode == kModeUniform) {
+      const int2 c = mb[ch];
+      const long long p = (long long)(acc + c.y) * (long long)c.x + rnd64;
+      y = ((int)(p >> 32)) >> sh;
+    } else {
+      const HiddenRq r = rq[ch];
+      const long long c64 = (long long)(((unsigned long long)r.c_hi << 32) | (unsigned long long)r.c_lo);
+      const long long p = (long long)acc * (long long)r.m0 + c64;
+      if (kMode == kModeFast) y = ((int)(p >> 32)) >> r.sh;
+      else y = (int)(p >> (32 + r.sh));
+    }
+    return kClip == kClipS8Relu ? max(y, 0) : clampi(y, lo, hi);
+  }
+  // 16 accumulator columns starting at channel ch0 -> one 16-byte chunk of the next A operand
+  __device__ __forceinline__ uint4 chunk(const uint32_t* r, int ch0) const {
+    uint32_t wd[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int y0 = one((int)r[4 * i], ch0 + 4 * i), y1 = one((int)r[4 * i + 1], ch0 + 4 * i + 1);
+      const int y2 = one((int)r[4 * i + 2], ch0 + 4 * i + 2), y3 = one((int)r[4 * i + 3], ch0 + 4 * i + 3);
+      wd[i] = kClip == kClipS8Relu ? pack4_sat(y0, y1, y2, y3) : pack4(y0, y1, y2, y3);
+    }
+    return make_uint4(wd[0], wd[1], wd[2], wd[3]);
+  }
+};
 
 // TMEM accumulator -> requantised int8 activations in the next GEMM's A layout. n is a multiple
 // of 16; kd (the next GEMM's K) is n rounded up to 32, the extra chunk being zero.
-template <bool kFast, bool kLo0>
-__device__ void epilogue_hidden_t(const Ctx& cx, int n, int kd, const HiddenRq* rq, int lo, int hi, uint8_t* sOut) {
+template <int kMode, int kClip>
+__device__ __forceinline__ void epilogue_hidden_t(const Ctx& cx, int n, int kd, const Requant<kMode, kClip> q,
+                                                  uint8_t* __restrict__ sOut) {
   const int nblk = (n + 31) >> 5;
   for (int b = cx.cs; b < nblk; b += cx.ncs) {
     const int c0 = b << 5;
@@ -188,45 +234,62 @@ __device__ void epilogue_hidden_t(const Ctx& cx, int n, int kd, const HiddenRq* 
     if (n - c0 >= 32) {
       uint32_t r[32];
       ptx::tmem_ld32(cx.tmem_slot + (uint32_t)c0, r);
-      ptx::tmem_ld_wait();
-      *reinterpret_cast<uint4*>(dst) = requant16<kFast, kLo0>(r, rq + c0, lo, hi);
-      *reinterpret_cast<uint4*>(dst + kTileM * 16) = requant16<kFast, kLo0>(r + 16, rq + c0 + 16, lo, hi);
+      ptx::tmem_ld_wait32(r);
+      *reinterpret_cast<uint4*>(dst) = q.chunk(r, c0);
+      *reinterpret_cast<uint4*>(dst + kTileM * 16) = q.chunk(r + 16, c0 + 16);
     } else {
       uint32_t r[16];
       ptx::tmem_ld16(cx.tmem_slot + (uint32_t)c0, r);
-      ptx::tmem_ld_wait();
-      *reinterpret_cast<uint4*>(dst) = requant16<kFast, kLo0>(r, rq + c0, lo, hi);
+      ptx::tmem_ld_wait16(r);
+      *reinterpret_cast<uint4*>(dst) = q.chunk(r, c0);
       if (c0 + 16 < kd) *reinterpret_cast<uint4*>(dst + kTileM * 16) = make_uint4(0u, 0u, 0u, 0u);
     }
   }
 }
 
-__device__ void epilogue_hidden(const Ctx& cx, int fast, int n, int kd, const HiddenRq* rq, int lo, int hi,
-                                uint8_t* sOut) {
-  if (fast) {
-    if (lo == 0) epilogue_hidden_t<true, true>(cx, n, kd, rq, lo, hi, sOut);
-    else epilogue_hidden_t<true, false>(cx, n, kd, rq, lo, hi, sOut);
+// mode: layer flavour (see above); us: the layer's uniform shift (kModeUniform only).
+__device__ __forceinline__ void epilogue_hidden(const Ctx& cx, int mode, int us, int n, int kd, const HiddenRq* rq,
+                                                const int2* mb, int lo, int hi, uint8_t* sOut) {
+  const bool s8relu = lo == 0 && hi == 127;
+  if (mode == kModeUniform) {
+    const long long rnd64 = 1ll << (30 + us);
+    if (s8relu) epilogue_hidden_t(cx, n, kd, Requant<kModeUniform, kClipS8Relu>{rq, mb, lo, hi, us - 1, rnd64}, sOut);
+    else epilogue_hidden_t(cx, n, kd, Requant<kModeUniform, kClipAny>{rq, mb, lo, hi, us - 1, rnd64}, sOut);
+  } else if (mode == kModeFast) {
+    epilogue_hidden_t(cx, n, kd, Requant<kModeFast, kClipAny>{rq, mb, lo, hi, 0, 0}, sOut);
   } else {
-    epilogue_hidden_t<false, false>(cx, n, kd, rq, lo, hi, sOut);
+    epilogue_hidden_t(cx, n, kd, Requant<kModeExact, kClipAny>{rq, mb, lo, hi, 0, 0}, sOut);
   }
 }
 
 // Per-tap partial products -> shifted sum into the translation accumulator. Column granule gi
-// (8 columns) belongs to tap gi / (cbp/8) and out channels (gi % (cbp/8))*8 .. +8.
-__device__ void epilogue_scatter(const Ctx& cx, int cb, int cbp, int32_t* acc, int pg, int w, const RowPos rp) {
+// (8 columns) belongs to tap gi / (cbp/8) and out channels (gi % (cbp/8))*8 .. +8. Loads are
+// issued four granules at a time.
+__device__ void epilogue_scatter(const Ctx& cx, int cb, int cbp, uint32_t recip_gpt, int32_t* __restrict__ acc, int pg,
+                                 int w, const RowPos rp) {
   const int gpt = cbp >> 3;
   const int ngran = 9 * gpt;
-  for (int gi = cx.cs; gi < ngran; gi += cx.ncs) {
-    uint32_t r[8];
-    ptx::tmem_ld8(cx.tmem_slot + (uint32_t)(gi << 3), r);
-    ptx::tmem_ld_wait();
-    const int tap = gi / gpt;
-    const int c0 = (gi - tap * gpt) << 3;
-    if (rp.valid && ((rp.smask >> tap) & 1u)) {
-      int32_t* dst = acc + c0 * pg + rp.p - tap_offset(tap, w);
+  for (int g0 = cx.cs; g0 < ngran; g0 += 4 * cx.ncs) {
+    uint32_t r[4][8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
-        if (c0 + i < cb) atomicAdd(dst + i * pg, (int32_t)r[i]);
+    for (int k = 0; k < 4; ++k) {
+      const int gi = g0 + k * cx.ncs;
+      if (gi < ngran) ptx::tmem_ld8(cx.tmem_slot + (uint32_t)(gi << 3), r[k]);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int gi = g0 + k * cx.ncs;
+      if (gi < ngran) {
+        ptx::tmem_ld_wait8(r[k]);
+        const int tap = (int)(((uint32_t)gi * recip_gpt) >> 16);
+        const int c0 = (gi - tap * gpt) << 3;
+        if (rp.valid && ((rp.smask >> tap) & 1u)) {
+          int32_t* dst = acc + c0 * pg + rp.p - tap_offset(tap, w);
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            if (c0 + i < cb) atomicAdd(dst + i * pg, (int32_t)r[k][i]);
+        }
+      }
     }
   }
 }
@@ -243,7 +306,7 @@ __device__ void epilogue_prior(const Ctx& cx, const LevelPlan& P, const LevelArg
   for (int gi = cx.cs; gi < ngran; gi += cx.ncs) {
     uint32_t r[8];
     ptx::tmem_ld8(cx.tmem_slot + (uint32_t)(gi << 3), r);
-    ptx::tmem_ld_wait();
+    ptx::tmem_ld_wait8(r);
     if (rp.valid) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
@@ -273,7 +336,7 @@ __device__ __forceinline__ const BlockRef& step_ref(const LevelPlan& P, const St
   return st.is_prior(i) ? P.prior : P.coupling[st.coupling_index(i)];
 }
 
-// ---- control thread ---------------------------------------------------------------------------
+// ---- MMA issue and weight traffic (elected threads) --------------------------------------------
 // D[128 x n] (+)= A[128 x kd] * B[n x kd]^T for B rows n0..n0+n of a matrix with n_total rows.
 __device__ void issue_gemm(uint32_t d_tmem, uint32_t sa, uint32_t sb, int n_total, int n0, int n, int kd) {
   const uint32_t idesc = ptx::umma_idesc_s8((uint32_t)n);
@@ -285,208 +348,125 @@ __device__ void issue_gemm(uint32_t d_tmem, uint32_t sa, uint32_t sb, int n_tota
   }
 }
 
-struct WSlot {
-  uint32_t full_par, free_par;
-  int uses_left, cur_uses;
-  bool inflight, need_free, exhausted;
-  int g_step, g_sub;      // position of the load-sequence generator
+__device__ __forceinline__ void bulk_load(const Ctx& cx, const uint8_t* blob, uint32_t off, uint32_t bytes,
+                                          uint32_t s_dst, uint64_t* bar) {
+  const uint32_t b = ptx::smem_u32(bar);
+  ptx::mbar_expect_tx(b, bytes);
+  ptx::bulk_g2s(ptx::smem_u32(cx.smem + s_dst), blob + off, bytes, b);
+}
+
+// Weight bookkeeping. Slots hold, in order of use: S0 the first matrix of every step (W1 of a
+// coupling, the prior head's matrix), S1 every coupling's W2, S2 every coupling's W3. A slot's
+// k-th load completes phase k of its mbarrier, so a consumer that knows k knows the parity to wait
+// for. With `alias` (one group only) S0 instead alternates W1 and W3 for every tile, S2 is unused,
+// and the single elected thread counts S0's loads itself.
+struct Weights {
+  int cur_step[3];        // loader: step whose matrix the slot holds or is receiving (-1: none)
+  uint32_t s0_loads;      // alias mode: loads requested into S0
+  uint32_t s0_used;       // alias mode: loads consumed from S0
 };
 
-struct Control {
-  const LevelPlan& P;
-  const LevelArgs& a;
-  uint8_t* smem;
-  Ctl* ctl;
-  Steps st;
-  int ntv;                // valid tiles of this CTA
-  bool alias;
-  WSlot ws[3];
+__device__ __forceinline__ bool slot_used_by(const Steps& st, int s, int step) {
+  return s == 0 || !st.is_prior(step);
+}
+// ordinal of step i among the loads of slot s
+__device__ __forceinline__ int load_ordinal(const Steps& st, int s, int i) {
+  return (s == 0) ? i : i - ((st.inverse && st.do_prior) ? 1 : 0);
+}
 
-  __device__ bool wait(uint64_t* bar, uint32_t par) { return wait_bar(ctl, a.status, bar, par); }
-
-  __device__ void bulk(uint32_t off, uint32_t bytes, uint32_t s_dst, uint64_t* bar) {
-    const uint32_t b = ptx::smem_u32(bar);
-    ptx::mbar_expect_tx(b, bytes);
-    ptx::bulk_g2s(ptx::smem_u32(smem + s_dst), a.blob + off, bytes, b);
+// Loader: every slot whose matrix belongs to a finished step (<= done) receives the matrix of the
+// next step that uses it.
+__device__ void top_up(const Ctx& cx, const LevelPlan& P, const LevelArgs& a, const Steps& st, Weights& W, int done,
+                       bool alias) {
+  for (int s = alias ? 1 : 0; s < (alias ? 2 : 3); ++s) {
+    if (W.cur_step[s] > done) continue;
+    int j = W.cur_step[s] + 1;
+    while (j < st.nsteps && !slot_used_by(st, s, j)) ++j;
+    if (j >= st.nsteps) { W.cur_step[s] = st.nsteps; continue; }
+    const BlockRef& br = step_ref(P, st, j);
+    bulk_load(cx, a.blob, br.w_off[s], br.w_bytes[s], P.s_w[s], &cx.ctl->w_full[s]);
+    W.cur_step[s] = j;
   }
+}
 
-  // Next matrix that weight slot s will hold, in the fixed order the MMAs consume them.
-  __device__ bool next_load(int s, uint32_t* off, uint32_t* bytes, int* uses) {
-    WSlot& w = ws[s];
-    for (;;) {
-      if (w.g_step >= st.nsteps) return false;
-      const BlockRef& br = step_ref(P, st, w.g_step);
-      if (st.is_prior(w.g_step)) {
-        if (s != 0 || w.g_sub > 0) { ++w.g_step; w.g_sub = 0; continue; }
-        *off = br.w_off[0]; *bytes = br.w_bytes[0]; *uses = ntv; w.g_sub = 1;
-        return true;
-      }
-      if (alias && s == 0) {                      // W1, W3, W1, W3, ... once per tile
-        if (w.g_sub >= 2 * ntv) { ++w.g_step; w.g_sub = 0; continue; }
-        const int which = (w.g_sub & 1) ? 2 : 0;
-        *off = br.w_off[which]; *bytes = br.w_bytes[which]; *uses = 1; ++w.g_sub;
-        return true;
-      }
-      if (alias && s == 2) return false;
-      if (w.g_sub > 0) { ++w.g_step; w.g_sub = 0; continue; }
-      *off = br.w_off[s]; *bytes = br.w_bytes[s]; *uses = ntv; w.g_sub = 1;
-      return true;
-    }
-  }
-
-  __device__ void issue_next(int s) {
-    uint32_t off, bytes;
-    int uses;
-    if (!next_load(s, &off, &bytes, &uses)) { ws[s].exhausted = true; return; }
-    bulk(off, bytes, P.s_w[s], &ctl->w_full[s]);
-    ws[s].inflight = true;
-    ws[s].cur_uses = uses;
-  }
-
-  __device__ void try_prefetch(int s) {
-    WSlot& w = ws[s];
-    if (w.uses_left != 0 || w.inflight || w.exhausted) return;
-    if (w.need_free) {
-      if (!ptx::mbar_try_wait(ptx::smem_u32(&ctl->w_free[s]), w.free_par)) return;
-      w.free_par ^= 1u;
-      w.need_free = false;
-    }
-    issue_next(s);
-  }
-
-  __device__ void acquire(int s) {
-    WSlot& w = ws[s];
-    if (w.uses_left != 0) return;
-    if (!w.inflight) {
-      if (w.need_free) { wait(&ctl->w_free[s], w.free_par); w.free_par ^= 1u; w.need_free = false; }
-      issue_next(s);
-    }
-    wait(&ctl->w_full[s], w.full_par);
-    w.full_par ^= 1u;
-    w.uses_left = w.cur_uses;
-    w.inflight = false;
-  }
-
-  __device__ void release(int s) {
-    WSlot& w = ws[s];
-    if (--w.uses_left == 0) {
-      ptx::umma_commit(ptx::smem_u32(&ctl->w_free[s]));
-      w.need_free = true;
-    }
-  }
-
-  __device__ void run(uint32_t tmem) {
-    for (int s = 0; s < 3; ++s) {
-      ws[s].full_par = ws[s].free_par = 0;
-      ws[s].uses_left = ws[s].cur_uses = 0;
-      ws[s].inflight = ws[s].need_free = ws[s].exhausted = false;
-      ws[s].g_step = ws[s].g_sub = 0;
-    }
-    for (int i = 0; i < st.nsteps && i < 2; ++i) {
-      const BlockRef& br = step_ref(P, st, i);
-      bulk(br.meta_off, br.meta_bytes, P.s_meta[i], &ctl->meta_full[i]);
-    }
-    for (int s = 0; s < 3; ++s) try_prefetch(s);
-
-    uint32_t apar[2] = {0u, 0u};
-    const int nslots = P.nslots;
-    for (int i = 0; i < st.nsteps; ++i) {
-      if (!wait(&ctl->meta_full[i & 1], (uint32_t)((i >> 1) & 1))) return;
-      const uint8_t* mb = smem + P.s_meta[i & 1];
-      const bool prior = st.is_prior(i);
-      int n[3], kd[3];
-      if (prior) {
-        const PriorMeta* M = reinterpret_cast<const PriorMeta*>(mb);
-        n[0] = M->n; kd[0] = M->kd;
-        n[1] = n[2] = kd[1] = kd[2] = 0;
-      } else {
-        const CouplingMeta* M = reinterpret_cast<const CouplingMeta*>(mb);
-        n[0] = M->n1; n[1] = M->n2; n[2] = M->n3;
-        kd[0] = M->kd1; kd[1] = M->kd2; kd[2] = M->kd3;
-      }
-      const int nstages = prior ? 1 : 3;
-      int tcur[2] = {0, 1}, stg[2] = {0, 0};
-      int remaining = ntv * nstages;
-      bool first = true;
-      uint32_t spin = 0;
-      while (remaining > 0) {
-        bool progress = false;
-        for (int s = 0; s < nslots; ++s) {
-          if (tcur[s] >= ntv) continue;
-          if (!ptx::mbar_try_wait(ptx::smem_u32(&ctl->a_ready[s]), apar[s])) continue;
-          apar[s] ^= 1u;
-          ptx::tc_fence_after();
-          if (first) {
-            // every worker has left step i-1, so its meta slot can take step i+1
-            first = false;
-            if (i >= 1 && i + 1 < st.nsteps) {
-              const BlockRef& br = step_ref(P, st, i + 1);
-              bulk(br.meta_off, br.meta_bytes, P.s_meta[(i + 1) & 1], &ctl->meta_full[(i + 1) & 1]);
-            }
-          }
-          const int stage = stg[s];
-          const int phys = prior ? 0 : ((stage == 2 && alias) ? 0 : stage);
-          acquire(phys);
-          const uint32_t d = tmem + (uint32_t)(s * kSlotCols);
-          const uint32_t sa = ptx::smem_u32(smem + P.s_a[s]);
-          const uint32_t sb = ptx::smem_u32(smem + P.s_w[phys]);
-          for (int n0 = 0; n0 < n[stage]; n0 += 256)
-            issue_gemm(d + (uint32_t)n0, sa, sb, n[stage], n0, min(256, n[stage] - n0), kd[stage]);
-          ptx::umma_commit(ptx::smem_u32(&ctl->d_ready[s]));
-          release(phys);
-          if (++stg[s] == nstages) { stg[s] = 0; tcur[s] += nslots; }
-          --remaining;
-          progress = true;
-        }
-        for (int s = 0; s < 3; ++s) try_prefetch(s);
-        if (progress) spin = 0;
-        else if (++spin > kSpinLimit || ctl->abort) {
-          if (!ctl->abort) { ctl->abort = 1; atomicExch(a.status, 1u); }
-          return;
-        }
-      }
-    }
-  }
-};
-
-// ---- workers ----------------------------------------------------------------------------------
+// ---- the level's steps ------------------------------------------------------------------------
 template <bool kInv>
-__device__ void run_workers(Ctx& cx, const LevelPlan& P, const LevelArgs& a, const Steps& st, int img0, int pvalid,
-                            int ntv) {
+__device__ void run_steps(Ctx& cx, const LevelPlan& P, const LevelArgs& a, const Steps& st, int img0, int pvalid,
+                          int ntv) {
   uint8_t* smem = cx.smem;
   Ctl* ctl = cx.ctl;
   int32_t* v = reinterpret_cast<int32_t*>(smem + P.s_v);
   int8_t* xa = reinterpret_cast<int8_t*>(smem + P.s_xa);
   int32_t* acc = reinterpret_cast<int32_t*>(smem + P.s_acc);
   uint8_t* sA = smem + P.s_a[cx.group];
-  const int pg = P.pg, ca = P.ca, cb = P.cb, w = P.w, h = P.h, px = P.px, cpad = P.cpad, cbp = P.cbp;
-  const int gthreads = (kWorkers / P.nslots);
-  uint64_t* a_ready = &ctl->a_ready[cx.group];
+  const uint32_t* rowinfo = reinterpret_cast<const uint32_t*>(smem + P.s_rowinfo);
+  const int pg = P.pg, ca = P.ca, cb = P.cb, w = P.w, cpad = P.cpad, cbp = P.cbp;
+  const uint32_t recip_a = P.recip_gpa, recip_b = P.recip_gpb;
+  const bool alias = P.w13_alias != 0;
   uint64_t* d_ready = &ctl->d_ready[cx.group];
   uint32_t dpar = 0;
   const CouplingMeta* prevM = nullptr;       // coupling whose translation is still to be applied
+  Weights W;
+  W.cur_step[0] = W.cur_step[1] = W.cur_step[2] = -1;
+  W.s0_loads = W.s0_used = 0;
 
-  auto arrive_a = [&]() {
+  if (cx.loader) {
+    for (int i = 0; i < st.nsteps && i < 2; ++i) {
+      const BlockRef& br = step_ref(P, st, i);
+      bulk_load(cx, a.blob, br.meta_off, br.meta_bytes, P.s_meta[i], &ctl->meta_full[i]);
+    }
+    top_up(cx, P, a, st, W, -1, alias);
+    if (alias && st.nsteps > 0) {
+      const BlockRef& br = step_ref(P, st, 0);
+      bulk_load(cx, a.blob, br.w_off[0], br.w_bytes[0], P.s_w[0], &ctl->w_full[0]);
+      W.s0_loads = 1;
+    }
+  }
+
+  // The group's A operand is written: hand it to the tensor core and wait for the accumulator.
+  //   slot: weight slot of this stage; k: ordinal of the load to wait for (first tile of the step
+  //   only, or every time in alias mode); n, kd: GEMM shape.
+  auto run_mma = [&](int slot, bool wait_w, uint32_t wpar, int n, int kd) {
     ptx::tc_fence_before();
     ptx::fence_async_smem();
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ptx::smem_u32(a_ready)) : "memory");
-  };
-  auto wait_d = [&]() {
+    group_barrier(cx.group, cx.gthreads);
+    if (cx.elected) {
+      if (wait_w) wait_bar(ctl, a.status, &ctl->w_full[slot], wpar);
+      ptx::tc_fence_after();
+      const uint32_t sa = ptx::smem_u32(sA), sb = ptx::smem_u32(smem + P.s_w[slot]);
+      for (int n0 = 0; n0 < n; n0 += 256) issue_gemm(cx.tmem_slot0 + (uint32_t)n0, sa, sb, n, n0, min(256, n - n0), kd);
+      ptx::umma_commit(ptx::smem_u32(d_ready));
+    }
     wait_bar(ctl, a.status, d_ready, dpar);
     dpar ^= 1u;
     ptx::tc_fence_after();
   };
+  // alias mode: S0 is free again (its MMA has completed): request its next matrix
+  auto s0_request = [&](const BlockRef& br, int which) {
+    bulk_load(cx, a.blob, br.w_off[which], br.w_bytes[which], P.s_w[0], &ctl->w_full[0]);
+    ++W.s0_loads;
+  };
+  auto s0_request_next_step = [&](int i) {
+    if (i + 1 < st.nsteps) s0_request(step_ref(P, st, i + 1), 0);
+  };
+
   // x_b +/-= rq(acc + bias) of the previous coupling for pixel p
   auto apply_translation = [&](int p) {
     const uint8_t* pm = reinterpret_cast<const uint8_t*>(prevM);
     const int32_t* colB = reinterpret_cast<const int32_t*>(pm + prevM->off_colB);
     const OutRq* orq = reinterpret_cast<const OutRq*>(pm + prevM->off_out);
-    for (int c = 0; c < cb; ++c) {
-      const OutRq o = orq[c];
-      const uint32_t t = (uint32_t)rq_exact(acc[c * pg + p] + o.bias, o.m0, o.s);
-      acc[c * pg + p] = 0;
-      uint32_t* vv = reinterpret_cast<uint32_t*>(&v[colB[c] * pg + p]);
-      *vv = kInv ? (*vv - t) : (*vv + t);
+    for (int c0 = 0; c0 < cb; c0 += 4) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int c = c0 + k;
+        if (c < cb) {
+          const OutRq o = orq[c];
+          const uint32_t t = (uint32_t)rq_exact(acc[c * pg + p] + o.bias, o.m0, o.s);
+          acc[c * pg + p] = 0;
+          uint32_t* vv = reinterpret_cast<uint32_t*>(&v[colB[c] * pg + p]);
+          *vv = kInv ? (*vv - t) : (*vv + t);
+        }
+      }
     }
   };
   // network input of pixel p: ca channels requantised to int8, padded to cpad bytes
@@ -507,57 +487,85 @@ __device__ void run_workers(Ctx& cx, const LevelPlan& P, const LevelArgs& a, con
     wait_bar(ctl, a.status, &ctl->meta_full[i & 1], (uint32_t)((i >> 1) & 1));
     const uint8_t* mb = smem + P.s_meta[i & 1];
     const bool prior = st.is_prior(i);
-    if (prior) {
-      const PriorMeta M = *reinterpret_cast<const PriorMeta*>(mb);
-      const OutRq* orq = reinterpret_cast<const OutRq*>(mb + M.off_out);
+    const CouplingMeta* Mp = reinterpret_cast<const CouplingMeta*>(mb);
+    const PriorMeta* Pp = reinterpret_cast<const PriorMeta*>(mb);
+    {
+      const int32_t* cols = prior ? P.col_out : reinterpret_cast<const int32_t*>(mb + Mp->off_colA);
+      const int32_t in_m0 = prior ? Pp->in_m0 : Mp->in_m0, in_s = prior ? Pp->in_s : Mp->in_s;
       for (int p = cx.tid; p < pvalid; p += kWorkers) {
         if (prevM) apply_translation(p);
-        requant_input(p, P.col_out, M.in_m0, M.in_s);
+        requant_input(p, cols, in_m0, in_s);
       }
-      prevM = nullptr;
-      worker_barrier();
+    }
+    prevM = prior ? nullptr : Mp;
+    worker_barrier();
+    // every thread has left step i-1: its meta slot can take step i+1
+    if (cx.loader && i >= 1 && i + 1 < st.nsteps) {
+      const BlockRef& br = step_ref(P, st, i + 1);
+      bulk_load(cx, a.blob, br.meta_off, br.meta_bytes, P.s_meta[(i + 1) & 1], &ctl->meta_full[(i + 1) & 1]);
+    }
+    const uint32_t par0 = (uint32_t)(load_ordinal(st, 0, i) & 1), par12 = (uint32_t)(load_ordinal(st, 1, i) & 1);
+    bool first = true;
+    if (prior) {
+      const PriorMeta M = *Pp;
+      const OutRq* orq = reinterpret_cast<const OutRq*>(mb + M.off_out);
       for (int t = cx.group; t < ntv; t += P.nslots) {
-        const RowPos rp = row_pos(t, cx.row, pvalid, px, h, w);
-        build_im2col(cx, sA, xa, cpad, w, M.kd, rp);
-        arrive_a();
-        wait_d();
+        const RowPos rp = row_pos(rowinfo, t, cx.row);
+        build_im2col(cx, sA, xa, cpad, w, M.kd, recip_a, rp);
+        if (alias) {
+          run_mma(0, first, W.s0_used & 1u, M.n, M.kd);
+          if (first) ++W.s0_used;
+          if (cx.loader && t + P.nslots >= ntv) s0_request_next_step(i);
+        } else {
+          run_mma(0, first, par0, M.n, M.kd);
+        }
+        first = false;
         epilogue_prior(cx, P, a, M, orq, img0, rp);
       }
-      worker_barrier();
-      continue;
-    }
-    const CouplingMeta* Mp = reinterpret_cast<const CouplingMeta*>(mb);
-    const CouplingMeta M = *Mp;
-    const int32_t* colA = reinterpret_cast<const int32_t*>(mb + M.off_colA);
-    const HiddenRq* h1 = reinterpret_cast<const HiddenRq*>(mb + M.off_h1);
-    const HiddenRq* h2 = reinterpret_cast<const HiddenRq*>(mb + M.off_h2);
-    for (int p = cx.tid; p < pvalid; p += kWorkers) {
-      if (prevM) apply_translation(p);
-      requant_input(p, colA, M.in_m0, M.in_s);
-    }
-    prevM = Mp;
-    worker_barrier();
-    for (int t = cx.group; t < ntv; t += P.nslots) {
-      const RowPos rp = row_pos(t, cx.row, pvalid, px, h, w);
-      build_im2col(cx, sA, xa, cpad, w, M.kd1, rp);
-      arrive_a();
-      wait_d();
-      epilogue_hidden(cx, M.fast1, M.n1, M.kd2, h1, M.lo1, M.hi1, sA);
-      arrive_a();
-      wait_d();
-      epilogue_hidden(cx, M.fast2, M.n2, M.kd3, h2, M.lo2, M.hi2, sA);
-      arrive_a();
-      wait_d();
-      epilogue_scatter(cx, cb, cbp, acc, pg, w, rp);
+    } else {
+      const CouplingMeta M = *Mp;
+      const HiddenRq* h1 = reinterpret_cast<const HiddenRq*>(mb + M.off_h1);
+      const HiddenRq* h2 = reinterpret_cast<const HiddenRq*>(mb + M.off_h2);
+      const int2* u1 = reinterpret_cast<const int2*>(mb + M.off_u1);
+      const int2* u2 = reinterpret_cast<const int2*>(mb + M.off_u2);
+      const BlockRef& br = step_ref(P, st, i);
+      for (int t = cx.group; t < ntv; t += P.nslots) {
+        const bool last_tile = t + P.nslots >= ntv;
+        const RowPos rp = row_pos(rowinfo, t, cx.row);
+        build_im2col(cx, sA, xa, cpad, w, M.kd1, recip_a, rp);
+        if (alias) {
+          run_mma(0, true, W.s0_used & 1u, M.n1, M.kd1);
+          ++W.s0_used;
+          if (cx.loader) s0_request(br, 2);
+        } else {
+          run_mma(0, first, par0, M.n1, M.kd1);
+        }
+        epilogue_hidden(cx, M.mode1, M.us1, M.n1, M.kd2, h1, u1, M.lo1, M.hi1, sA);
+        run_mma(1, first, par12, M.n2, M.kd2);
+        epilogue_hidden(cx, M.mode2, M.us2, M.n2, M.kd3, h2, u2, M.lo2, M.hi2, sA);
+        if (alias) {
+          run_mma(0, true, W.s0_used & 1u, M.n3, M.kd3);
+          ++W.s0_used;
+          if (cx.loader) {
+            if (last_tile) s0_request_next_step(i);
+            else s0_request(br, 0);
+          }
+        } else {
+          run_mma(2, first, par12, M.n3, M.kd3);
+        }
+        first = false;
+        epilogue_scatter(cx, cb, cbp, recip_b, acc, pg, w, rp);
+      }
     }
     ptx::tc_fence_before();
     worker_barrier();
+    // every MMA of step i has completed (each group waited for its last accumulator)
+    if (cx.loader) top_up(cx, P, a, st, W, i, alias);
   }
   if (prevM) {
     for (int p = cx.tid; p < pvalid; p += kWorkers) apply_translation(p);
     worker_barrier();
   }
-  (void)gthreads;
 }
 
 template <bool kInv>
@@ -566,19 +574,14 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
   __shared__ Ctl ctl;
   const LevelPlan& P = *a.plan;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const bool is_worker = warp < kWorkerWarps;
   const int wpg = kWorkerWarps / P.nslots;       // warps per group
 
   if (tid == 0) {
     for (int s = 0; s < 2; ++s) {
-      ptx::mbar_init(ptx::smem_u32(&ctl.a_ready[s]), (uint32_t)(wpg * 32));
       ptx::mbar_init(ptx::smem_u32(&ctl.d_ready[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&ctl.meta_full[s]), 1);
     }
-    for (int s = 0; s < 3; ++s) {
-      ptx::mbar_init(ptx::smem_u32(&ctl.w_full[s]), 1);
-      ptx::mbar_init(ptx::smem_u32(&ctl.w_free[s]), 1);
-    }
+    for (int s = 0; s < 3; ++s) ptx::mbar_init(ptx::smem_u32(&ctl.w_full[s]), 1);
     ptx::mbar_init_fence();
     ctl.abort = 0;
   }
@@ -602,12 +605,7 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
   st.nsteps = P.n_couplings + (st.do_prior ? 1 : 0);
   st.inverse = kInv;
 
-  if (!is_worker) {
-    if (lane == 0) {
-      Control ctrl{P, a, smem, &ctl, st, ntv, P.w13_alias != 0};
-      ctrl.run(tmem);
-    }
-  } else {
+  {
     Ctx cx;
     cx.smem = smem;
     cx.ctl = &ctl;
@@ -619,11 +617,17 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
     cx.group = warp / wpg;
     cx.cs = (warp % wpg) >> 2;
     cx.ncs = wpg >> 2;
+    cx.gthreads = wpg * 32;
     cx.row = cx.wq * 32 + lane;
-    cx.tmem_slot = tmem + ((uint32_t)(cx.wq * 32) << 16) + (uint32_t)(cx.group * kSlotCols);
+    cx.elected = (warp % wpg) == 0 && lane == 0;
+    cx.loader = tid == 0;
+    cx.tmem_slot0 = tmem + (uint32_t)(cx.group * kSlotCols);
+    cx.tmem_slot = cx.tmem_slot0 + ((uint32_t)(cx.wq * 32) << 16);
 
     int32_t* acc = reinterpret_cast<int32_t*>(smem + P.s_acc);
     for (int idx = tid; idx < P.cb * pg; idx += kWorkers) acc[idx] = 0;
+    uint32_t* rowinfo = reinterpret_cast<uint32_t*>(smem + P.s_rowinfo);
+    for (int idx = tid; idx < P.tiles * kTileM; idx += kWorkers) rowinfo[idx] = row_record(idx, pvalid, px, P.h, w);
     if (!kInv) {
       // space-to-depth on load: plane c*4 + dy*2 + dx, pixel (i, j) <- in[c][2i+dy][2j+dx]
       const int w2 = 2 * w;
@@ -650,7 +654,7 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
     }
     worker_barrier();
 
-    run_workers<kInv>(cx, P, a, st, img0, pvalid, ntv);
+    run_steps<kInv>(cx, P, a, st, img0, pvalid, ntv);
 
     if (!kInv) {
       // split on store: factored-out half -> z block of this level; kept half -> next level (or
