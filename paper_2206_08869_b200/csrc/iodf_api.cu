@@ -452,7 +452,10 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
   }
 
   // device objects
-  CU(m, configure_level_kernels(max_smem));
+  // The attribute belongs to the kernel, not to a model: always raise it to the device maximum so
+  // that creating a second, smaller model cannot lower it under a first model's needs.
+  (void)max_smem;
+  CU(m, configure_level_kernels((uint32_t)smem_limit));
   const size_t L = desc->n_levels;
   m->d_plan.assign(L, nullptr); m->d_blob.assign(L, nullptr); m->d_keep.assign(L, nullptr);
   for (size_t li = 0; li < L; ++li) {

@@ -89,12 +89,6 @@ __device__ __forceinline__ int32_t rq_exact(int32_t a, int32_t m0, int32_t s) {
 
 __device__ __forceinline__ int clampi(int v, int lo, int hi) { return min(max(v, lo), hi); }
 
-__device__ __forceinline__ int min_relu(int v, int hi) {
-  int r;
-  asm("min.relu.s32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(hi));
-  return r;
-}
-
 __device__ __forceinline__ uint32_t pack4(int y0, int y1, int y2, int y3) {
   const uint32_t a = __byte_perm((uint32_t)y0, (uint32_t)y1, 0x0040);
   const uint32_t b = __byte_perm((uint32_t)y2, (uint32_t)y3, 0x0040);
