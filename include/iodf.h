@@ -44,7 +44,8 @@ typedef enum {
   IODF_EVERSION = -4,     /* abi_version mismatch                                                    */
   IODF_ETIMEOUT = -5,     /* a bounded device-side wait gave up (reported by iodf_check)             */
   IODF_EUNSUPPORTED = -6, /* a valid model whose shape this build cannot run (see iodf_create)       */
-  IODF_EOVERFLOW = -7     /* a worst-case accumulator |sum| + |bias| would leave the int32 range     */
+  IODF_EOVERFLOW = -7,    /* a worst-case accumulator |sum| + |bias| would leave the int32 range     */
+  IODF_ELIMIT = -8        /* the request needs more than the fixed scratch of iodf_forward_static   */
 } iodf_status;
 
 /*
@@ -180,6 +181,36 @@ int iodf_forward_timed(iodf_model* m, const uint8_t* x_u8, int B, int32_t* z, in
                        float* level_ms);
 int iodf_inverse_timed(iodf_model* m, const int32_t* z, int B, uint8_t* x_u8, int32_t* prior,
                        uint32_t* out_of_range_count, void* cuda_stream, float* level_ms);
+
+/*
+ * Encode without touching any allocator (the paper has no counterpart; this exists for deployment).
+ *
+ * iodf_forward hands the kept channels from one level's kernel to the next through a workspace
+ * that iodf_create sized with cudaMalloc for the model's max_batch. Some callers cannot have that:
+ * a plug-in inside a host process that owns the device memory pool and forbids allocation, a
+ * service whose model object was created for a small max_batch and which later sees a larger
+ * batch at a point where allocating is not allowed (inside a latency-critical loop, or after the
+ * rest of the device memory has been handed out). For them this entry point does the same encode,
+ * with identical results, but keeps the inter-level data in a fixed array that is part of the
+ * library image itself: IODF_STATIC_SCRATCH_BYTES of device memory on every GPU that loads the
+ * library, held until the process exits. It calls no allocation or free routine of any kind.
+ *
+ * Limits and rules
+ *   - B is NOT limited by the model's max_batch but by the array: the call needs
+ *     B * iodf_static_scratch_bytes_per_image(m) bytes and returns IODF_ELIMIT if that exceeds
+ *     IODF_STATIC_SCRATCH_BYTES (nothing is launched).
+ *   - The first call on a device looks up the array's device address (once per device, with the
+ *     model's device made current for the lookup). Make that first call before any stream capture.
+ *   - All calls, for all models on the device, share the one array; it keeps whatever the last
+ *     call left in it. Nothing in it needs to start at zero (every level writes its part before the
+ *     next level reads it), but two calls that overlap on the GPU (different streams, or this
+ *     entry point from two threads without ordering) race on it. Serialise them on one stream.
+ *   - x_u8, z, prior: DEV, as for iodf_forward.
+ */
+#define IODF_STATIC_SCRATCH_BYTES (8u * 1024u * 1024u)
+int iodf_forward_static(iodf_model* m, const uint8_t* x_u8, int B, int32_t* z, int32_t* prior, void* cuda_stream);
+/* Bytes of the fixed array one image needs for this model (0 for a single-level model). */
+size_t iodf_static_scratch_bytes_per_image(const iodf_model* m);
 
 /* Number of kernel launches one iodf_forward / iodf_inverse call enqueues. */
 int iodf_launches_per_call(const iodf_model* m, int inverse);

@@ -12,7 +12,8 @@ IODF_ABI_VERSION = 1
 IODF_MAX_LEVELS = 8
 
 DECLARED_SYMBOLS = ["iodf_create", "iodf_destroy", "iodf_get_layout", "iodf_forward", "iodf_inverse",
-                    "iodf_forward_host", "iodf_inverse_host", "iodf_forward_timed", "iodf_inverse_timed", "iodf_check", "iodf_launches_per_call",
+                    "iodf_forward_host", "iodf_inverse_host", "iodf_forward_timed", "iodf_inverse_timed", "iodf_forward_static",
+                    "iodf_static_scratch_bytes_per_image", "iodf_check", "iodf_launches_per_call",
                     "iodf_strerror", "iodf_last_cuda_error"]
 
 
@@ -84,6 +85,10 @@ def load_library(path=None):
     L.iodf_forward_timed.argtypes = [vp, vp, C.c_int, vp, vp, vp, C.POINTER(C.c_float)]
     L.iodf_inverse_timed.restype = C.c_int
     L.iodf_inverse_timed.argtypes = [vp, vp, C.c_int, vp, vp, vp, vp, C.POINTER(C.c_float)]
+    L.iodf_forward_static.restype = C.c_int
+    L.iodf_forward_static.argtypes = [vp, vp, C.c_int, vp, vp, vp]
+    L.iodf_static_scratch_bytes_per_image.restype = C.c_size_t
+    L.iodf_static_scratch_bytes_per_image.argtypes = [vp]
     L.iodf_check.restype = C.c_int
     L.iodf_check.argtypes = [vp, vp]
     L.iodf_launches_per_call.restype = C.c_int
@@ -258,6 +263,22 @@ def iodf_inverse_timed(model, z, x_u8, prior=None, out_of_range=None, stream=Non
     if rc != 0:
         raise IodfError(rc, "iodf_inverse_timed")
     return list(ms)
+
+
+IODF_STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
+
+
+def iodf_static_scratch_bytes_per_image(model):
+    return int(load_library().iodf_static_scratch_bytes_per_image(model.handle))
+
+
+def iodf_forward_static(model, x_u8, z, prior=None, stream=None):
+    """Encode using the library's fixed scratch array instead of the model's allocated workspace.
+    The caller passes every buffer (this wrapper allocates nothing either)."""
+    rc = load_library().iodf_forward_static(model.handle, _ptr(x_u8), x_u8.shape[0], _ptr(z), _ptr(prior),
+                                            _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_forward_static")
 
 
 def iodf_check(model, stream=None):

@@ -3,8 +3,10 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -539,6 +541,94 @@ int read_level_times(iodf_model* m, cudaStream_t st, bool inverse, float* level_
 
 }  // namespace
 
+// ---- allocation-free encode -----------------------------------------------------------------------
+// Fixed inter-level scratch for iodf_forward_static. In host code `g_static_scratch` is only a
+// handle for the symbol, not a device address: the address is looked up once per device with
+// cudaGetSymbolAddress and that pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_static_scratch[IODF_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+unsigned char* g_scratch_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the static scratch on `device` (looked up on first use, cached afterwards).
+int static_scratch_address(iodf_model* m, int device, unsigned char** out) {
+  if (device < 0 || device >= kMaxDevices) return IODF_EINVAL;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_ptr[device]) {
+    int prev = -1;
+    CU(m, cudaGetDevice(&prev));
+    CU(m, cudaSetDevice(device));
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+    cudaError_t e2 = cudaSetDevice(prev);
+    if (e != cudaSuccess) return cuda_fail(m, e);
+    if (e2 != cudaSuccess) return cuda_fail(m, e2);
+    if (!p) return IODF_ECUDA;
+    g_scratch_ptr[device] = static_cast<unsigned char*>(p);
+  }
+  *out = g_scratch_ptr[device];
+  return IODF_OK;
+}
+
+size_t static_bytes_per_image(const iodf_model* m) {
+  size_t bytes = 0;
+  for (size_t li = 0; li + 1 < m->levels.size(); ++li) {
+    const LevelPlan& P = m->levels[li].plan;
+    bytes += ((size_t)P.keep_c * P.px * sizeof(int32_t) + 255) / 256 * 256;
+  }
+  return bytes;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t iodf_static_scratch_bytes_per_image(const iodf_model* m) { return m ? static_bytes_per_image(m) : 0; }
+
+int iodf_forward_static(iodf_model* m, const uint8_t* x_u8, int B, int32_t* z, int32_t* prior, void* cuda_stream) {
+  if (!m || !x_u8 || !z || B < 1) return IODF_EINVAL;
+  if (!aligned16(x_u8) || !aligned16(z) || !aligned16(prior)) return IODF_EINVAL;
+  const size_t per_image = static_bytes_per_image(m);
+  if ((size_t)B > (size_t)IODF_STATIC_SCRATCH_BYTES / (per_image ? per_image : 1) && per_image) return IODF_ELIMIT;
+  unsigned char* base = nullptr;
+  int rc = static_scratch_address(m, m->device, &base);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int32_t* prior_arg = m->layout.d_fact ? prior : nullptr;
+  // the kept channels of level l live at keep[l] inside the fixed array, sized for this call's B
+  const size_t L = m->levels.size();
+  int32_t* keep[IODF_MAX_LEVELS];
+  size_t off = 0;
+  for (size_t li = 0; li < L; ++li) {
+    keep[li] = reinterpret_cast<int32_t*>(base + off);
+    if (li + 1 < L) {
+      const LevelPlan& P = m->levels[li].plan;
+      off += ((size_t)P.keep_c * P.px * sizeof(int32_t) + 255) / 256 * 256 * (size_t)B;
+    }
+  }
+  for (size_t li = 0; li < L; ++li) {
+    const LevelPlan& P = m->levels[li].plan;
+    LevelArgs a{};
+    a.plan = m->d_plan[li];
+    a.blob = m->d_blob[li];
+    a.in = li == 0 ? (const void*)x_u8 : (const void*)keep[li - 1];
+    a.in_stride = 0;
+    a.z = z;
+    a.prior = prior_arg;
+    a.out = keep[li];
+    a.oor = nullptr;
+    a.status = m->d_status;
+    a.batch = B;
+    CU(m, launch_level(a, false, (B + P.group - 1) / P.group, P.s_total, st));
+  }
+  return IODF_OK;
+}
+
+}  // extern "C"
+
 extern "C" {
 
 int iodf_create(const iodf_model_desc* desc, const int8_t* weights, size_t weights_count, const int32_t* requant,
@@ -667,6 +757,7 @@ const char* iodf_strerror(int status) {
     case IODF_ETIMEOUT: return "a bounded device-side wait gave up";
     case IODF_EUNSUPPORTED: return "model shape not supported by this build";
     case IODF_EOVERFLOW: return "worst-case accumulator leaves the int32 range";
+    case IODF_ELIMIT: return "request exceeds the fixed scratch of iodf_forward_static";
     default: return "unknown status";
   }
 }
