@@ -21,7 +21,7 @@ namespace iodf {
 constexpr int kTileM = 128;          // pixels per MMA tile (UMMA M)
 constexpr int kWorkerWarps = 16;     // four per TMEM lane quarter
 constexpr int kWorkers = kWorkerWarps * 32;
-constexpr int kThreads = kWorkers;
+constexpr int kThreads = kWorkers + 32;   // + one control warp (bulk copies and MMA issue)
 constexpr int kMaxCouplings = 32;    // per level
 constexpr int kMaxC = 256;           // flow channels per level
 constexpr int kMaxHidden = 256;      // kept hidden channels per layer (padded)

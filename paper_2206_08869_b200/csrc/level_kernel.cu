@@ -24,12 +24,15 @@
 // coupling addresses v through its table of physical columns (the composition of all permutations
 // so far), and the level's outputs are written through the final table.
 //
-// Execution structure: 16 warps form one or two groups; each group owns a tile slot (an A-operand
-// buffer in shared memory and a range of TMEM columns) and walks its tiles through build ->
-// epilogue 1 -> epilogue 2 -> scatter. Between stages the group meets at a named barrier, one
-// elected thread issues the stage's MMAs and commits them to the slot's mbarrier, and the group
-// waits on it; so while one group requantises, the tensor core works for the other. One thread
-// of the CTA also issues the bulk copies that bring the next coupling's weights in.
+// Execution structure: 16 worker warps and one control warp. All workers work on the same phase
+// of one tile (four warps per TMEM lane quarter split the columns four ways). Two tiles are in
+// flight, each with its own A-operand buffer and TMEM columns, and their phases alternate:
+// build(A) build(B) epi1(A) epi1(B) epi2(A) epi2(B) scatter(A) scatter(B). A worker that has
+// finished its part of a phase arrives on the tile's "A ready" mbarrier and goes straight on to the
+// other tile's phase (after waiting for that tile's accumulator); the control thread waits for the
+// arrivals, issues the tile's next MMAs and commits them to the tile's "D ready" mbarrier. So the
+// tensor core always works under a requantisation phase and no worker waits for an MMA issue. The
+// control thread also issues the bulk copies that bring the next coupling's weights in.
 #include "iodf_dev.h"
 #include "level_kernel.h"
 #include "ptx.cuh"
@@ -39,7 +42,8 @@ namespace iodf {
 namespace {
 
 struct __align__(16) Ctl {
-  uint64_t d_ready[2];    // tensor core -> group: the slot's accumulator is complete
+  uint64_t a_ready[2];    // workers -> control: the tile slot's A operand is written (count = workers)
+  uint64_t d_ready[2];    // tensor core -> workers: the tile slot's accumulator is complete
   uint64_t w_full[3];     // bulk copy -> elected threads: weight slot filled
   uint64_t meta_full[2];  // bulk copy -> everyone: meta block of step (i & 1) has landed
   uint32_t tmem_base;
@@ -52,13 +56,10 @@ struct Ctx {
   uint32_t* status;
   int tid, warp, lane;
   int wq;                 // TMEM lane quarter of this warp
-  int group, cs, ncs;     // tile slot, column-split index and count inside the group
-  int gthreads;           // threads per group
+  int cs, ncs;            // column-split index and count
   int row;                // tile row (= TMEM lane) of this thread
-  bool elected;           // issues this group's MMAs
-  bool loader;            // issues the CTA's bulk copies (the elected thread of group 0)
-  uint32_t tmem_slot;     // TMEM address of the slot's first column, this warp's lane quarter
-  uint32_t tmem_slot0;    // the same with lane field 0 (MMA destination)
+  uint32_t tmem_base;     // first allocated TMEM column, lane field 0
+  uint32_t tmem_slot;     // current tile slot's first column, this warp's lane quarter
 };
 
 // Bounded wait on an mbarrier phase. After one wait in the CTA has given up, every later wait
@@ -76,10 +77,8 @@ __device__ __noinline__ bool wait_bar(Ctl* ctl, uint32_t* status, uint64_t* bar,
   return false;
 }
 
-__device__ __forceinline__ void worker_barrier() { __syncthreads(); }
-__device__ __forceinline__ void group_barrier(int group, int nthreads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(group + 1), "r"(nthreads) : "memory");
-}
+__device__ __forceinline__ void cta_barrier() { __syncthreads(); }
+
 
 __device__ __forceinline__ int32_t rq_exact(int32_t a, int32_t m0, int32_t s) {
   const long long p = (long long)a * (long long)m0 + (1ll << (30 + s));
@@ -256,33 +255,48 @@ __device__ __forceinline__ void epilogue_hidden(const Ctx& cx, int mode, int us,
   }
 }
 
-// Per-tap partial products -> shifted sum into the translation accumulator. Column granule gi
-// (8 columns) belongs to tap gi / (cbp/8) and out channels (gi % (cbp/8))*8 .. +8. Loads are
-// issued four granules at a time.
-__device__ void epilogue_scatter(const Ctx& cx, int cb, int cbp, uint32_t recip_gpt, int32_t* __restrict__ acc, int pg,
-                                 int w, const RowPos rp) {
+// Per-tap partial products -> shifted sum into the translation accumulator.
+// Column granule (tap, gq) holds out channels gq*8 .. gq*8+8 of that tap. The partial product of
+// pixel p and tap (du, dv) belongs to output pixel p - (du-1)*w - (dv-1). Consecutive lanes hold
+// consecutive pixels, so the three dv-contributions that meet in one output pixel sit in lanes
+// L-1, L, L+1: they are summed with two warp shuffles, and one shared-memory atomic per (du,
+// channel) adds the row sum. A warp's two edge lanes add their outward contribution themselves.
+// Masked contributions (target outside the image) are zero before the shuffle. Work unit =
+// (du, gq); units are dealt round-robin to the column splits.
+__device__ void epilogue_scatter(const Ctx& cx, int cb, int cbp, int32_t* __restrict__ acc, int pg, int w,
+                                 const RowPos rp) {
   const int gpt = cbp >> 3;
-  const int ngran = 9 * gpt;
-  for (int g0 = cx.cs; g0 < ngran; g0 += 4 * cx.ncs) {
-    uint32_t r[4][8];
+  const int nunits = 3 * gpt;
+  const uint32_t sm = rp.valid ? rp.smask : 0u;
+  for (int u = cx.cs; u < nunits; u += cx.ncs) {
+    const int du = (u >= 2 * gpt) ? 2 : ((u >= gpt) ? 1 : 0);
+    const int gq = u - du * gpt;
+    uint32_t r0[8], r1[8], r2[8];
+    ptx::tmem_ld8(cx.tmem_slot + (uint32_t)(((du * 3 + 0) * gpt + gq) << 3), r0);
+    ptx::tmem_ld8(cx.tmem_slot + (uint32_t)(((du * 3 + 1) * gpt + gq) << 3), r1);
+    ptx::tmem_ld8(cx.tmem_slot + (uint32_t)(((du * 3 + 2) * gpt + gq) << 3), r2);
+    ptx::tmem_ld_wait8(r0);
+    ptx::tmem_ld_wait8(r1);
+    ptx::tmem_ld_wait8(r2);
+    const bool ok_m = ((sm >> (du * 3 + 0)) & 1u) != 0;   // dv = -1: target column j + 1
+    const bool ok_0 = ((sm >> (du * 3 + 1)) & 1u) != 0;   // dv =  0: target column j
+    const bool ok_p = ((sm >> (du * 3 + 2)) & 1u) != 0;   // dv = +1: target column j - 1
+    const int c0 = gq << 3;
+    int32_t* dst = acc + c0 * pg + rp.p - (du - 1) * w;   // this lane's own output pixel for this du
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int gi = g0 + k * cx.ncs;
-      if (gi < ngran) ptx::tmem_ld8(cx.tmem_slot + (uint32_t)(gi << 3), r[k]);
-    }
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int gi = g0 + k * cx.ncs;
-      if (gi < ngran) {
-        ptx::tmem_ld_wait8(r[k]);
-        const int tap = (int)(((uint32_t)gi * recip_gpt) >> 16);
-        const int c0 = (gi - tap * gpt) << 3;
-        if (rp.valid && ((rp.smask >> tap) & 1u)) {
-          int32_t* dst = acc + c0 * pg + rp.p - tap_offset(tap, w);
-#pragma unroll
-          for (int i = 0; i < 8; ++i)
-            if (c0 + i < cb) atomicAdd(dst + i * pg, (int32_t)r[k][i]);
-        }
+    for (int i = 0; i < 8; ++i) {
+      if (c0 + i < cb) {                                  // uniform across the warp
+        const int v_m = ok_m ? (int)r0[i] : 0;
+        const int v_0 = ok_0 ? (int)r1[i] : 0;
+        const int v_p = ok_p ? (int)r2[i] : 0;
+        const int from_next = __shfl_down_sync(0xFFFFFFFFu, v_p, 1);   // lane L+1's dv=+1 lands here
+        const int from_prev = __shfl_up_sync(0xFFFFFFFFu, v_m, 1);     // lane L-1's dv=-1 lands here
+        int sum = v_0;
+        if (cx.lane < 31) sum += from_next;
+        if (cx.lane > 0) sum += from_prev;
+        if (sum != 0) atomicAdd(dst + i * pg, sum);
+        if (cx.lane == 31 && v_m != 0) atomicAdd(dst + i * pg + 1, v_m);
+        if (cx.lane == 0 && v_p != 0) atomicAdd(dst + i * pg - 1, v_p);
       }
     }
   }
@@ -332,13 +346,22 @@ __device__ __forceinline__ const BlockRef& step_ref(const LevelPlan& P, const St
 
 // ---- MMA issue and weight traffic (elected threads) --------------------------------------------
 // D[128 x n] (+)= A[128 x kd] * B[n x kd]^T for B rows n0..n0+n of a matrix with n_total rows.
-__device__ void issue_gemm(uint32_t d_tmem, uint32_t sa, uint32_t sb, int n_total, int n0, int n, int kd) {
+// The control thread competes for issue slots with sixteen busy worker warps, so the loop body is
+// kept to the MMA and two descriptor increments (K advances by 32 bytes = two 16-byte chunks).
+__device__ __forceinline__ void issue_gemm(uint32_t d_tmem, uint32_t sa, uint32_t sb, int n_total, int n0, int n,
+                                           int kd) {
   const uint32_t idesc = ptx::umma_idesc_s8((uint32_t)n);
   const uint32_t lbo_b = (uint32_t)n_total * 16u;
-  for (int k = 0; k < (kd >> 5); ++k) {
-    const uint64_t da = ptx::umma_desc(sa + (uint32_t)k * 2u * (kTileM * 16), kTileM * 16, 128);
-    const uint64_t db = ptx::umma_desc(sb + (uint32_t)n0 * 16u + (uint32_t)k * 2u * lbo_b, lbo_b, 128);
-    ptx::umma_i8(d_tmem, da, db, idesc, k > 0 ? 1u : 0u);
+  uint64_t da = ptx::umma_desc(sa, kTileM * 16, 128);
+  uint64_t db = ptx::umma_desc(sb + (uint32_t)n0 * 16u, lbo_b, 128);
+  const uint64_t da_step = (uint64_t)((2u * kTileM * 16u) >> 4);
+  const uint64_t db_step = (uint64_t)((2u * lbo_b) >> 4);
+  const int ksteps = kd >> 5;
+  ptx::umma_i8_first(d_tmem, da, db, idesc);
+  for (int k = 1; k < ksteps; ++k) {
+    da += da_step;
+    db += db_step;
+    ptx::umma_i8_acc(d_tmem, da, db, idesc);
   }
 }
 
@@ -383,28 +406,21 @@ __device__ void top_up(const Ctx& cx, const LevelPlan& P, const LevelArgs& a, co
   }
 }
 
-// ---- the level's steps ------------------------------------------------------------------------
-template <bool kInv>
-__device__ void run_steps(Ctx& cx, const LevelPlan& P, const LevelArgs& a, const Steps& st, int img0, int pvalid,
-                          int ntv) {
+// ---- control thread -----------------------------------------------------------------------------
+// Issues, in the fixed order in which the workers produce them, the MMAs of every tile phase, and
+// keeps the weight and meta slots filled. Takes part in the two CTA barriers of every step.
+__device__ void run_control(const Ctx& cx, const LevelPlan& P, const LevelArgs& a, const Steps& st, int ntv) {
   uint8_t* smem = cx.smem;
   Ctl* ctl = cx.ctl;
-  int32_t* v = reinterpret_cast<int32_t*>(smem + P.s_v);
-  int8_t* xa = reinterpret_cast<int8_t*>(smem + P.s_xa);
-  int32_t* acc = reinterpret_cast<int32_t*>(smem + P.s_acc);
-  uint8_t* sA = smem + P.s_a[cx.group];
-  const uint32_t* rowinfo = reinterpret_cast<const uint32_t*>(smem + P.s_rowinfo);
-  const int pg = P.pg, ca = P.ca, cb = P.cb, w = P.w, cpad = P.cpad, cbp = P.cbp;
-  const uint32_t recip_a = P.recip_gpa, recip_b = P.recip_gpb;
+  const bool lead = cx.lane == 0;
   const bool alias = P.w13_alias != 0;
-  uint64_t* d_ready = &ctl->d_ready[cx.group];
-  uint32_t dpar = 0;
-  const CouplingMeta* prevM = nullptr;       // coupling whose translation is still to be applied
+  const int nslots = P.nslots;
+  uint32_t apar[2] = {0u, 0u}, dpar[2] = {0u, 0u};
   Weights W;
   W.cur_step[0] = W.cur_step[1] = W.cur_step[2] = -1;
   W.s0_loads = W.s0_used = 0;
 
-  if (cx.loader) {
+  if (lead) {
     for (int i = 0; i < st.nsteps && i < 2; ++i) {
       const BlockRef& br = step_ref(P, st, i);
       bulk_load(cx, a.blob, br.meta_off, br.meta_bytes, P.s_meta[i], &ctl->meta_full[i]);
@@ -416,32 +432,120 @@ __device__ void run_steps(Ctx& cx, const LevelPlan& P, const LevelArgs& a, const
       W.s0_loads = 1;
     }
   }
-
-  // The group's A operand is written: hand it to the tensor core and wait for the accumulator.
-  //   slot: weight slot of this stage; k: ordinal of the load to wait for (first tile of the step
-  //   only, or every time in alias mode); n, kd: GEMM shape.
-  auto run_mma = [&](int slot, bool wait_w, uint32_t wpar, int n, int kd) {
-    ptx::tc_fence_before();
-    ptx::fence_async_smem();
-    group_barrier(cx.group, cx.gthreads);
-    if (cx.elected) {
-      if (wait_w) wait_bar(ctl, a.status, &ctl->w_full[slot], wpar);
-      ptx::tc_fence_after();
-      const uint32_t sa = ptx::smem_u32(sA), sb = ptx::smem_u32(smem + P.s_w[slot]);
-      for (int n0 = 0; n0 < n; n0 += 256) issue_gemm(cx.tmem_slot0 + (uint32_t)n0, sa, sb, n, n0, min(256, n - n0), kd);
-      ptx::umma_commit(ptx::smem_u32(d_ready));
-    }
-    wait_bar(ctl, a.status, d_ready, dpar);
-    dpar ^= 1u;
+  // wait for tile slot sl's A operand, then D = A * W^T into the slot's TMEM columns
+  auto mma = [&](int sl, int wslot, bool wait_w, uint32_t wpar, int n, int kd) {
+    wait_bar(ctl, a.status, &ctl->a_ready[sl], apar[sl]);
+    apar[sl] ^= 1u;
+    if (wait_w) wait_bar(ctl, a.status, &ctl->w_full[wslot], wpar);
     ptx::tc_fence_after();
+    const uint32_t sa = ptx::smem_u32(smem + P.s_a[sl]), sb = ptx::smem_u32(smem + P.s_w[wslot]);
+    const uint32_t d = cx.tmem_base + (uint32_t)(sl * kSlotCols);
+    for (int n0 = 0; n0 < n; n0 += 256) issue_gemm(d + (uint32_t)n0, sa, sb, n, n0, min(256, n - n0), kd);
+    ptx::umma_commit(ptx::smem_u32(&ctl->d_ready[sl]));
   };
-  // alias mode: S0 is free again (its MMA has completed): request its next matrix
-  auto s0_request = [&](const BlockRef& br, int which) {
+  // alias mode only: wait until the MMA just issued for slot 0 has completed, then refill S0
+  auto s0_refill = [&](const BlockRef& br, int which) {
+    wait_bar(ctl, a.status, &ctl->d_ready[0], dpar[0]);
     bulk_load(cx, a.blob, br.w_off[which], br.w_bytes[which], P.s_w[0], &ctl->w_full[0]);
     ++W.s0_loads;
   };
-  auto s0_request_next_step = [&](int i) {
-    if (i + 1 < st.nsteps) s0_request(step_ref(P, st, i + 1), 0);
+
+  for (int i = 0; i < st.nsteps; ++i) {
+    const bool prior = st.is_prior(i);
+    int n[3] = {0, 0, 0}, kd[3] = {0, 0, 0};
+    if (lead) {
+      wait_bar(ctl, a.status, &ctl->meta_full[i & 1], (uint32_t)((i >> 1) & 1));
+      const uint8_t* mb = smem + P.s_meta[i & 1];
+      if (prior) {
+        const PriorMeta* M = reinterpret_cast<const PriorMeta*>(mb);
+        n[0] = M->n; kd[0] = M->kd;
+      } else {
+        const CouplingMeta* M = reinterpret_cast<const CouplingMeta*>(mb);
+        n[0] = M->n1; n[1] = M->n2; n[2] = M->n3;
+        kd[0] = M->kd1; kd[1] = M->kd2; kd[2] = M->kd3;
+      }
+    }
+    cta_barrier();     // the workers have finished the pixel pass: step i-1's meta slot is free
+    if (lead) {
+      if (i >= 1 && i + 1 < st.nsteps) {
+        const BlockRef& br = step_ref(P, st, i + 1);
+        bulk_load(cx, a.blob, br.meta_off, br.meta_bytes, P.s_meta[(i + 1) & 1], &ctl->meta_full[(i + 1) & 1]);
+      }
+      const uint32_t par0 = (uint32_t)(load_ordinal(st, 0, i) & 1), par12 = (uint32_t)(load_ordinal(st, 1, i) & 1);
+      const BlockRef& br = step_ref(P, st, i);
+      const int nstages = prior ? 1 : 3;
+      bool first = true;
+      for (int t0 = 0; t0 < ntv; t0 += nslots) {
+        const int nt = min(nslots, ntv - t0);
+        const bool last_tile = t0 + nslots >= ntv;
+        for (int stage = 0; stage < nstages; ++stage) {
+          for (int sl = 0; sl < nt; ++sl) {
+            if (!alias) {
+              const int wslot = prior ? 0 : stage;
+              mma(sl, wslot, first && sl == 0, wslot == 0 ? par0 : par12, n[stage], kd[stage]);
+              dpar[sl] ^= 1u;
+            } else if (stage == 1) {
+              mma(sl, 1, first, par12, n[1], kd[1]);
+              dpar[sl] ^= 1u;
+            } else {
+              // S0 holds, in turn: W1, W3 of every tile (coupling) or the prior matrix for all tiles
+              const bool ww = prior ? first : true;
+              mma(sl, 0, ww, W.s0_used & 1u, n[stage], kd[stage]);
+              if (ww) ++W.s0_used;
+              if (prior) {
+                if (last_tile && i + 1 < st.nsteps) s0_refill(step_ref(P, st, i + 1), 0);
+              } else if (stage == 0) {
+                s0_refill(br, 2);
+              } else if (!last_tile) {
+                s0_refill(br, 0);
+              } else if (i + 1 < st.nsteps) {
+                s0_refill(step_ref(P, st, i + 1), 0);
+              }
+              dpar[sl] ^= 1u;
+            }
+          }
+        }
+        first = false;
+      }
+    }
+    __syncwarp();
+    cta_barrier();     // every MMA of step i has completed (the workers waited for each accumulator)
+    if (lead) top_up(cx, P, a, st, W, i, alias);
+  }
+  if (st.nsteps > 0 && !st.is_prior(st.nsteps - 1)) cta_barrier();   // trailing translation pass
+}
+
+// ---- workers ----------------------------------------------------------------------------------
+template <bool kInv>
+__device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const LevelArgs& a, const Steps& st, int img0, int pvalid,
+                            int ntv) {
+  uint8_t* smem = cx.smem;
+  Ctl* ctl = cx.ctl;
+  int32_t* v = reinterpret_cast<int32_t*>(smem + P.s_v);
+  int8_t* xa = reinterpret_cast<int8_t*>(smem + P.s_xa);
+  int32_t* acc = reinterpret_cast<int32_t*>(smem + P.s_acc);
+  uint8_t* sA = smem + P.s_a[0];          // A-operand buffer of the current tile slot
+  const uint32_t* rowinfo = reinterpret_cast<const uint32_t*>(smem + P.s_rowinfo);
+  const int pg = P.pg, ca = P.ca, cb = P.cb, w = P.w, cpad = P.cpad, cbp = P.cbp;
+  const uint32_t recip_a = P.recip_gpa;
+  uint32_t dpar[2] = {0u, 0u};
+  const int nslots = P.nslots;
+  const CouplingMeta* prevM = nullptr;       // coupling whose translation is still to be applied
+
+  auto use_slot = [&](int sl) {
+    sA = smem + P.s_a[sl];
+    cx.tmem_slot = cx.tmem_base + (uint32_t)(sl * kSlotCols) + ((uint32_t)(cx.wq * 32) << 16);
+  };
+  // this thread's part of tile slot sl's A operand is written (and its TMEM reads are done)
+  auto arrive_a = [&](int sl) {
+    ptx::tc_fence_before();
+    ptx::fence_async_smem();
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ptx::smem_u32(&ctl->a_ready[sl])) : "memory");
+  };
+  auto wait_d = [&](int sl) {
+    wait_bar(ctl, a.status, &ctl->d_ready[sl], dpar[sl]);
+    dpar[sl] ^= 1u;
+    ptx::tc_fence_after();
   };
 
   // x_b +/-= rq(acc + bias) of the previous coupling for pixel p
@@ -492,29 +596,24 @@ __device__ void run_steps(Ctx& cx, const LevelPlan& P, const LevelArgs& a, const
       }
     }
     prevM = prior ? nullptr : Mp;
-    worker_barrier();
-    // every thread has left step i-1: its meta slot can take step i+1
-    if (cx.loader && i >= 1 && i + 1 < st.nsteps) {
-      const BlockRef& br = step_ref(P, st, i + 1);
-      bulk_load(cx, a.blob, br.meta_off, br.meta_bytes, P.s_meta[(i + 1) & 1], &ctl->meta_full[(i + 1) & 1]);
-    }
-    const uint32_t par0 = (uint32_t)(load_ordinal(st, 0, i) & 1), par12 = (uint32_t)(load_ordinal(st, 1, i) & 1);
-    bool first = true;
+    cta_barrier();
+    RowPos rp[2];
     if (prior) {
       const PriorMeta M = *Pp;
       const OutRq* orq = reinterpret_cast<const OutRq*>(mb + M.off_out);
-      for (int t = cx.group; t < ntv; t += P.nslots) {
-        const RowPos rp = row_pos(rowinfo, t, cx.row);
-        build_im2col(cx, sA, xa, cpad, w, M.kd, recip_a, rp);
-        if (alias) {
-          run_mma(0, first, W.s0_used & 1u, M.n, M.kd);
-          if (first) ++W.s0_used;
-          if (cx.loader && t + P.nslots >= ntv) s0_request_next_step(i);
-        } else {
-          run_mma(0, first, par0, M.n, M.kd);
+      for (int t0 = 0; t0 < ntv; t0 += nslots) {
+        const int nt = min(nslots, ntv - t0);
+        for (int sl = 0; sl < nt; ++sl) {
+          use_slot(sl);
+          rp[sl] = row_pos(rowinfo, t0 + sl, cx.row);
+          build_im2col(cx, sA, xa, cpad, w, M.kd, recip_a, rp[sl]);
+          arrive_a(sl);
         }
-        first = false;
-        epilogue_prior(cx, P, a, M, orq, img0, rp);
+        for (int sl = 0; sl < nt; ++sl) {
+          wait_d(sl);
+          use_slot(sl);
+          epilogue_prior(cx, P, a, M, orq, img0, rp[sl]);
+        }
       }
     } else {
       const CouplingMeta M = *Mp;
@@ -522,43 +621,39 @@ __device__ void run_steps(Ctx& cx, const LevelPlan& P, const LevelArgs& a, const
       const HiddenRq* h2 = reinterpret_cast<const HiddenRq*>(mb + M.off_h2);
       const int2* u1 = reinterpret_cast<const int2*>(mb + M.off_u1);
       const int2* u2 = reinterpret_cast<const int2*>(mb + M.off_u2);
-      const BlockRef& br = step_ref(P, st, i);
-      for (int t = cx.group; t < ntv; t += P.nslots) {
-        const bool last_tile = t + P.nslots >= ntv;
-        const RowPos rp = row_pos(rowinfo, t, cx.row);
-        build_im2col(cx, sA, xa, cpad, w, M.kd1, recip_a, rp);
-        if (alias) {
-          run_mma(0, true, W.s0_used & 1u, M.n1, M.kd1);
-          ++W.s0_used;
-          if (cx.loader) s0_request(br, 2);
-        } else {
-          run_mma(0, first, par0, M.n1, M.kd1);
+      for (int t0 = 0; t0 < ntv; t0 += nslots) {
+        const int nt = min(nslots, ntv - t0);
+        for (int sl = 0; sl < nt; ++sl) {                     // conv 3x3: input -> hidden 1
+          use_slot(sl);
+          rp[sl] = row_pos(rowinfo, t0 + sl, cx.row);
+          build_im2col(cx, sA, xa, cpad, w, M.kd1, recip_a, rp[sl]);
+          arrive_a(sl);
         }
-        epilogue_hidden(cx, M.mode1, M.us1, M.n1, M.kd2, h1, u1, M.lo1, M.hi1, sA);
-        run_mma(1, first, par12, M.n2, M.kd2);
-        epilogue_hidden(cx, M.mode2, M.us2, M.n2, M.kd3, h2, u2, M.lo2, M.hi2, sA);
-        if (alias) {
-          run_mma(0, true, W.s0_used & 1u, M.n3, M.kd3);
-          ++W.s0_used;
-          if (cx.loader) {
-            if (last_tile) s0_request_next_step(i);
-            else s0_request(br, 0);
-          }
-        } else {
-          run_mma(2, first, par12, M.n3, M.kd3);
+        for (int sl = 0; sl < nt; ++sl) {                     // requant, conv 1x1
+          wait_d(sl);
+          use_slot(sl);
+          epilogue_hidden(cx, M.mode1, M.us1, M.n1, M.kd2, h1, u1, M.lo1, M.hi1, sA);
+          arrive_a(sl);
         }
-        first = false;
-        epilogue_scatter(cx, cb, cbp, recip_b, acc, pg, w, rp);
+        for (int sl = 0; sl < nt; ++sl) {                     // requant, conv 3x3 as per-tap partials
+          wait_d(sl);
+          use_slot(sl);
+          epilogue_hidden(cx, M.mode2, M.us2, M.n2, M.kd3, h2, u2, M.lo2, M.hi2, sA);
+          arrive_a(sl);
+        }
+        for (int sl = 0; sl < nt; ++sl) {                     // shifted sum into the accumulator
+          wait_d(sl);
+          use_slot(sl);
+          epilogue_scatter(cx, cb, cbp, acc, pg, w, rp[sl]);
+        }
       }
     }
     ptx::tc_fence_before();
-    worker_barrier();
-    // every MMA of step i has completed (each group waited for its last accumulator)
-    if (cx.loader) top_up(cx, P, a, st, W, i, alias);
+    cta_barrier();
   }
   if (prevM) {
     for (int p = cx.tid; p < pvalid; p += kWorkers) apply_translation(p);
-    worker_barrier();
+    cta_barrier();
   }
 }
 
@@ -568,10 +663,10 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
   __shared__ Ctl ctl;
   const LevelPlan& P = *a.plan;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int wpg = kWorkerWarps / P.nslots;       // warps per group
 
   if (tid == 0) {
     for (int s = 0; s < 2; ++s) {
+      ptx::mbar_init(ptx::smem_u32(&ctl.a_ready[s]), (uint32_t)kWorkers);
       ptx::mbar_init(ptx::smem_u32(&ctl.d_ready[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&ctl.meta_full[s]), 1);
     }
@@ -599,25 +694,24 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
   st.nsteps = P.n_couplings + (st.do_prior ? 1 : 0);
   st.inverse = kInv;
 
-  {
-    Ctx cx;
-    cx.smem = smem;
-    cx.ctl = &ctl;
-    cx.status = a.status;
-    cx.tid = tid;
-    cx.warp = warp;
-    cx.lane = lane;
-    cx.wq = warp & 3;
-    cx.group = warp / wpg;
-    cx.cs = (warp % wpg) >> 2;
-    cx.ncs = wpg >> 2;
-    cx.gthreads = wpg * 32;
-    cx.row = cx.wq * 32 + lane;
-    cx.elected = (warp % wpg) == 0 && lane == 0;
-    cx.loader = tid == 0;
-    cx.tmem_slot0 = tmem + (uint32_t)(cx.group * kSlotCols);
-    cx.tmem_slot = cx.tmem_slot0 + ((uint32_t)(cx.wq * 32) << 16);
+  Ctx cx;
+  cx.smem = smem;
+  cx.ctl = &ctl;
+  cx.status = a.status;
+  cx.tid = tid;
+  cx.warp = warp;
+  cx.lane = lane;
+  cx.wq = warp & 3;
+  cx.cs = warp >> 2;
+  cx.ncs = kWorkerWarps >> 2;
+  cx.row = cx.wq * 32 + lane;
+  cx.tmem_base = tmem;
+  cx.tmem_slot = tmem + ((uint32_t)(cx.wq * 32) << 16);
 
+  if (warp >= kWorkerWarps) {
+    cta_barrier();                       // the workers have loaded the flow variable
+    run_control(cx, P, a, st, ntv);
+  } else {
     int32_t* acc = reinterpret_cast<int32_t*>(smem + P.s_acc);
     for (int idx = tid; idx < P.cb * pg; idx += kWorkers) acc[idx] = 0;
     uint32_t* rowinfo = reinterpret_cast<uint32_t*>(smem + P.s_rowinfo);
@@ -646,9 +740,9 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
         v[P.col_out[k] * pg + g * px + q] = val;
       }
     }
-    worker_barrier();
+    cta_barrier();
 
-    run_steps<kInv>(cx, P, a, st, img0, pvalid, ntv);
+    run_workers<kInv>(cx, P, a, st, img0, pvalid, ntv);
 
     if (!kInv) {
       // split on store: factored-out half -> z block of this level; kept half -> next level (or
