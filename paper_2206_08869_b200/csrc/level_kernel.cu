@@ -548,15 +548,18 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
     ptx::tc_fence_after();
   };
 
-  // x_b +/-= rq(acc + bias) of the previous coupling for pixel p
-  auto apply_translation = [&](int p) {
+  // x_b +/-= rq(acc + bias) of the previous coupling. Work item = (pixel, group of four output
+  // channels), so that levels with few pixels per CTA still use every thread.
+  auto apply_translation_all = [&]() {
     const uint8_t* pm = reinterpret_cast<const uint8_t*>(prevM);
     const int32_t* colB = reinterpret_cast<const int32_t*>(pm + prevM->off_colB);
     const OutRq* orq = reinterpret_cast<const OutRq*>(pm + prevM->off_out);
-    for (int c0 = 0; c0 < cb; c0 += 4) {
+    const int items = ((cb + 3) >> 2) * pvalid;
+    for (int it = cx.tid; it < items; it += kWorkers) {
+      const int cg = it / pvalid, p = it - cg * pvalid;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        const int c = c0 + k;
+        const int c = cg * 4 + k;
         if (c < cb) {
           const OutRq o = orq[c];
           const uint32_t t = (uint32_t)rq_exact(acc[c * pg + p] + o.bias, o.m0, o.s);
@@ -567,9 +570,13 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
       }
     }
   };
-  // network input of pixel p: ca channels requantised to int8, padded to cpad bytes
-  auto requant_input = [&](int p, const int32_t* cols, int32_t m0, int32_t s) {
-    for (int g0 = 0; g0 < cpad; g0 += 8) {
+  // network input: ca channels requantised to int8, padded to cpad bytes per pixel. Work item =
+  // (pixel, granule of eight channels).
+  auto requant_input_all = [&](const int32_t* cols, int32_t m0, int32_t s) {
+    const int items = (cpad >> 3) * pvalid;
+    for (int it = cx.tid; it < items; it += kWorkers) {
+      const int g = it / pvalid, p = it - g * pvalid;
+      const int g0 = g << 3;
       int y[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
@@ -580,6 +587,7 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
           make_uint2(pack4(y[0], y[1], y[2], y[3]), pack4(y[4], y[5], y[6], y[7]));
     }
   };
+  auto worker_barrier = [&]() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); };
 
   for (int i = 0; i < st.nsteps; ++i) {
     wait_bar(ctl, a.status, &ctl->meta_full[i & 1], (uint32_t)((i >> 1) & 1));
@@ -590,10 +598,11 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
     {
       const int32_t* cols = prior ? P.col_out : reinterpret_cast<const int32_t*>(mb + Mp->off_colA);
       const int32_t in_m0 = prior ? Pp->in_m0 : Mp->in_m0, in_s = prior ? Pp->in_s : Mp->in_s;
-      for (int p = cx.tid; p < pvalid; p += kWorkers) {
-        if (prevM) apply_translation(p);
-        requant_input(p, cols, in_m0, in_s);
+      if (prevM) {
+        apply_translation_all();
+        worker_barrier();            // the network input may read channels that were just updated
       }
+      requant_input_all(cols, in_m0, in_s);
     }
     prevM = prior ? nullptr : Mp;
     cta_barrier();
@@ -652,7 +661,7 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
     cta_barrier();
   }
   if (prevM) {
-    for (int p = cx.tid; p < pvalid; p += kWorkers) apply_translation(p);
+    apply_translation_all();
     cta_barrier();
   }
 }
