@@ -282,22 +282,27 @@ __device__ void epilogue_scatter(const Ctx& cx, int cb, int cbp, int32_t* __rest
     const bool ok_0 = ((sm >> (du * 3 + 1)) & 1u) != 0;   // dv =  0: target column j
     const bool ok_p = ((sm >> (du * 3 + 2)) & 1u) != 0;   // dv = +1: target column j - 1
     const int c0 = gq << 3;
-    int32_t* dst = acc + c0 * pg + rp.p - (du - 1) * w;   // this lane's own output pixel for this du
+    // this lane's own output pixel for this du; the row sum is zero whenever that pixel is
+    // outside the image (all three contributions share its row, hence its vertical validity)
+    const uint32_t dst = ptx::smem_u32(acc + c0 * pg + rp.p - (du - 1) * w);
+    const uint32_t plane = (uint32_t)pg * 4u;
+    const bool edge_hi = cx.lane == 31 && ok_m, edge_lo = cx.lane == 0 && ok_p;
+    int sum[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {                        // branch-free: eight independent chains
+      const int v_m = ok_m ? (int)r0[i] : 0;
+      const int v_0 = ok_0 ? (int)r1[i] : 0;
+      const int v_p = ok_p ? (int)r2[i] : 0;
+      const int from_next = __shfl_down_sync(0xFFFFFFFFu, v_p, 1);   // lane L+1's dv=+1 lands here
+      const int from_prev = __shfl_up_sync(0xFFFFFFFFu, v_m, 1);     // lane L-1's dv=-1 lands here
+      sum[i] = v_0 + (cx.lane < 31 ? from_next : 0) + (cx.lane > 0 ? from_prev : 0);
+    }
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      if (c0 + i < cb) {                                  // uniform across the warp
-        const int v_m = ok_m ? (int)r0[i] : 0;
-        const int v_0 = ok_0 ? (int)r1[i] : 0;
-        const int v_p = ok_p ? (int)r2[i] : 0;
-        const int from_next = __shfl_down_sync(0xFFFFFFFFu, v_p, 1);   // lane L+1's dv=+1 lands here
-        const int from_prev = __shfl_up_sync(0xFFFFFFFFu, v_m, 1);     // lane L-1's dv=-1 lands here
-        int sum = v_0;
-        if (cx.lane < 31) sum += from_next;
-        if (cx.lane > 0) sum += from_prev;
-        if (sum != 0) atomicAdd(dst + i * pg, sum);
-        if (cx.lane == 31 && v_m != 0) atomicAdd(dst + i * pg + 1, v_m);
-        if (cx.lane == 0 && v_p != 0) atomicAdd(dst + i * pg - 1, v_p);
-      }
+      const bool ch = c0 + i < cb;
+      ptx::red_add_s32(dst + (uint32_t)i * plane, sum[i], ch && ok_0);
+      ptx::red_add_s32(dst + (uint32_t)i * plane + 4u, (int)r0[i], ch && edge_hi);
+      ptx::red_add_s32(dst + (uint32_t)i * plane - 4u, (int)r2[i], ch && edge_lo);
     }
   }
 }

@@ -45,6 +45,16 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+// Predicated fire-and-forget add to a 32-bit word in shared memory.
+__device__ __forceinline__ void red_add_s32(uint32_t saddr, int val, bool pred) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %2, 0;\n\t"
+      "@p red.shared.add.s32 [%0], %1;\n\t}" ::"r"(saddr),
+      "r"(val), "r"((uint32_t)pred)
+      : "memory");
+}
+
 // ---- bulk copy global -> shared, completion counted on an mbarrier ---------------------------
 // dst, src and bytes must be multiples of 16.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
