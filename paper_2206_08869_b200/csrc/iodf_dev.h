@@ -26,7 +26,7 @@ constexpr int kMaxCouplings = 32;    // per level
 constexpr int kMaxC = 256;           // flow channels per level
 constexpr int kMaxHidden = 256;      // kept hidden channels per layer (padded)
 constexpr int kSlotCols = 256;       // TMEM columns per tile slot when two tiles are in flight
-constexpr uint32_t kSpinLimit = 4000000u;
+constexpr uint32_t kSpinLimit = 20000u;   // bounded waits: tries of up to 100 us each
 
 // Per-hidden-channel constants of the fast requantisation path (16 bytes).
 //   y = hi32(acc * m0 + c64) >> sh,  c64 = bias * m0 + 2^(30+s),  sh = s - 1   (needs s >= 1)

@@ -70,7 +70,7 @@ __device__ __noinline__ bool wait_bar(Ctl* ctl, uint32_t* status, uint64_t* bar,
   const uint32_t b = ptx::smem_u32(bar);
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
     if (ptx::mbar_try_wait(b, parity)) return true;
-    if ((it & 255u) == 255u && *ab) return false;
+    if (*ab) return false;
   }
   *ab = 1;
   atomicExch(status, 1u);
@@ -205,13 +205,30 @@ struct Requant {
   // 16 accumulator columns starting at channel ch0 -> one 16-byte chunk of the next A operand
   __device__ __forceinline__ uint4 chunk(const uint32_t* r, int ch0) const {
     uint32_t wd[4];
+    if (kMode == kModeUniform) {
+      // {m0, bias} pairs of two channels per 16-byte shared-memory load (the table is 16-byte aligned)
+      const int4* q = reinterpret_cast<const int4*>(mb + ch0);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int y0 = one((int)r[4 * i], ch0 + 4 * i), y1 = one((int)r[4 * i + 1], ch0 + 4 * i + 1);
-      const int y2 = one((int)r[4 * i + 2], ch0 + 4 * i + 2), y3 = one((int)r[4 * i + 3], ch0 + 4 * i + 3);
-      wd[i] = kClip == kClipS8Relu ? pack4_sat(y0, y1, y2, y3) : pack4(y0, y1, y2, y3);
+      for (int i = 0; i < 4; ++i) {
+        const int4 c01 = q[2 * i], c23 = q[2 * i + 1];
+        const int y0 = uniform_one((int)r[4 * i], c01.x, c01.y), y1 = uniform_one((int)r[4 * i + 1], c01.z, c01.w);
+        const int y2 = uniform_one((int)r[4 * i + 2], c23.x, c23.y), y3 = uniform_one((int)r[4 * i + 3], c23.z, c23.w);
+        wd[i] = kClip == kClipS8Relu ? pack4_sat(y0, y1, y2, y3) : pack4(y0, y1, y2, y3);
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int y0 = one((int)r[4 * i], ch0 + 4 * i), y1 = one((int)r[4 * i + 1], ch0 + 4 * i + 1);
+        const int y2 = one((int)r[4 * i + 2], ch0 + 4 * i + 2), y3 = one((int)r[4 * i + 3], ch0 + 4 * i + 3);
+        wd[i] = kClip == kClipS8Relu ? pack4_sat(y0, y1, y2, y3) : pack4(y0, y1, y2, y3);
+      }
     }
     return make_uint4(wd[0], wd[1], wd[2], wd[3]);
+  }
+  __device__ __forceinline__ int uniform_one(int acc, int m0, int bias) const {
+    const long long p = (long long)(acc + bias) * (long long)m0 + rnd64;
+    const int y = ((int)(p >> 32)) >> sh;
+    return kClip == kClipS8Relu ? max(y, 0) : clampi(y, lo, hi);
   }
 };
 
