@@ -106,6 +106,27 @@ def run_reference(args, rank):
         "gpu_launches": 0}))
 
 
+def max_over_ranks(values, world, device=None):
+    """Element-wise maximum of a list of floats over all ranks (identity for one rank)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def job_throughput(images_per_rank_per_step, world, steps, seconds):
+    """Whole-job images/s: every rank processes its own batch, the slowest rank sets the time."""
+    return images_per_rank_per_step * world * steps / seconds
+
+
+def rank_seed_offset(rank, i):
+    """Distinct synthetic input sets per rank and per rotating buffer."""
+    return 100 * rank + i
+
+
 def workload(args):
     c = S.CONFIGS[args.config]
     return {"workload": "config %s: ImageNet%d-shaped pruned IODF encode, batch %d of uint8 3x%dx%d, %d levels x %d "
@@ -150,7 +171,7 @@ def main():
     lay = m.layout
     macs = int(lay.macs_per_image)
 
-    xs = [torch.from_numpy(S.config_images(cfg, batch=B, seed_offset=100 * rank + i)).to(dev) for i in range(N_SETS)]
+    xs = [torch.from_numpy(S.config_images(cfg, batch=B, seed_offset=rank_seed_offset(rank, i))).to(dev) for i in range(N_SETS)]
     zs = [torch.empty((B, m.d), dtype=torch.int32, device=dev) for _ in range(N_SETS)]
     ps = [torch.empty((B, 2, m.d_fact), dtype=torch.int32, device=dev) for _ in range(N_SETS)]
     stream = torch.cuda.current_stream()
@@ -201,7 +222,7 @@ def main():
                 "whole_step_frac": (2.0 * macs * B / (total_ms / args.steps * 1e-3) / 1e12) / peak_int8}
 
     # ---- end to end through the host-buffer entry point --------------------------------------
-    hx = [torch.from_numpy(S.config_images(cfg, batch=B, seed_offset=100 * rank + i)).pin_memory() for i in range(2)]
+    hx = [torch.from_numpy(S.config_images(cfg, batch=B, seed_offset=rank_seed_offset(rank, i))).pin_memory() for i in range(2)]
     hz = [torch.empty((B, m.d), dtype=torch.int32).pin_memory() for _ in range(2)]
     hp = [torch.empty((B, 2, m.d_fact), dtype=torch.int32).pin_memory() for _ in range(2)]
     e2e_steps = max(10, min(args.steps, 100))
@@ -216,20 +237,17 @@ def main():
     e2e_s = time.perf_counter() - t0
     G.iodf_check(m)
 
-    t = torch.tensor([total_ms, e2e_s], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_s = float(t[0]), float(t[1])
+    total_ms, e2e_s = max_over_ranks([total_ms, e2e_s], world, dev)
 
     if rank == 0:
         cores = os.cpu_count() or 1
         out = {
-            "metric": METRIC, "value": B * world * args.steps / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": job_throughput(B, world, args.steps, total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
             "ms_per_sample": total_ms / args.steps / B,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
             "config": workload(args), "clocks": sampler.summary(), "roofline": roofline,
-            "e2e": {"value": B * world * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": B * m.d,
+            "e2e": {"value": job_throughput(B, world, e2e_steps, e2e_s), "unit": UNIT, "h2d_bytes_per_step": B * m.d,
                     "d2h_bytes_per_step": B * m.d * 4 + B * 2 * m.d_fact * 4, "steps": e2e_steps},
             "gpu_launches": G.iodf_launches_per_call(m) * args.steps,
             "gops_per_image": 2.0 * macs / 1e9,
