@@ -143,6 +143,7 @@ inline size_t wpos(int n_pad, int n, int k) { return (size_t)(k >> 4) * n_pad * 
 
 struct PackedBlock {
   std::vector<uint8_t> meta, w[3];
+  uint32_t k_slices[3] = {0, 0, 0};
 };
 
 void append_block(std::vector<uint8_t>& blob, const PackedBlock& pb, BlockRef* ref) {
@@ -153,7 +154,10 @@ void append_block(std::vector<uint8_t>& blob, const PackedBlock& pb, BlockRef* r
     blob.insert(blob.end(), part.begin(), part.end());
   };
   add(pb.meta, &ref->meta_off, &ref->meta_bytes);
-  for (int i = 0; i < 3; ++i) add(pb.w[i], &ref->w_off[i], &ref->w_bytes[i]);
+  for (int i = 0; i < 3; ++i) {
+    add(pb.w[i], &ref->w_off[i], &ref->w_bytes[i]);
+    ref->k_slices[i] = pb.k_slices[i];
+  }
   blob.resize(up((uint32_t)blob.size(), kAlign), 0);
 }
 
@@ -175,24 +179,28 @@ PackedBlock pack_coupling(const iodf_coupling_desc& cp, const Blobs& B, int ca, 
   M.in_m0 = cp.in_m0; M.in_s = cp.in_s;
   M.n1 = d.n1; M.n2 = d.n2; M.kd1 = d.kd1; M.kd2 = d.kd2; M.kd3 = d.kd3; M.n3 = d.n3;
   M.lo1 = a1.lo; M.hi1 = a1.hi; M.lo2 = a2.lo; M.hi2 = a2.hi;
+  // requantisation tables: both flavours are built, only the one the layer's mode reads is kept
+  std::vector<HiddenRq> h1(d.n1), h2(d.n2);
+  std::vector<int32_t> u1(2 * d.n1), u2(2 * d.n2);
+  put_hidden_rq(h1.data(), u1.data(), L1, B, d.n1, &M.mode1, &M.us1);
+  put_hidden_rq(h2.data(), u2.data(), L2, B, d.n2, &M.mode2, &M.us2);
   uint32_t off = sizeof(CouplingMeta);
   M.off_colA = (int)off; off += up(4 * ca, 16);
   M.off_colB = (int)off; off += up(4 * cb, 16);
   M.off_out = (int)off;  off += (uint32_t)sizeof(OutRq) * cb;
-  M.off_h1 = (int)off;   off += (uint32_t)sizeof(HiddenRq) * d.n1;
-  M.off_h2 = (int)off;   off += (uint32_t)sizeof(HiddenRq) * d.n2;
-  M.off_u1 = (int)off;   off += 8u * d.n1;
-  M.off_u2 = (int)off;   off += 8u * d.n2;
+  M.off_h1 = M.off_u1 = (int)off; off += M.mode1 == 2 ? 8u * d.n1 : (uint32_t)sizeof(HiddenRq) * d.n1;
+  M.off_h2 = M.off_u2 = (int)off; off += M.mode2 == 2 ? 8u * d.n2 : (uint32_t)sizeof(HiddenRq) * d.n2;
   pb.meta.assign(off, 0);
   std::memcpy(pb.meta.data() + M.off_colA, colA, 4 * ca);
   std::memcpy(pb.meta.data() + M.off_colB, colB, 4 * cb);
   put_out_rq(reinterpret_cast<OutRq*>(pb.meta.data() + M.off_out), L3, B);
-  put_hidden_rq(reinterpret_cast<HiddenRq*>(pb.meta.data() + M.off_h1),
-                reinterpret_cast<int32_t*>(pb.meta.data() + M.off_u1), L1, B, d.n1, &M.mode1, &M.us1);
-  put_hidden_rq(reinterpret_cast<HiddenRq*>(pb.meta.data() + M.off_h2),
-                reinterpret_cast<int32_t*>(pb.meta.data() + M.off_u2), L2, B, d.n2, &M.mode2, &M.us2);
+  if (M.mode1 == 2) std::memcpy(pb.meta.data() + M.off_u1, u1.data(), 8u * d.n1);
+  else std::memcpy(pb.meta.data() + M.off_h1, h1.data(), sizeof(HiddenRq) * d.n1);
+  if (M.mode2 == 2) std::memcpy(pb.meta.data() + M.off_u2, u2.data(), 8u * d.n2);
+  else std::memcpy(pb.meta.data() + M.off_h2, h2.data(), sizeof(HiddenRq) * d.n2);
   std::memcpy(pb.meta.data(), &M, sizeof(M));
 
+  pb.k_slices[0] = d.kd1 / 32; pb.k_slices[1] = d.kd2 / 32; pb.k_slices[2] = d.kd3 / 32;
   // W1: row = hidden channel, K index = tap*cpad + c
   pb.w[0].assign((size_t)d.n1 * d.kd1, 0);
   const int8_t* w1 = B.w + L1.weight_off;
@@ -228,6 +236,7 @@ PackedBlock pack_prior(const iodf_level_desc& lv, const Blobs& B, int ca, int cb
   pb.meta.assign(sizeof(PriorMeta) + sizeof(OutRq) * 2 * cb, 0);
   put_out_rq(reinterpret_cast<OutRq*>(pb.meta.data() + M.off_out), L, B);
   std::memcpy(pb.meta.data(), &M, sizeof(M));
+  pb.k_slices[0] = M.kd / 32;
   pb.w[0].assign((size_t)M.n * M.kd, 0);
   const int8_t* w = B.w + L.weight_off;
   for (int o = 0; o < 2 * cb; ++o)
@@ -249,14 +258,18 @@ uint32_t pow2_cols(uint32_t need) {
 //   mode 0: two tile slots, every weight matrix resident      (needs all N <= 256 and >= 2 tiles)
 //   mode 1: one tile slot, every weight matrix resident
 //   mode 2: one tile slot, W1 and W3 share a slot and are re-fetched per tile
+//   mode 3: one tile slot, weights streamed per tile in 32-byte K-slices through a small ring
+//           (the only mode for hidden widths above 256: a 512 x 512 matrix alone is 256 KB)
 bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32_t wmax[3], uint32_t n_max,
                uint32_t limit, uint32_t max_batch) {
   int group = P.px >= kTileM ? 1 : kTileM / P.px;
   group = std::max(1, std::min<int>(group, (int)max_batch));
   for (; group >= 1; group = (group > 1 ? group / 2 : 0)) {
     const int tiles = (group * P.px + kTileM - 1) / kTileM;
-    for (int mode = 0; mode < 3; ++mode) {
+    for (int mode = 0; mode < 4; ++mode) {
       if (mode == 0 && (tiles < 2 || n_max > (uint32_t)kSlotCols)) continue;
+      if (mode < 3 && n_max > 2u * kSlotCols) continue;
+      if (mode == 3 && n_max <= (uint32_t)kSlotCols) continue;   // resident weights are faster when they fit
       const uint32_t pg = up((uint32_t)group * P.px, 32);
       uint32_t off = 0;
       auto take = [&](uint32_t bytes) { uint32_t o = off; off = up(off + bytes, kAlign); return o; };
@@ -268,11 +281,18 @@ bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32
       P.s_a[1] = mode == 0 ? take(a_bytes) : P.s_a[0];
       P.s_meta[0] = take(meta_bytes);
       P.s_meta[1] = take(meta_bytes);
-      P.s_w[0] = take(mode == 2 ? std::max(wmax[0], wmax[2]) : wmax[0]);
-      P.s_w[1] = take(wmax[1]);
-      P.s_w[2] = mode == 2 ? P.s_w[0] : take(wmax[2]);
+      P.ring_slot_bytes = up(32u * n_max, kAlign);
+      if (mode == 3) {
+        P.s_w[0] = take(P.ring_slot_bytes * kRingDepth);
+        P.s_w[1] = P.s_w[2] = P.s_w[0];
+      } else {
+        P.s_w[0] = take(mode == 2 ? std::max(wmax[0], wmax[2]) : wmax[0]);
+        P.s_w[1] = take(wmax[1]);
+        P.s_w[2] = mode == 2 ? P.s_w[0] : take(wmax[2]);
+      }
       P.s_total = off;
       P.w13_alias = mode == 2;
+      P.streamed = mode == 3;
       P.nslots = mode == 0 ? 2 : 1;
       P.tmem_cols = (int)(mode == 0 ? 2 * kSlotCols : pow2_cols(n_max));
       P.group = group;

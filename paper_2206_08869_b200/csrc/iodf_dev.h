@@ -24,7 +24,8 @@ constexpr int kWorkers = kWorkerWarps * 32;
 constexpr int kThreads = kWorkers + 32;   // + one control warp (bulk copies and MMA issue)
 constexpr int kMaxCouplings = 32;    // per level
 constexpr int kMaxC = 256;           // flow channels per level
-constexpr int kMaxHidden = 256;      // kept hidden channels per layer (padded)
+constexpr int kMaxHidden = 512;      // kept hidden channels per layer (padded): the TMEM column count
+constexpr int kRingDepth = 3;        // weight K-slices in flight when weights are streamed
 constexpr int kSlotCols = 256;       // TMEM columns per tile slot when two tiles are in flight
 constexpr uint32_t kSpinLimit = 20000u;   // bounded waits: tries of up to 100 us each
 
@@ -75,6 +76,7 @@ static_assert(sizeof(PriorMeta) == 128, "meta header is 128 bytes");
 struct BlockRef {                // where a block's parts sit in the level blob (byte offsets)
   uint32_t meta_off, meta_bytes;
   uint32_t w_off[3], w_bytes[3];
+  uint32_t k_slices[3];          // K / 32 of each matrix (a K-slice of 32 bytes is w_bytes / k_slices contiguous bytes)
 };
 
 // Everything a level kernel needs; lives in global memory.
@@ -91,6 +93,9 @@ struct LevelPlan {
   int32_t nslots;                // tiles in flight per CTA: 1 or 2
   int32_t tmem_cols;
   int32_t w13_alias;             // 1: W1 and W3 share a slot and are re-fetched per tile
+  int32_t streamed;              // 1: weights are streamed per tile in 32-byte K-slices through a ring of
+                                 //    kRingDepth slots at s_w[0] (hidden widths above 256, one tile in flight)
+  uint32_t ring_slot_bytes;
   // shared-memory byte offsets
   uint32_t s_v, s_xa, s_acc, s_rowinfo, s_a[2], s_meta[2], s_w[3], s_total;
   uint32_t recip_gpa, recip_gpb; // floor(g / (cpad/8)) = (g * recip_gpa) >> 16 for g < 4096; same for cbp/8

@@ -44,7 +44,8 @@ namespace {
 struct __align__(16) Ctl {
   uint64_t a_ready[2];    // workers -> control: the tile slot's A operand is written (count = workers)
   uint64_t d_ready[2];    // tensor core -> workers: the tile slot's accumulator is complete
-  uint64_t w_full[3];     // bulk copy -> elected threads: weight slot filled
+  uint64_t w_full[3];     // bulk copy -> control: weight slot (or ring slot) filled
+  uint64_t w_empty[3];    // tensor core -> control: the MMAs reading a ring slot have completed
   uint64_t meta_full[2];  // bulk copy -> everyone: meta block of step (i & 1) has landed
   uint32_t tmem_base;
   uint32_t abort;
@@ -537,6 +538,114 @@ __device__ void run_control(const Ctx& cx, const LevelPlan& P, const LevelArgs& 
   if (st.nsteps > 0 && !st.is_prior(st.nsteps - 1)) cta_barrier();   // trailing translation pass
 }
 
+// ---- control thread, streamed weights --------------------------------------------------------------
+// For hidden widths above 256 no weight matrix stays resident: every tile re-reads W1, W2, W3 from
+// L2 in K-slices of 32 bytes (one MMA K step: N x 32 bytes, contiguous in the packed matrix) through
+// a ring of kRingDepth slots. The thread runs a producer cursor (bulk copies, up to kRingDepth
+// slices ahead, across stage, tile and step boundaries) and a consumer cursor (MMAs) over the same
+// fixed sequence of slices. Slice g uses ring slot g % depth; its load completes phase g / depth of
+// that slot's "full" barrier, and the MMAs that read it commit to the slot's "empty" barrier.
+struct SliceCursor {
+  int step, tile, stage, k;
+  uint32_t g;            // running slice number
+};
+
+__device__ void run_control_streamed(const Ctx& cx, const LevelPlan& P, const LevelArgs& a, const Steps& st, int ntv) {
+  uint8_t* smem = cx.smem;
+  Ctl* ctl = cx.ctl;
+  const bool lead = cx.lane == 0;
+  uint32_t apar = 0u;
+  SliceCursor prod{0, 0, 0, 0, 0u};
+
+  auto stages_of = [&](int step) { return st.is_prior(step) ? 1 : 3; };
+  // advance a cursor to the next slice of the fixed sequence; false when the level is finished
+  auto advance = [&](SliceCursor& c) {
+    const BlockRef& br = step_ref(P, st, c.step);
+    ++c.g;
+    if (++c.k < (int)br.k_slices[c.stage]) return true;
+    c.k = 0;
+    if (++c.stage < stages_of(c.step)) return true;
+    c.stage = 0;
+    if (++c.tile < ntv) return true;
+    c.tile = 0;
+    return ++c.step < st.nsteps;
+  };
+  bool prod_live = st.nsteps > 0 && ntv > 0;
+  // issue the loads of every slice up to `limit` slices ahead of consumer slice number g_cons
+  auto produce = [&](uint32_t g_cons) {
+    while (prod_live && prod.g < g_cons + (uint32_t)kRingDepth) {
+      const uint32_t slot = prod.g % (uint32_t)kRingDepth, round = prod.g / (uint32_t)kRingDepth;
+      if (round > 0) wait_bar(ctl, a.status, &ctl->w_empty[slot], (round - 1u) & 1u);
+      const BlockRef& br = step_ref(P, st, prod.step);
+      const uint32_t bytes = br.w_bytes[prod.stage] / br.k_slices[prod.stage];
+      bulk_load(cx, a.blob, br.w_off[prod.stage] + (uint32_t)prod.k * bytes, bytes,
+                P.s_w[0] + slot * P.ring_slot_bytes, &ctl->w_full[slot]);
+      prod_live = advance(prod);
+    }
+  };
+
+  if (lead) {
+    for (int i = 0; i < st.nsteps && i < 2; ++i) {
+      const BlockRef& br = step_ref(P, st, i);
+      bulk_load(cx, a.blob, br.meta_off, br.meta_bytes, P.s_meta[i], &ctl->meta_full[i]);
+    }
+    produce(0u);
+  }
+  uint32_t g = 0u;       // consumer slice number
+  for (int i = 0; i < st.nsteps; ++i) {
+    const bool prior = st.is_prior(i);
+    int n[3] = {0, 0, 0};
+    if (lead) {
+      wait_bar(ctl, a.status, &ctl->meta_full[i & 1], (uint32_t)((i >> 1) & 1));
+      const uint8_t* mb = smem + P.s_meta[i & 1];
+      if (prior) {
+        n[0] = reinterpret_cast<const PriorMeta*>(mb)->n;
+      } else {
+        const CouplingMeta* M = reinterpret_cast<const CouplingMeta*>(mb);
+        n[0] = M->n1; n[1] = M->n2; n[2] = M->n3;
+      }
+    }
+    cta_barrier();     // the workers have finished the pixel pass: step i-1's meta slot is free
+    if (lead) {
+      if (i >= 1 && i + 1 < st.nsteps) {
+        const BlockRef& br = step_ref(P, st, i + 1);
+        bulk_load(cx, a.blob, br.meta_off, br.meta_bytes, P.s_meta[(i + 1) & 1], &ctl->meta_full[(i + 1) & 1]);
+      }
+      const BlockRef& br = step_ref(P, st, i);
+      const int nstages = prior ? 1 : 3;
+      const uint32_t sa = ptx::smem_u32(smem + P.s_a[0]);
+      for (int t = 0; t < ntv; ++t) {
+        for (int stage = 0; stage < nstages; ++stage) {
+          wait_bar(ctl, a.status, &ctl->a_ready[0], apar);
+          apar ^= 1u;
+          ptx::tc_fence_after();
+          const int nn = n[stage];
+          const uint32_t lbo_b = (uint32_t)nn * 16u;
+          for (int k = 0; k < (int)br.k_slices[stage]; ++k, ++g) {
+            produce(g);
+            const uint32_t slot = g % (uint32_t)kRingDepth;
+            wait_bar(ctl, a.status, &ctl->w_full[slot], (g / (uint32_t)kRingDepth) & 1u);
+            const uint32_t sb = ptx::smem_u32(smem + P.s_w[0] + slot * P.ring_slot_bytes);
+            const uint64_t da = ptx::umma_desc(sa + (uint32_t)k * 2u * (kTileM * 16), kTileM * 16, 128);
+            for (int n0 = 0; n0 < nn; n0 += 256) {
+              const uint64_t db = ptx::umma_desc(sb + (uint32_t)n0 * 16u, lbo_b, 128);
+              const uint32_t idesc = ptx::umma_idesc_s8((uint32_t)min(256, nn - n0));
+              if (k == 0) ptx::umma_i8_first(cx.tmem_base + (uint32_t)n0, da, db, idesc);
+              else ptx::umma_i8_acc(cx.tmem_base + (uint32_t)n0, da, db, idesc);
+            }
+            ptx::umma_commit(ptx::smem_u32(&ctl->w_empty[slot]));
+          }
+          ptx::umma_commit(ptx::smem_u32(&ctl->d_ready[0]));
+          produce(g);   // keep the ring full while the workers requantise
+        }
+      }
+    }
+    __syncwarp();
+    cta_barrier();     // every MMA of step i has completed (the workers waited for each accumulator)
+  }
+  if (st.nsteps > 0 && !st.is_prior(st.nsteps - 1)) cta_barrier();   // trailing translation pass
+}
+
 // ---- workers ----------------------------------------------------------------------------------
 template <bool kInv>
 __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const LevelArgs& a, const Steps& st, int img0, int pvalid,
@@ -701,7 +810,10 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
       ptx::mbar_init(ptx::smem_u32(&ctl.d_ready[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&ctl.meta_full[s]), 1);
     }
-    for (int s = 0; s < 3; ++s) ptx::mbar_init(ptx::smem_u32(&ctl.w_full[s]), 1);
+    for (int s = 0; s < 3; ++s) {
+      ptx::mbar_init(ptx::smem_u32(&ctl.w_full[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl.w_empty[s]), 1);
+    }
     ptx::mbar_init_fence();
     ctl.abort = 0;
   }
@@ -741,7 +853,8 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
 
   if (warp >= kWorkerWarps) {
     cta_barrier();                       // the workers have loaded the flow variable
-    run_control(cx, P, a, st, ntv);
+    if (P.streamed) run_control_streamed(cx, P, a, st, ntv);
+    else run_control(cx, P, a, st, ntv);
   } else {
     int32_t* acc = reinterpret_cast<int32_t*>(smem + P.s_acc);
     for (int idx = tid; idx < P.cb * pg; idx += kWorkers) acc[idx] = 0;

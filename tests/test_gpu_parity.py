@@ -56,6 +56,8 @@ def _check_both_ways(G, model, x, max_batch=None, sample=None):
     (12, [True, False], 20, (0.4, 0.7), 7),      # 36-px and 9-px levels: tiles straddle images
     (4, [True], 8, None, 70),                    # 4-px level: 32 images per CTA, three CTAs
     (32, [True, True], 64, (0.4, 0.7), 3),       # 256-px level: two tiles per image
+    (16, [True, True], 320, None, 5),            # hidden width above 256: weights streamed in K-slices
+    (8, [True], 500, (0.6, 1.0), 3),             # odd widths between 300 and 500
 ])
 def test_small_models_bit_exact(G, hw, splits, hidden, prune, batch):
     model = S.make_model(100 + hw, 3, hw, hw, splits, 3, hidden, prune=prune)
@@ -190,6 +192,21 @@ def test_config4_batch_sweep_pruned(G, batch):
     model = S.config_model(4)
     x = S.config_images(4, batch=batch)
     pick = sorted(set([0, batch - 1] + S.Stream(batch, "pick").integers(0, batch, 10).tolist()))
+    m, z = _check_both_ways(G, model, x, sample=pick)
+    if batch > 64:
+        for b0 in range(0, batch, 64):
+            z64, _ = G.iodf_forward(m, _t(x[b0:b0 + 64]))
+            np.testing.assert_array_equal(z64.cpu().numpy(), z[b0:b0 + 64])
+        G.iodf_check(m)
+
+
+@pytest.mark.parametrize("batch", [1, 8, 64, 512, 2048])
+def test_config4_batch_sweep_stress_width_512(G, batch):
+    """The unpruned width-512 variant of the ImageNet64-shaped flow (weights streamed from L2 per
+    tile). The oracle checks up to 6 sampled images per batch size."""
+    model = S.config_model("4s")
+    x = S.config_images("4s", batch=batch)
+    pick = sorted(set([0, batch - 1] + S.Stream(batch, "pick512").integers(0, batch, 4).tolist()))
     m, z = _check_both_ways(G, model, x, sample=pick)
     if batch > 64:
         for b0 in range(0, batch, 64):
