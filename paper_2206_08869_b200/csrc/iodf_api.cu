@@ -261,9 +261,13 @@ uint32_t pow2_cols(uint32_t need) {
 //   mode 3: one tile slot, weights streamed per tile in 32-byte K-slices through a small ring
 //           (the only mode for hidden widths above 256: a 512 x 512 matrix alone is 256 KB)
 bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32_t wmax[3], uint32_t n_max,
-               uint32_t limit, uint32_t max_batch) {
+               uint32_t limit, uint32_t max_batch, int num_sms) {
   int group = P.px >= kTileM ? 1 : kTileM / P.px;
   group = std::max(1, std::min<int>(group, (int)max_batch));
+  // A level's time is set by the serial chain of its couplings inside one CTA, not by how many
+  // rows of the 128-row tile are filled: while the CTAs of a full batch would not fill the SMs,
+  // smaller groups (more CTAs, emptier tiles) are faster.
+  while (group > 1 && ((int)max_batch + group - 1) / group < num_sms) group /= 2;
   for (; group >= 1; group = (group > 1 ? group / 2 : 0)) {
     const int tiles = (group * P.px + kTileM - 1) / kTileM;
     for (int mode = 0; mode < 4; ++mode) {
@@ -406,6 +410,8 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
   CU(m, cudaSetDevice(device));
   CU(m, cudaDeviceGetAttribute(&smem_limit, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
   smem_limit -= 1024;   // static control block and alignment slack
+  int num_sms = 1;
+  CU(m, cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, device));
 
   // pass 2: pack and plan
   m->levels.resize(desc->n_levels);
@@ -467,7 +473,7 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
       wmax[0] = std::max(wmax[0], P.prior.w_bytes[0]);
     }
     if (hl.blob.empty()) hl.blob.resize(kAlign, 0);
-    if (!plan_smem(P, a_bytes, meta, wmax, n_max, (uint32_t)smem_limit, desc->max_batch))
+    if (!plan_smem(P, a_bytes, meta, wmax, n_max, (uint32_t)smem_limit, desc->max_batch, num_sms))
       return IODF_EUNSUPPORTED;
     max_smem = std::max(max_smem, P.s_total);
     if (lv.split) c = (uint32_t)ca;

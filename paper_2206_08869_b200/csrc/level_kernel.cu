@@ -234,27 +234,32 @@ struct Requant {
 };
 
 // TMEM accumulator -> requantised int8 activations in the next GEMM's A layout. n is a multiple
-// of 16; kd (the next GEMM's K) is n rounded up to 32, the extra chunk being zero.
+// of 16; kd (the next GEMM's K) is n rounded up to 32, the extra chunk being zero. The unit of work
+// is one 16-column chunk (= one 16-byte piece of the A row), dealt round-robin to the column
+// splits so that they differ by at most one chunk; a warp takes its chunks two at a time.
 template <int kMode, int kClip>
 __device__ __forceinline__ void epilogue_hidden_t(const Ctx& cx, int n, int kd, const Requant<kMode, kClip> q,
                                                   uint8_t* __restrict__ sOut) {
-  const int nblk = (n + 31) >> 5;
-  for (int b = cx.cs; b < nblk; b += cx.ncs) {
-    const int c0 = b << 5;
-    uint8_t* dst = sOut + (size_t)(2 * b) * (kTileM * 16) + cx.row * 16;
-    if (n - c0 >= 32) {
-      uint32_t r[32];
-      ptx::tmem_ld32(cx.tmem_slot + (uint32_t)c0, r);
-      ptx::tmem_ld_wait32(r);
-      *reinterpret_cast<uint4*>(dst) = q.chunk(r, c0);
-      *reinterpret_cast<uint4*>(dst + kTileM * 16) = q.chunk(r + 16, c0 + 16);
-    } else {
-      uint32_t r[16];
-      ptx::tmem_ld16(cx.tmem_slot + (uint32_t)c0, r);
-      ptx::tmem_ld_wait16(r);
-      *reinterpret_cast<uint4*>(dst) = q.chunk(r, c0);
-      if (c0 + 16 < kd) *reinterpret_cast<uint4*>(dst + kTileM * 16) = make_uint4(0u, 0u, 0u, 0u);
-    }
+  const int nch = n >> 4;
+  uint8_t* out = sOut + cx.row * 16;
+  if (kd > n && (nch % cx.ncs) == cx.cs)
+    *reinterpret_cast<uint4*>(out + (size_t)nch * (kTileM * 16)) = make_uint4(0u, 0u, 0u, 0u);
+  int ch = cx.cs;
+  for (; ch + cx.ncs < nch; ch += 2 * cx.ncs) {
+    const int ch2 = ch + cx.ncs;
+    uint32_t ra[16], rb[16];
+    ptx::tmem_ld16(cx.tmem_slot + (uint32_t)(ch << 4), ra);
+    ptx::tmem_ld16(cx.tmem_slot + (uint32_t)(ch2 << 4), rb);
+    ptx::tmem_ld_wait16(ra);
+    ptx::tmem_ld_wait16(rb);
+    *reinterpret_cast<uint4*>(out + (size_t)ch * (kTileM * 16)) = q.chunk(ra, ch << 4);
+    *reinterpret_cast<uint4*>(out + (size_t)ch2 * (kTileM * 16)) = q.chunk(rb, ch2 << 4);
+  }
+  if (ch < nch) {
+    uint32_t ra[16];
+    ptx::tmem_ld16(cx.tmem_slot + (uint32_t)(ch << 4), ra);
+    ptx::tmem_ld_wait16(ra);
+    *reinterpret_cast<uint4*>(out + (size_t)ch * (kTileM * 16)) = q.chunk(ra, ch << 4);
   }
 }
 
