@@ -291,6 +291,7 @@ __device__ void epilogue_scatter(const Ctx& cx, int cb, int cbp, int32_t* __rest
   const int gpt = cbp >> 3;
   const int nunits = 3 * gpt;
   const uint32_t sm = rp.valid ? rp.smask : 0u;
+  const bool rows_align = (32 % w) == 0;     // every image row lies inside one warp's 32 pixels
   for (int u = cx.cs; u < nunits; u += cx.ncs) {
     const int du = (u >= 2 * gpt) ? 2 : ((u >= gpt) ? 1 : 0);
     const int gq = u - du * gpt;
@@ -309,23 +310,39 @@ __device__ void epilogue_scatter(const Ctx& cx, int cb, int cbp, int32_t* __rest
     // outside the image (all three contributions share its row, hence its vertical validity)
     const uint32_t dst = ptx::smem_u32(acc + c0 * pg + rp.p - (du - 1) * w);
     const uint32_t plane = (uint32_t)pg * 4u;
-    const bool edge_hi = cx.lane == 31 && ok_m, edge_lo = cx.lane == 0 && ok_p;
-    int sum[8];
+    if (rows_align) {
+      // Image rows never straddle a warp (w divides 32): the lane that a rotating shuffle wraps to
+      // holds the first (last) pixel of a row, whose dv = +1 (-1) contribution is masked, i.e.
+      // zero. So no edge handling is needed at all.
+      int sum[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {                        // branch-free: eight independent chains
-      const int v_m = ok_m ? (int)r0[i] : 0;
-      const int v_0 = ok_0 ? (int)r1[i] : 0;
-      const int v_p = ok_p ? (int)r2[i] : 0;
-      const int from_next = __shfl_down_sync(0xFFFFFFFFu, v_p, 1);   // lane L+1's dv=+1 lands here
-      const int from_prev = __shfl_up_sync(0xFFFFFFFFu, v_m, 1);     // lane L-1's dv=-1 lands here
-      sum[i] = v_0 + (cx.lane < 31 ? from_next : 0) + (cx.lane > 0 ? from_prev : 0);
-    }
+      for (int i = 0; i < 8; ++i) {
+        const int v_m = ok_m ? (int)r0[i] : 0;
+        const int v_0 = ok_0 ? (int)r1[i] : 0;
+        const int v_p = ok_p ? (int)r2[i] : 0;
+        sum[i] = v_0 + __shfl_sync(0xFFFFFFFFu, v_p, (cx.lane + 1) & 31) + __shfl_sync(0xFFFFFFFFu, v_m, (cx.lane + 31) & 31);
+      }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const bool ch = c0 + i < cb;
-      ptx::red_add_s32(dst + (uint32_t)i * plane, sum[i], ch && ok_0);
-      ptx::red_add_s32(dst + (uint32_t)i * plane + 4u, (int)r0[i], ch && edge_hi);
-      ptx::red_add_s32(dst + (uint32_t)i * plane - 4u, (int)r2[i], ch && edge_lo);
+      for (int i = 0; i < 8; ++i) ptx::red_add_s32(dst + (uint32_t)i * plane, sum[i], (c0 + i < cb) && ok_0);
+    } else {
+      const bool edge_hi = cx.lane == 31 && ok_m, edge_lo = cx.lane == 0 && ok_p;
+      int sum[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {                        // branch-free: eight independent chains
+        const int v_m = ok_m ? (int)r0[i] : 0;
+        const int v_0 = ok_0 ? (int)r1[i] : 0;
+        const int v_p = ok_p ? (int)r2[i] : 0;
+        const int from_next = __shfl_down_sync(0xFFFFFFFFu, v_p, 1);   // lane L+1's dv=+1 lands here
+        const int from_prev = __shfl_up_sync(0xFFFFFFFFu, v_m, 1);     // lane L-1's dv=-1 lands here
+        sum[i] = v_0 + (cx.lane < 31 ? from_next : 0) + (cx.lane > 0 ? from_prev : 0);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const bool ch = c0 + i < cb;
+        ptx::red_add_s32(dst + (uint32_t)i * plane, sum[i], ch && ok_0);
+        ptx::red_add_s32(dst + (uint32_t)i * plane + 4u, (int)r0[i], ch && edge_hi);
+        ptx::red_add_s32(dst + (uint32_t)i * plane - 4u, (int)r2[i], ch && edge_lo);
+      }
     }
   }
 }
