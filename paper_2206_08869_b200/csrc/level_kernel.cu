@@ -314,16 +314,23 @@ __device__ void epilogue_scatter(const Ctx& cx, int cb, int cbp, int32_t* __rest
       // Image rows never straddle a warp (w divides 32): the lane that a rotating shuffle wraps to
       // holds the first (last) pixel of a row, whose dv = +1 (-1) contribution is masked, i.e.
       // zero. So no edge handling is needed at all.
+      // Masks are applied at the receiver as 0/1 multipliers (the neighbours' mask bits come over
+      // with one shuffle per unit), so each channel costs two shuffles and three multiply-adds.
+      const int k_0 = ok_0 ? 1 : 0;
+      const int k_p = __shfl_sync(0xFFFFFFFFu, ok_p ? 1 : 0, (cx.lane + 1) & 31);
+      const int k_m = __shfl_sync(0xFFFFFFFFu, ok_m ? 1 : 0, (cx.lane + 31) & 31);
       int sum[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        const int v_m = ok_m ? (int)r0[i] : 0;
-        const int v_0 = ok_0 ? (int)r1[i] : 0;
-        const int v_p = ok_p ? (int)r2[i] : 0;
-        sum[i] = v_0 + __shfl_sync(0xFFFFFFFFu, v_p, (cx.lane + 1) & 31) + __shfl_sync(0xFFFFFFFFu, v_m, (cx.lane + 31) & 31);
+        const int n_p = __shfl_sync(0xFFFFFFFFu, (int)r2[i], (cx.lane + 1) & 31);
+        const int n_m = __shfl_sync(0xFFFFFFFFu, (int)r0[i], (cx.lane + 31) & 31);
+        sum[i] = (int)r1[i] * k_0 + n_p * k_p + n_m * k_m;
       }
+      if (ok_0) {      // the row sum is zero otherwise
 #pragma unroll
-      for (int i = 0; i < 8; ++i) ptx::red_add_s32(dst + (uint32_t)i * plane, sum[i], (c0 + i < cb) && ok_0);
+        for (int i = 0; i < 8; ++i)
+          if (c0 + i < cb) ptx::red_add_s32_always(dst + (uint32_t)i * plane, sum[i]);
+      }
     } else {
       const bool edge_hi = cx.lane == 31 && ok_m, edge_lo = cx.lane == 0 && ok_p;
       int sum[8];

@@ -57,6 +57,10 @@ __device__ __forceinline__ void red_add_s32(uint32_t saddr, int val, bool pred) 
       : "memory");
 }
 
+__device__ __forceinline__ void red_add_s32_always(uint32_t saddr, int val) {
+  asm volatile("red.shared.add.s32 [%0], %1;" ::"r"(saddr), "r"(val) : "memory");
+}
+
 // ---- bulk copy global -> shared, completion counted on an mbarrier ---------------------------
 // dst, src and bytes must be multiples of 16.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
