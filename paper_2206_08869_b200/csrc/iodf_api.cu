@@ -433,6 +433,9 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
     P.d = lay.d; P.d_fact = lay.d_fact;
 
     P.cpad = (int)up(ca, 8); P.cbp = (int)up(cb, 8);
+    auto magic = [](uint64_t d) -> uint32_t { return d <= 1 ? 0u : (uint32_t)(((1ull << 32) + d - 1) / d); };
+    P.mul_per_img = magic((uint64_t)c * h * w); P.mul_4px = magic(4ull * h * w); P.mul_w2 = magic(2ull * w);
+    P.mul_px = magic((uint64_t)h * w); P.mul_w = magic(w);
     P.recip_gpa = 65536u / (uint32_t)(P.cpad / 8) + 1u;
     P.recip_gpb = 65536u / (uint32_t)(P.cbp / 8) + 1u;
     std::vector<int> pi(c);
@@ -475,6 +478,8 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
     if (hl.blob.empty()) hl.blob.resize(kAlign, 0);
     if (!plan_smem(P, a_bytes, meta, wmax, n_max, (uint32_t)smem_limit, desc->max_batch, num_sms))
       return IODF_EUNSUPPORTED;
+    // the index maps divide numbers below group * c * px by at most c * px with a 32-bit magic multiplier
+    if ((uint64_t)P.group * c * h * w * ((uint64_t)c * h * w) >= (1ull << 32)) return IODF_EUNSUPPORTED;
     max_smem = std::max(max_smem, P.s_total);
     if (lv.split) c = (uint32_t)ca;
   }

@@ -98,6 +98,8 @@ struct LevelPlan {
   uint32_t ring_slot_bytes;
   // shared-memory byte offsets
   uint32_t s_v, s_xa, s_acc, s_rowinfo, s_a[2], s_meta[2], s_w[3], s_total;
+  // magic multipliers for the index maps: n / d = umulhi(n, ceil(2^32 / d)) for n * d < 2^32 (0: d = 1)
+  uint32_t mul_per_img, mul_4px, mul_w2, mul_px, mul_w;
   uint32_t recip_gpa, recip_gpb; // floor(g / (cpad/8)) = (g * recip_gpa) >> 16 for g < 4096; same for cbp/8
   // global layout
   uint64_t z_off, prior_off, z_final_off, d, d_fact;

@@ -89,6 +89,9 @@ __device__ __forceinline__ int32_t rq_exact(int32_t a, int32_t m0, int32_t s) {
 
 __device__ __forceinline__ int clampi(int v, int lo, int hi) { return min(max(v, lo), hi); }
 
+// n / d with the plan's magic multiplier ceil(2^32 / d) (0 stands for d = 1); exact while n * d < 2^32
+__device__ __forceinline__ int fdiv(int n, uint32_t mul) { return mul ? (int)__umulhi((uint32_t)n, mul) : n; }
+
 __device__ __forceinline__ uint32_t pack4(int y0, int y1, int y2, int y3) {
   const uint32_t a = __byte_perm((uint32_t)y0, (uint32_t)y1, 0x0040);
   const uint32_t b = __byte_perm((uint32_t)y2, (uint32_t)y3, 0x0040);
@@ -104,11 +107,12 @@ struct RowPos {
 };
 
 // Packed row record: bit 0 valid, bits 1..9 gather mask, bits 10..18 scatter mask.
-__device__ __forceinline__ uint32_t row_record(int p, int pvalid, int px, int h, int w) {
+__device__ __forceinline__ uint32_t row_record(int p, int pvalid, int px, int h, int w, uint32_t mul_px,
+                                               uint32_t mul_w) {
   if (p >= pvalid) return 0u;
   uint32_t r = 1u;
-  const int q = p % px;
-  const int i = q / w, j = q - i * w;
+  const int q = p - fdiv(p, mul_px) * px;
+  const int i = fdiv(q, mul_w), j = q - i * w;
 #pragma unroll
   for (int u = 0; u < 3; ++u)
 #pragma unroll
@@ -888,14 +892,15 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
     int32_t* acc = reinterpret_cast<int32_t*>(smem + P.s_acc);
     for (int idx = tid; idx < P.cb * pg; idx += kWorkers) acc[idx] = 0;
     uint32_t* rowinfo = reinterpret_cast<uint32_t*>(smem + P.s_rowinfo);
-    for (int idx = tid; idx < P.tiles * kTileM; idx += kWorkers) rowinfo[idx] = row_record(idx, pvalid, px, P.h, w);
+    for (int idx = tid; idx < P.tiles * kTileM; idx += kWorkers) rowinfo[idx] = row_record(idx, pvalid, px, P.h, w, P.mul_px, P.mul_w);
     if (!kInv) {
       // space-to-depth on load: plane c*4 + dy*2 + dx, pixel (i, j) <- in[c][2i+dy][2j+dx]
       const int w2 = 2 * w;
+#pragma unroll 4
       for (int e = tid; e < nimg * per_img; e += kWorkers) {
-        const int g = e / per_img, r = e - g * per_img;
-        const int ci = r / (4 * px), r2 = r - ci * 4 * px;
-        const int y = r2 / w2, x = r2 - y * w2;
+        const int g = fdiv(e, P.mul_per_img), r = e - g * per_img;
+        const int ci = fdiv(r, P.mul_4px), r2 = r - ci * 4 * px;
+        const int y = fdiv(r2, P.mul_w2), x = r2 - y * w2;
         const size_t src = (size_t)(img0 + g) * per_img + r;
         const int32_t val = P.is_first ? (int32_t) reinterpret_cast<const uint8_t*>(a.in)[src]
                                        : reinterpret_cast<const int32_t*>(a.in)[src];
@@ -903,9 +908,10 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
       }
     } else {
       // merge: logical channel k < keep_c from the deeper level, the rest from z's block of this level
+#pragma unroll 4
       for (int e = tid; e < nimg * per_img; e += kWorkers) {
-        const int g = e / per_img, r = e - g * per_img;
-        const int k = r / px, q = r - k * px;
+        const int g = fdiv(e, P.mul_per_img), r = e - g * per_img;
+        const int k = fdiv(r, P.mul_px), q = r - k * px;
         const size_t b = (size_t)(img0 + g);
         const int32_t val =
             (k < P.keep_c) ? reinterpret_cast<const int32_t*>(a.in)[b * (size_t)a.in_stride + (size_t)k * px + q]
@@ -921,9 +927,10 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
       // split on store: factored-out half -> z block of this level; kept half -> next level (or
       // the final z block)
       int32_t* keep_out = reinterpret_cast<int32_t*>(a.out);
+#pragma unroll 4
       for (int e = tid; e < nimg * per_img; e += kWorkers) {
-        const int g = e / per_img, r = e - g * per_img;
-        const int k = r / px, q = r - k * px;
+        const int g = fdiv(e, P.mul_per_img), r = e - g * per_img;
+        const int k = fdiv(r, P.mul_px), q = r - k * px;
         const size_t b = (size_t)(img0 + g);
         const int32_t val = v[P.col_out[k] * pg + g * px + q];
         if (k >= P.keep_c) a.z[b * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q] = val;
@@ -934,10 +941,11 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
       // depth-to-space on store
       const int w2 = 2 * w;
       uint32_t bad = 0;
+#pragma unroll 4
       for (int e = tid; e < nimg * per_img; e += kWorkers) {
-        const int g = e / per_img, r = e - g * per_img;
-        const int ci = r / (4 * px), r2 = r - ci * 4 * px;
-        const int y = r2 / w2, x = r2 - y * w2;
+        const int g = fdiv(e, P.mul_per_img), r = e - g * per_img;
+        const int ci = fdiv(r, P.mul_4px), r2 = r - ci * 4 * px;
+        const int y = fdiv(r2, P.mul_w2), x = r2 - y * w2;
         const int32_t val = v[(ci * 4 + (y & 1) * 2 + (x & 1)) * pg + g * px + (y >> 1) * w + (x >> 1)];
         const size_t dst = (size_t)(img0 + g) * per_img + r;
         if (P.is_first) {
