@@ -488,6 +488,8 @@ __device__ void run_control(const Ctx& cx, const LevelPlan& P, const LevelArgs& 
       W.s0_loads = 1;
     }
   }
+  __syncwarp();
+  cta_barrier();                         // the workers have loaded the flow variable
   // wait for tile slot sl's A operand, then D = A * W^T into the slot's TMEM columns
   auto mma = [&](int sl, int wslot, bool wait_w, uint32_t wpar, int n, int kd) {
     wait_bar(ctl, a.status, &ctl->a_ready[sl], apar[sl]);
@@ -837,6 +839,7 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
   const LevelPlan& P = *a.plan;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
+  ptx::grid_launch_dependents();         // the next kernel in the stream may start its prologue
   if (tid == 0) {
     for (int s = 0; s < 2; ++s) {
       ptx::mbar_init(ptx::smem_u32(&ctl.a_ready[s]), (uint32_t)kWorkers);
@@ -885,14 +888,22 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
   cx.tmem_slot = tmem + ((uint32_t)(cx.wq * 32) << 16);
 
   if (warp >= kWorkerWarps) {
-    cta_barrier();                       // the workers have loaded the flow variable
-    if (P.streamed) run_control_streamed(cx, P, a, st, ntv);
-    else run_control(cx, P, a, st, ntv);
+    // The packed blocks are written once at model creation, so the first copies need not wait for
+    // the previous kernel; run_control starts them before it joins the workers' first barrier.
+    if (P.streamed) {
+      cta_barrier();                     // the workers have loaded the flow variable
+      run_control_streamed(cx, P, a, st, ntv);
+    } else {
+      run_control(cx, P, a, st, ntv);
+    }
   } else {
     int32_t* acc = reinterpret_cast<int32_t*>(smem + P.s_acc);
     for (int idx = tid; idx < P.cb * pg; idx += kWorkers) acc[idx] = 0;
     uint32_t* rowinfo = reinterpret_cast<uint32_t*>(smem + P.s_rowinfo);
     for (int idx = tid; idx < P.tiles * kTileM; idx += kWorkers) rowinfo[idx] = row_record(idx, pvalid, px, P.h, w, P.mul_px, P.mul_w);
+    // Everything above used only the plan; from here on the kernel reads what the previous kernel
+    // in the stream wrote and writes what it may still be reading.
+    ptx::grid_dependency_wait();
     if (!kInv) {
       // space-to-depth on load: plane c*4 + dy*2 + dx, pixel (i, j) <- in[c][2i+dy][2j+dx]
       const int w2 = 2 * w;
@@ -970,9 +981,21 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
 }  // namespace
 
 cudaError_t launch_level(const LevelArgs& args, bool inverse, int grid, uint32_t smem_bytes, cudaStream_t stream) {
-  if (inverse) level_kernel<true><<<grid, kThreads, smem_bytes, stream>>>(args);
-  else level_kernel<false><<<grid, kThreads, smem_bytes, stream>>>(args);
-  return cudaGetLastError();
+  // Programmatic dependent launch: the CTAs of this level may start (barrier set-up, TMEM
+  // allocation, index records) while the previous kernel in the stream drains; the kernel itself
+  // waits for that kernel's completion before it touches anything a kernel writes.
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)kThreads);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (inverse) return cudaLaunchKernelEx(&cfg, level_kernel<true>, args);
+  return cudaLaunchKernelEx(&cfg, level_kernel<false>, args);
 }
 
 cudaError_t configure_level_kernels(uint32_t max_smem_bytes) {
