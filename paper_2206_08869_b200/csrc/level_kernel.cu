@@ -42,7 +42,7 @@ namespace iodf {
 namespace {
 
 struct __align__(16) Ctl {
-  uint64_t a_ready[2];    // workers -> control: the tile slot's A operand is written (count = workers)
+  uint64_t a_ready[2];    // workers -> control: the tile slot's A operand is written (count = worker warps)
   uint64_t d_ready[2];    // tensor core -> workers: the tile slot's accumulator is complete
   uint64_t w_full[3];     // bulk copy -> control: weight slot (or ring slot) filled
   uint64_t w_empty[3];    // tensor core -> control: the MMAs reading a ring slot have completed
@@ -702,11 +702,14 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
     sA = smem + P.s_a[sl];
     cx.tmem_slot = cx.tmem_base + (uint32_t)(sl * kSlotCols) + ((uint32_t)(cx.wq * 32) << 16);
   };
-  // this thread's part of tile slot sl's A operand is written (and its TMEM reads are done)
+  // this warp's part of tile slot sl's A operand is written (and its TMEM reads are done): every
+  // lane fences its own writes towards the async proxy, the warp synchronises, one lane arrives
   auto arrive_a = [&](int sl) {
     ptx::tc_fence_before();
     ptx::fence_async_smem();
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ptx::smem_u32(&ctl->a_ready[sl])) : "memory");
+    __syncwarp();
+    if (cx.lane == 0)
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ptx::smem_u32(&ctl->a_ready[sl])) : "memory");
   };
   auto wait_d = [&](int sl) {
     wait_bar(ctl, a.status, &ctl->d_ready[sl], dpar[sl]);
@@ -842,7 +845,7 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
   ptx::grid_launch_dependents();         // the next kernel in the stream may start its prologue
   if (tid == 0) {
     for (int s = 0; s < 2; ++s) {
-      ptx::mbar_init(ptx::smem_u32(&ctl.a_ready[s]), (uint32_t)kWorkers);
+      ptx::mbar_init(ptx::smem_u32(&ctl.a_ready[s]), (uint32_t)kWorkerWarps);
       ptx::mbar_init(ptx::smem_u32(&ctl.d_ready[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&ctl.meta_full[s]), 1);
     }
