@@ -221,6 +221,38 @@ def main():
                 "level_ms": [float(v) for v in lvl],
                 "whole_step_frac": (2.0 * macs * B / (total_ms / args.steps * 1e-3) / 1e12) / peak_int8}
 
+    # ---- decode of the same workload, and batch-1 latency of both directions ------------------
+    # zs hold valid latents of the encoded sets; the decoder must give the images back.
+    xo = [torch.empty_like(xs[0]) for _ in range(N_SETS)]
+    dec_steps = max(10, min(args.steps, 200))
+    for i in range(max(3, min(args.warmup, 10))):
+        G.iodf_inverse(m, zs[i % N_SETS], xo[i % N_SETS])
+    barrier()
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    d0.record(stream)
+    for i in range(dec_steps):
+        G.iodf_inverse(m, zs[i % N_SETS], xo[i % N_SETS])
+    d1.record(stream)
+    barrier()
+    dec_ms = d0.elapsed_time(d1)
+    G.iodf_check(m)
+    dec_ok = bool(all(torch.equal(xo[i], xs[i]) for i in range(min(N_SETS, args.steps + args.warmup))))
+
+    def latency_b1(fn):
+        ts = []
+        for i in range(23):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn(i % N_SETS)
+            b.record(stream)
+            b.synchronize()
+            ts.append(a.elapsed_time(b))
+        ts = sorted(ts[3:])
+        return {"median_ms": ts[len(ts) // 2], "min_ms": ts[0]}
+    lat = {"encode": latency_b1(lambda i: G.iodf_forward(m, xs[i][:1], zs[i][:1], ps[i][:1])),
+           "decode": latency_b1(lambda i: G.iodf_inverse(m, zs[i][:1], xo[i][:1]))}
+    G.iodf_check(m)
+
     # ---- end to end through the host-buffer entry point --------------------------------------
     hx = [torch.from_numpy(S.config_images(cfg, batch=B, seed_offset=rank_seed_offset(rank, i))).pin_memory() for i in range(2)]
     hz = [torch.empty((B, m.d), dtype=torch.int32).pin_memory() for _ in range(2)]
@@ -237,7 +269,7 @@ def main():
     e2e_s = time.perf_counter() - t0
     G.iodf_check(m)
 
-    total_ms, e2e_s = max_over_ranks([total_ms, e2e_s], world, dev)
+    total_ms, e2e_s, dec_ms = max_over_ranks([total_ms, e2e_s, dec_ms], world, dev)
 
     if rank == 0:
         cores = os.cpu_count() or 1
@@ -251,6 +283,10 @@ def main():
                     "d2h_bytes_per_step": B * m.d * 4 + B * 2 * m.d_fact * 4, "steps": e2e_steps},
             "gpu_launches": G.iodf_launches_per_call(m) * args.steps,
             "gops_per_image": 2.0 * macs / 1e9,
+            "decode": {"metric": "flow_decode_images_per_sec", "value": job_throughput(B, world, dec_steps, dec_ms * 1e-3),
+                       "unit": UNIT, "ms_per_step": dec_ms / dec_steps, "steps": dec_steps,
+                       "round_trip_exact": dec_ok},
+            "latency_batch1": lat,
         }
         if world == 1:
             r, n, dt = oracle_rate(model, cfg, B, cores)
