@@ -78,6 +78,15 @@ __device__ __noinline__ bool wait_bar(Ctl* ctl, uint32_t* status, uint64_t* bar,
   return false;
 }
 
+// The control thread's waits are short and on the critical path of every tile phase: it polls
+// inline first (no call, no suspension) and only then falls back to the bounded blocking wait.
+__device__ __forceinline__ void spin_then_wait(Ctl* ctl, uint32_t* status, uint64_t* bar, uint32_t parity) {
+  const uint32_t b = ptx::smem_u32(bar);
+  for (int it = 0; it < 2048; ++it)
+    if (ptx::mbar_test_wait(b, parity)) return;
+  wait_bar(ctl, status, bar, parity);
+}
+
 __device__ __forceinline__ void cta_barrier() { __syncthreads(); }
 
 
@@ -492,9 +501,9 @@ __device__ void run_control(const Ctx& cx, const LevelPlan& P, const LevelArgs& 
   cta_barrier();                         // the workers have loaded the flow variable
   // wait for tile slot sl's A operand, then D = A * W^T into the slot's TMEM columns
   auto mma = [&](int sl, int wslot, bool wait_w, uint32_t wpar, int n, int kd) {
-    wait_bar(ctl, a.status, &ctl->a_ready[sl], apar[sl]);
+    spin_then_wait(ctl, a.status, &ctl->a_ready[sl], apar[sl]);
     apar[sl] ^= 1u;
-    if (wait_w) wait_bar(ctl, a.status, &ctl->w_full[wslot], wpar);
+    if (wait_w) spin_then_wait(ctl, a.status, &ctl->w_full[wslot], wpar);
     ptx::tc_fence_after();
     const uint32_t sa = ptx::smem_u32(smem + P.s_a[sl]), sb = ptx::smem_u32(smem + P.s_w[wslot]);
     const uint32_t d = cx.tmem_base + (uint32_t)(sl * kSlotCols);
