@@ -80,11 +80,13 @@ __device__ __noinline__ bool wait_bar(Ctl* ctl, uint32_t* status, uint64_t* bar,
 
 // The control thread's waits are short and on the critical path of every tile phase: it polls
 // inline first (no call, no suspension) and only then falls back to the bounded blocking wait.
-__device__ __forceinline__ void spin_then_wait(Ctl* ctl, uint32_t* status, uint64_t* bar, uint32_t parity) {
-  const uint32_t b = ptx::smem_u32(bar);
+__device__ __forceinline__ void spin_then_wait(Ctl* ctl, uint32_t* status, uint64_t* bar, uint32_t b, uint32_t parity) {
   for (int it = 0; it < 2048; ++it)
     if (ptx::mbar_test_wait(b, parity)) return;
   wait_bar(ctl, status, bar, parity);
+}
+__device__ __forceinline__ void spin_then_wait(Ctl* ctl, uint32_t* status, uint64_t* bar, uint32_t parity) {
+  spin_then_wait(ctl, status, bar, ptx::smem_u32(bar), parity);
 }
 
 __device__ __forceinline__ void cta_barrier() { __syncthreads(); }
@@ -542,6 +544,52 @@ __device__ void run_control(const Ctx& cx, const LevelPlan& P, const LevelArgs& 
       const BlockRef& br = step_ref(P, st, i);
       const int nstages = prior ? 1 : 3;
       bool first = true;
+      // Common case (a coupling, every matrix resident, no accumulator wider than one MMA): every
+      // instruction of this thread between a tile's last arrival and its commit delays the tile, so
+      // the descriptors of the step's three GEMMs are built once and the issue path is unrolled.
+      const bool lean = !alias && !prior && n[0] <= 256 && n[1] <= 256 && n[2] <= 256;
+      if (lean) {
+        uint32_t idesc[3], db_lo[3], db_step[3];
+        int ks[3];
+#pragma unroll
+        for (int sg = 0; sg < 3; ++sg) {
+          const uint32_t lbo_b = (uint32_t)n[sg] * 16u;
+          idesc[sg] = ptx::umma_idesc_s8((uint32_t)n[sg]);
+          db_lo[sg] = ptx::umma_desc_lo(ptx::smem_u32(smem + P.s_w[sg]), lbo_b);
+          db_step[sg] = (2u * lbo_b) >> 4;
+          ks[sg] = kd[sg] >> 5;
+        }
+        const uint32_t da_lo[2] = {ptx::umma_desc_lo(ptx::smem_u32(smem + P.s_a[0]), kTileM * 16),
+                                   ptx::umma_desc_lo(ptx::smem_u32(smem + P.s_a[1]), kTileM * 16)};
+        const uint32_t da_step = (2u * kTileM * 16u) >> 4;
+        const uint32_t abar[2] = {ptx::smem_u32(&ctl->a_ready[0]), ptx::smem_u32(&ctl->a_ready[1])};
+        const uint32_t dbar[2] = {ptx::smem_u32(&ctl->d_ready[0]), ptx::smem_u32(&ctl->d_ready[1])};
+        for (int t0 = 0; t0 < ntv; t0 += nslots) {
+          const int nt = min(nslots, ntv - t0);
+#pragma unroll
+          for (int sg = 0; sg < 3; ++sg) {
+#pragma unroll
+            for (int sl = 0; sl < 2; ++sl) {
+              if (sl < nt) {
+                spin_then_wait(ctl, a.status, &ctl->a_ready[sl], abar[sl], apar[sl]);
+                apar[sl] ^= 1u;
+                if (first && sl == 0) spin_then_wait(ctl, a.status, &ctl->w_full[sg], sg == 0 ? par0 : par12);
+                ptx::tc_fence_after();
+                const uint32_t d = cx.tmem_base + (uint32_t)(sl * kSlotCols);
+                uint32_t da = da_lo[sl], db = db_lo[sg];
+                ptx::umma_i8_lo(d, da, db, idesc[sg], 0u);
+                for (int k = 1; k < ks[sg]; ++k) {
+                  da += da_step;
+                  db += db_step[sg];
+                  ptx::umma_i8_lo(d, da, db, idesc[sg], 1u);
+                }
+                ptx::umma_commit(dbar[sl]);
+              }
+            }
+          }
+          first = false;
+        }
+      } else
       for (int t0 = 0; t0 < ntv; t0 += nslots) {
         const int nt = min(nslots, ntv - t0);
         const bool last_tile = t0 + nslots >= ntv;
