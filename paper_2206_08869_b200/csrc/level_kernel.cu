@@ -769,7 +769,8 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
       asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ptx::smem_u32(&ctl->a_ready[sl])) : "memory");
   };
   auto wait_d = [&](int sl) {
-    wait_bar(ctl, a.status, &ctl->d_ready[sl], dpar[sl]);
+    // often already complete: test inline before the call
+    if (!ptx::mbar_test_wait(ptx::smem_u32(&ctl->d_ready[sl]), dpar[sl])) wait_bar(ctl, a.status, &ctl->d_ready[sl], dpar[sl]);
     dpar[sl] ^= 1u;
     ptx::tc_fence_after();
   };
