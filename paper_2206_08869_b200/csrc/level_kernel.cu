@@ -770,7 +770,12 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
   };
   auto wait_d = [&](int sl) {
     // often already complete: test inline before the call
-    if (!ptx::mbar_test_wait(ptx::smem_u32(&ctl->d_ready[sl]), dpar[sl])) wait_bar(ctl, a.status, &ctl->d_ready[sl], dpar[sl]);
+    {
+      const uint32_t b = ptx::smem_u32(&ctl->d_ready[sl]);
+      // already complete (common), or complete within one suspended try: no call; else the bounded wait
+      if (!ptx::mbar_test_wait(b, dpar[sl]) && !ptx::mbar_try_wait(b, dpar[sl]))
+        wait_bar(ctl, a.status, &ctl->d_ready[sl], dpar[sl]);
+    }
     dpar[sl] ^= 1u;
     ptx::tc_fence_after();
   };
