@@ -564,6 +564,10 @@ __device__ void run_control(const Ctx& cx, const LevelPlan& P, const LevelArgs& 
         const uint32_t da_step = (2u * kTileM * 16u) >> 4;
         const uint32_t abar[2] = {ptx::smem_u32(&ctl->a_ready[0]), ptx::smem_u32(&ctl->a_ready[1])};
         const uint32_t dbar[2] = {ptx::smem_u32(&ctl->d_ready[0]), ptx::smem_u32(&ctl->d_ready[1])};
+        // The step's matrices were requested when the previous step ended and are normally here by
+        // now; waiting for them before the first arrival keeps the waits off the tiles' critical path.
+#pragma unroll
+        for (int sg = 0; sg < 3; ++sg) spin_then_wait(ctl, a.status, &ctl->w_full[sg], sg == 0 ? par0 : par12);
         for (int t0 = 0; t0 < ntv; t0 += nslots) {
           const int nt = min(nslots, ntv - t0);
 #pragma unroll
@@ -573,7 +577,6 @@ __device__ void run_control(const Ctx& cx, const LevelPlan& P, const LevelArgs& 
               if (sl < nt) {
                 spin_then_wait(ctl, a.status, &ctl->a_ready[sl], abar[sl], apar[sl]);
                 apar[sl] ^= 1u;
-                if (first && sl == 0) spin_then_wait(ctl, a.status, &ctl->w_full[sg], sg == 0 ? par0 : par12);
                 ptx::tc_fence_after();
                 const uint32_t d = cx.tmem_base + (uint32_t)(sl * kSlotCols);
                 uint32_t da = da_lo[sl], db = db_lo[sg];
@@ -587,7 +590,6 @@ __device__ void run_control(const Ctx& cx, const LevelPlan& P, const LevelArgs& 
               }
             }
           }
-          first = false;
         }
       } else
       for (int t0 = 0; t0 < ntv; t0 += nslots) {
