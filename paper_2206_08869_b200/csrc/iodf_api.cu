@@ -98,13 +98,33 @@ int hidden_range(const iodf_layer_desc& L, Act* out) {
   return IODF_OK;
 }
 
-// Fills both constant tables of a hidden layer and picks its requantisation flavour.
+// Bias folded into the GEMM: the A operand carries kBiasRows constant columns (1, 127, 127, ...)
+// and the weight matrix one row per column with bias = w[0] + 127 * (w[1] + ... + w[kBiasRows-1]),
+// every |w[j]| <= 127, so the accumulator already holds acc + bias and the epilogue needs the
+// multiplier only. Exact (integer sums); possible while |bias| <= kFoldMaxBias.
+constexpr int kBiasRows = 8;
+constexpr int64_t kFoldMaxBias = 63 + 127ll * 127ll * (kBiasRows - 1);
+void fold_bias(int32_t bias, int8_t w[kBiasRows]) {
+  const int64_t b = bias;
+  int64_t q = b >= 0 ? (b + 63) / 127 : -((-b + 63) / 127);
+  w[0] = (int8_t)(b - 127 * q);
+  for (int j = 1; j < kBiasRows; ++j) {
+    const int64_t t = std::max<int64_t>(-127, std::min<int64_t>(127, q));
+    w[j] = (int8_t)t;
+    q -= t;
+  }
+}
+
+// Fills the constant tables of a hidden layer and picks its requantisation flavour:
+//   3: one shift s >= 1 for the whole layer and every bias foldable: table of multipliers (mb[i])
+//   2: one shift s >= 1: table of {m0, bias} pairs (mb[2i], mb[2i+1])
+//   1 / 0: per-channel shifts (HiddenRq table)
 void put_hidden_rq(HiddenRq* dst, int32_t* mb, const iodf_layer_desc& L, const Blobs& B, int n_pad, int* mode,
                    int* uniform_s) {
   const int32_t* bias = B.r + L.requant_off;
   const int32_t* m0 = bias + L.c_out;
   const int32_t* s = m0 + L.c_out;
-  bool fast = true, uniform = true;
+  bool fast = true, uniform = true, foldable = true;
   for (int i = 0; i < n_pad; ++i) {
     HiddenRq h;
     if (i < (int)L.c_out) {
@@ -115,6 +135,7 @@ void put_hidden_rq(HiddenRq* dst, int32_t* mb, const iodf_layer_desc& L, const B
       h.c_hi = (uint32_t)((unsigned long long)c64 >> 32);
       if (s[i] < 1) fast = false;
       if (s[i] != s[0] || s[i] < 1) uniform = false;
+      if (std::llabs((long long)bias[i]) > kFoldMaxBias) foldable = false;
       mb[2 * i] = m0[i];
       mb[2 * i + 1] = bias[i];
     } else {  // padding channel: acc = 0 -> 0 (its weights in the next layer are zero anyway)
@@ -127,8 +148,10 @@ void put_hidden_rq(HiddenRq* dst, int32_t* mb, const iodf_layer_desc& L, const B
     }
     dst[i] = h;
   }
-  *mode = uniform ? 2 : (fast ? 1 : 0);
+  *mode = uniform ? (foldable ? 3 : 2) : (fast ? 1 : 0);
   *uniform_s = uniform ? s[0] : 0;
+  if (*mode == 3)
+    for (int i = 0; i < n_pad; ++i) mb[i] = i < (int)L.c_out ? m0[i] : (1 << 30);
 }
 
 void put_out_rq(OutRq* dst, const iodf_layer_desc& L, const Blobs& B) {
@@ -172,7 +195,8 @@ PackedBlock pack_coupling(const iodf_coupling_desc& cp, const Blobs& B, int ca, 
   const int cpad = (int)up(ca, 8), cbp = (int)up(cb, 8);
   Dims d;
   d.n1 = (int)up(k1, 16); d.n2 = (int)up(k2, 16); d.n3 = (int)up(9 * cbp, 16);
-  d.kd1 = (int)up(9 * cpad, 32); d.kd2 = (int)up(k1, 32); d.kd3 = (int)up(k2, 32);
+  // K of the first two GEMMs leaves room for the kBiasRows constant columns after the data
+  d.kd1 = (int)up(9 * cpad + kBiasRows, 32); d.kd2 = (int)up(d.n1 + kBiasRows, 32); d.kd3 = (int)up(k2, 32);
   *dims = d;
   PackedBlock pb;
   CouplingMeta M{};
@@ -188,15 +212,16 @@ PackedBlock pack_coupling(const iodf_coupling_desc& cp, const Blobs& B, int ca, 
   M.off_colA = (int)off; off += up(4 * ca, 16);
   M.off_colB = (int)off; off += up(4 * cb, 16);
   M.off_out = (int)off;  off += (uint32_t)sizeof(OutRq) * cb;
-  M.off_h1 = M.off_u1 = (int)off; off += M.mode1 == 2 ? 8u * d.n1 : (uint32_t)sizeof(HiddenRq) * d.n1;
-  M.off_h2 = M.off_u2 = (int)off; off += M.mode2 == 2 ? 8u * d.n2 : (uint32_t)sizeof(HiddenRq) * d.n2;
+  auto table_bytes = [](int mode, int n) { return mode == 3 ? 4u * n : mode == 2 ? 8u * n : (uint32_t)sizeof(HiddenRq) * n; };
+  M.off_h1 = M.off_u1 = (int)off; off += table_bytes(M.mode1, d.n1);
+  M.off_h2 = M.off_u2 = (int)off; off += table_bytes(M.mode2, d.n2);
   pb.meta.assign(off, 0);
   std::memcpy(pb.meta.data() + M.off_colA, colA, 4 * ca);
   std::memcpy(pb.meta.data() + M.off_colB, colB, 4 * cb);
   put_out_rq(reinterpret_cast<OutRq*>(pb.meta.data() + M.off_out), L3, B);
-  if (M.mode1 == 2) std::memcpy(pb.meta.data() + M.off_u1, u1.data(), 8u * d.n1);
+  if (M.mode1 >= 2) std::memcpy(pb.meta.data() + M.off_u1, u1.data(), table_bytes(M.mode1, d.n1));
   else std::memcpy(pb.meta.data() + M.off_h1, h1.data(), sizeof(HiddenRq) * d.n1);
-  if (M.mode2 == 2) std::memcpy(pb.meta.data() + M.off_u2, u2.data(), 8u * d.n2);
+  if (M.mode2 >= 2) std::memcpy(pb.meta.data() + M.off_u2, u2.data(), table_bytes(M.mode2, d.n2));
   else std::memcpy(pb.meta.data() + M.off_h2, h2.data(), sizeof(HiddenRq) * d.n2);
   std::memcpy(pb.meta.data(), &M, sizeof(M));
 
@@ -208,11 +233,27 @@ PackedBlock pack_coupling(const iodf_coupling_desc& cp, const Blobs& B, int ca, 
     for (int tap = 0; tap < 9; ++tap)
       for (int c = 0; c < ca; ++c)
         pb.w[0][wpos(d.n1, n, tap * cpad + c)] = (uint8_t)w1[((size_t)n * 9 + tap) * ca + c];
+  if (M.mode1 == 3) {            // bias rows right after the nine taps
+    const int32_t* b1 = B.r + L1.requant_off;
+    for (int n = 0; n < k1; ++n) {
+      int8_t bw[kBiasRows];
+      fold_bias(b1[n], bw);
+      for (int j = 0; j < kBiasRows; ++j) pb.w[0][wpos(d.n1, n, 9 * cpad + j)] = (uint8_t)bw[j];
+    }
+  }
   // W2: 1x1
   pb.w[1].assign((size_t)d.n2 * d.kd2, 0);
   const int8_t* w2 = B.w + L2.weight_off;
   for (int n = 0; n < k2; ++n)
     for (int k = 0; k < k1; ++k) pb.w[1][wpos(d.n2, n, k)] = (uint8_t)w2[(size_t)n * k1 + k];
+  if (M.mode2 == 3) {            // bias rows right after the (padded) hidden channels
+    const int32_t* b2 = B.r + L2.requant_off;
+    for (int n = 0; n < k2; ++n) {
+      int8_t bw[kBiasRows];
+      fold_bias(b2[n], bw);
+      for (int j = 0; j < kBiasRows; ++j) pb.w[1][wpos(d.n2, n, d.n1 + j)] = (uint8_t)bw[j];
+    }
+  }
   // W3': row = tap*cbp + c, K index = hidden channel
   pb.w[2].assign((size_t)d.n3 * d.kd3, 0);
   const int8_t* w3 = B.w + L3.weight_off;

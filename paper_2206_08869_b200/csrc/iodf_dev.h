@@ -9,6 +9,10 @@
 //     bytes; consecutive 8-row groups are 128 bytes apart (stride-dimension offset) and
 //     consecutive 16-byte K chunks are N*16 bytes apart (leading-dimension offset).
 //   * Activation tiles (128 pixels x K bytes) use the same scheme: [K/16][128][16 bytes].
+//   * Bias columns: right after the data columns of the first two GEMMs' K (after the nine taps;
+//     after the padded hidden channels) every A row carries the eight constants (1, 127, ..., 127), and a
+//     layer whose biases fit has them decomposed over the matching eight weight rows
+//     (bias = w0 * 1 + (w1 + ... + w7) * 127), so that its accumulator already includes the bias.
 //   * K of a 3x3 conv over the coupling input is ordered tap-major with the channel count padded
 //     to 8 (k = tap*cpad + c), so every im2col granule is an aligned 8-byte copy. N of the last
 //     3x3 conv is one row per (tap, out channel) with the channel count padded to 8
@@ -28,6 +32,8 @@ constexpr int kMaxHidden = 512;      // kept hidden channels per layer (padded):
 constexpr int kRingDepth = 3;        // weight K-slices in flight when weights are streamed
 constexpr int kSlotCols = 256;       // TMEM columns per tile slot when two tiles are in flight
 constexpr uint32_t kSpinLimit = 20000u;   // bounded waits: tries of up to 100 us each
+// The eight constant A-operand bytes that multiply a layer's bias rows: 1, then seven times 127.
+constexpr uint32_t kBiasColumnsLo = 0x7F7F7F01u, kBiasColumnsHi = 0x7F7F7F7Fu;
 
 // Per-hidden-channel constants of the fast requantisation path (16 bytes).
 //   y = hi32(acc * m0 + c64) >> sh,  c64 = bias * m0 + 2^(30+s),  sh = s - 1   (needs s >= 1)
@@ -52,12 +58,13 @@ struct CouplingMeta {
   int32_t n3;                    // 9*cbp padded to 16 (per-tap partial outputs of the last conv)
   int32_t lo1, hi1, lo2, hi2;    // effective activation clips (ReLU folded in)
   int32_t mode1, mode2;          // requantisation flavour of the two hidden layers:
+                                 //   3: one shift s >= 1 and the bias folded into the GEMM (m0 table)
                                  //   2: one shift s >= 1 for the whole layer ({m0, bias} table)
                                  //   1: per-channel shifts, all >= 1 (HiddenRq table, high-word path)
                                  //   0: any shift (HiddenRq table, full 64-bit shift)
-  int32_t us1, us2;              // the uniform shift (mode 2)
+  int32_t us1, us2;              // the uniform shift (modes 2 and 3)
   int32_t off_colA, off_colB, off_out, off_h1, off_h2;   // byte offsets from the meta start
-  int32_t off_u1, off_u2;        // {m0, bias} tables (int2 per channel)
+  int32_t off_u1, off_u2;        // {m0, bias} tables (int2 per channel; mode 3: int32 m0 per channel)
   int32_t pad[9];
 };
 static_assert(sizeof(CouplingMeta) == 128, "meta header is 128 bytes");

@@ -152,6 +152,7 @@ __device__ __forceinline__ int tap_offset(int tap, int w) {
 }
 
 // A[row][tap*cpad + c] = xa[p + tap offset][c] (0 outside the image), as aligned 8-byte granules,
+// followed by the granule of bias columns (where K has room for it),
 // written in 16-byte chunks into the MMA operand layout [K/16][128][16].
 __device__ void build_im2col(const Ctx& cx, uint8_t* __restrict__ sA, const int8_t* __restrict__ xa, int cpad, int w,
                              int kd, uint32_t recip_gpt, const RowPos rp) {
@@ -169,6 +170,8 @@ __device__ void build_im2col(const Ctx& cx, uint8_t* __restrict__ sA, const int8
         const int tap = (int)(((uint32_t)g * recip_gpt) >> 16), i = g - tap * gpt;
         if ((rp.gmask >> tap) & 1u)
           g2[half] = *reinterpret_cast<const uint2*>(base + tap_offset(tap, w) * cpad + 8 * i);
+      } else if (g == ngran) {
+        g2[half] = make_uint2(kBiasColumnsLo, kBiasColumnsHi);      // the bias columns
       }
     }
     *reinterpret_cast<uint4*>(sA + (size_t)jc * (kTileM * 16) + cx.row * 16) =
@@ -177,15 +180,18 @@ __device__ void build_im2col(const Ctx& cx, uint8_t* __restrict__ sA, const int8
 }
 
 // Requantisation flavours of a hidden layer (chosen per layer when the model is packed):
+//   kModeFolded   the same shift s >= 1 for every channel and the bias already in the accumulator
+//                 (bias rows of the GEMM): constant m0 per channel, y = hi32(acc * m0 + 2^(30+s)) >> (s-1)
 //   kModeUniform  every channel has the same shift s >= 1: constants {m0, bias} per channel,
 //                 y = hi32((acc + bias) * m0 + 2^(30+s)) >> (s-1)
 //   kModeFast     per-channel shifts, all s >= 1: y = hi32(acc * m0 + c64) >> (s-1)
 //   kModeExact    any s: y = (acc * m0 + c64) >> (31 + s) in 64 bits
 // All three are exact: for s >= 1, floor(x / 2^(31+s)) = floor(floor(x / 2^32) / 2^(s-1)).
-constexpr int kModeUniform = 2, kModeFast = 1, kModeExact = 0;
+constexpr int kModeFolded = 3, kModeUniform = 2, kModeFast = 1, kModeExact = 0;
 
-// Clip flavours: kClipS8Relu is the common ReLU + clip to [0, 127]: max(y, 0) followed by the
-// saturating 32->8 bit pack (which clips at 127); kClipAny is max/min with the layer's bounds.
+// Clip flavours: kClipS8Relu is the common ReLU + clip to [0, 127]: the saturating 32->8 bit pack
+// clips to [-128, 127] and the negative bytes are then cleared; kClipAny is max/min with the
+// layer's bounds.
 constexpr int kClipS8Relu = 1, kClipAny = 0;
 
 // d = {sat8(y3), sat8(y2), sat8(y1), sat8(y0)} (y0 in the lowest byte)
@@ -194,6 +200,14 @@ __device__ __forceinline__ uint32_t pack4_sat(int y0, int y1, int y2, int y3) {
   asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(y3), "r"(y2), "r"(0));
   asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(y1), "r"(y0), "r"(t));
   return w;
+}
+// clip(y, 0, 127) of four values: saturate to int8 while packing, then clear the negative bytes
+// (a byte permute with sign replication builds the mask): two instructions for the four ReLUs.
+__device__ __forceinline__ uint32_t pack4_relu_sat(int y0, int y1, int y2, int y3) {
+  const uint32_t w = pack4_sat(y0, y1, y2, y3);
+  uint32_t neg;          // every byte replaced by eight copies of its sign bit
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(neg) : "r"(w), "r"(0u), "r"(0xBA98u));
+  return w & ~neg;
 }
 
 template <int kMode, int kClip>
@@ -216,12 +230,22 @@ struct Requant {
       if (kMode == kModeFast) y = ((int)(p >> 32)) >> r.sh;
       else y = (int)(p >> (32 + r.sh));
     }
-    return kClip == kClipS8Relu ? max(y, 0) : clampi(y, lo, hi);
+    return kClip == kClipS8Relu ? y : clampi(y, lo, hi);     // kClipS8Relu: clipped while packing
   }
   // 16 accumulator columns starting at channel ch0 -> one 16-byte chunk of the next A operand
   __device__ __forceinline__ uint4 chunk(const uint32_t* r, int ch0) const {
     uint32_t wd[4];
-    if (kMode == kModeUniform) {
+    if (kMode == kModeFolded) {
+      // multipliers of four channels per 16-byte shared-memory load
+      const int4* q = reinterpret_cast<const int4*>(reinterpret_cast<const int32_t*>(mb) + ch0);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int4 c = q[i];
+        const int y0 = uniform_one((int)r[4 * i], c.x, 0), y1 = uniform_one((int)r[4 * i + 1], c.y, 0);
+        const int y2 = uniform_one((int)r[4 * i + 2], c.z, 0), y3 = uniform_one((int)r[4 * i + 3], c.w, 0);
+        wd[i] = kClip == kClipS8Relu ? pack4_relu_sat(y0, y1, y2, y3) : pack4(y0, y1, y2, y3);
+      }
+    } else if (kMode == kModeUniform) {
       // {m0, bias} pairs of two channels per 16-byte shared-memory load (the table is 16-byte aligned)
       const int4* q = reinterpret_cast<const int4*>(mb + ch0);
 #pragma unroll
@@ -229,14 +253,14 @@ struct Requant {
         const int4 c01 = q[2 * i], c23 = q[2 * i + 1];
         const int y0 = uniform_one((int)r[4 * i], c01.x, c01.y), y1 = uniform_one((int)r[4 * i + 1], c01.z, c01.w);
         const int y2 = uniform_one((int)r[4 * i + 2], c23.x, c23.y), y3 = uniform_one((int)r[4 * i + 3], c23.z, c23.w);
-        wd[i] = kClip == kClipS8Relu ? pack4_sat(y0, y1, y2, y3) : pack4(y0, y1, y2, y3);
+        wd[i] = kClip == kClipS8Relu ? pack4_relu_sat(y0, y1, y2, y3) : pack4(y0, y1, y2, y3);
       }
     } else {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int y0 = one((int)r[4 * i], ch0 + 4 * i), y1 = one((int)r[4 * i + 1], ch0 + 4 * i + 1);
         const int y2 = one((int)r[4 * i + 2], ch0 + 4 * i + 2), y3 = one((int)r[4 * i + 3], ch0 + 4 * i + 3);
-        wd[i] = kClip == kClipS8Relu ? pack4_sat(y0, y1, y2, y3) : pack4(y0, y1, y2, y3);
+        wd[i] = kClip == kClipS8Relu ? pack4_relu_sat(y0, y1, y2, y3) : pack4(y0, y1, y2, y3);
       }
     }
     return make_uint4(wd[0], wd[1], wd[2], wd[3]);
@@ -244,7 +268,7 @@ struct Requant {
   __device__ __forceinline__ int uniform_one(int acc, int m0, int bias) const {
     const long long p = (long long)(acc + bias) * (long long)m0 + rnd64;
     const int y = ((int)(p >> 32)) >> sh;
-    return kClip == kClipS8Relu ? max(y, 0) : clampi(y, lo, hi);
+    return kClip == kClipS8Relu ? y : clampi(y, lo, hi);
   }
 };
 
@@ -254,11 +278,14 @@ struct Requant {
 // splits so that they differ by at most one chunk; a warp takes its chunks two at a time.
 template <int kMode, int kClip>
 __device__ __forceinline__ void epilogue_hidden_t(const Ctx& cx, int n, int kd, const Requant<kMode, kClip> q,
-                                                  uint8_t* __restrict__ sOut) {
+                                                  uint32_t pad_lo, uint32_t pad_hi, uint8_t* __restrict__ sOut) {
   const int nch = n >> 4;
   uint8_t* out = sOut + cx.row * 16;
-  if (kd > n && (nch % cx.ncs) == cx.cs)
-    *reinterpret_cast<uint4*>(out + (size_t)nch * (kTileM * 16)) = make_uint4(0u, 0u, 0u, 0u);
+  // chunks past the data: the first one starts with the bias columns of the next GEMM (pad_lo,
+  // pad_hi; zero if it has none), the others are zero
+  for (int j = nch + ((cx.cs - nch) & (cx.ncs - 1)); j < (kd >> 4); j += cx.ncs)
+    *reinterpret_cast<uint4*>(out + (size_t)j * (kTileM * 16)) =
+        j == nch ? make_uint4(pad_lo, pad_hi, 0u, 0u) : make_uint4(0u, 0u, 0u, 0u);
   int ch = cx.cs;
   for (; ch + cx.ncs < nch; ch += 2 * cx.ncs) {
     const int ch2 = ch + cx.ncs;
@@ -280,16 +307,22 @@ __device__ __forceinline__ void epilogue_hidden_t(const Ctx& cx, int n, int kd, 
 
 // mode: layer flavour (see above); us: the layer's uniform shift (kModeUniform only).
 __device__ __forceinline__ void epilogue_hidden(const Ctx& cx, int mode, int us, int n, int kd, const HiddenRq* rq,
-                                                const int2* mb, int lo, int hi, uint8_t* sOut) {
+                                                const int2* mb, int lo, int hi, uint32_t pad_lo, uint32_t pad_hi,
+                                                uint8_t* sOut) {
   const bool s8relu = lo == 0 && hi == 127;
-  if (mode == kModeUniform) {
+  if (mode >= kModeUniform) {
     const long long rnd64 = 1ll << (30 + us);
-    if (s8relu) epilogue_hidden_t(cx, n, kd, Requant<kModeUniform, kClipS8Relu>{rq, mb, lo, hi, us - 1, rnd64}, sOut);
-    else epilogue_hidden_t(cx, n, kd, Requant<kModeUniform, kClipAny>{rq, mb, lo, hi, us - 1, rnd64}, sOut);
+    if (mode == kModeFolded) {
+      if (s8relu) epilogue_hidden_t(cx, n, kd, Requant<kModeFolded, kClipS8Relu>{rq, mb, lo, hi, us - 1, rnd64}, pad_lo, pad_hi, sOut);
+      else epilogue_hidden_t(cx, n, kd, Requant<kModeFolded, kClipAny>{rq, mb, lo, hi, us - 1, rnd64}, pad_lo, pad_hi, sOut);
+    } else {
+      if (s8relu) epilogue_hidden_t(cx, n, kd, Requant<kModeUniform, kClipS8Relu>{rq, mb, lo, hi, us - 1, rnd64}, pad_lo, pad_hi, sOut);
+      else epilogue_hidden_t(cx, n, kd, Requant<kModeUniform, kClipAny>{rq, mb, lo, hi, us - 1, rnd64}, pad_lo, pad_hi, sOut);
+    }
   } else if (mode == kModeFast) {
-    epilogue_hidden_t(cx, n, kd, Requant<kModeFast, kClipAny>{rq, mb, lo, hi, 0, 0}, sOut);
+    epilogue_hidden_t(cx, n, kd, Requant<kModeFast, kClipAny>{rq, mb, lo, hi, 0, 0}, pad_lo, pad_hi, sOut);
   } else {
-    epilogue_hidden_t(cx, n, kd, Requant<kModeExact, kClipAny>{rq, mb, lo, hi, 0, 0}, sOut);
+    epilogue_hidden_t(cx, n, kd, Requant<kModeExact, kClipAny>{rq, mb, lo, hi, 0, 0}, pad_lo, pad_hi, sOut);
   }
 }
 
@@ -875,13 +908,13 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
         for (int sl = 0; sl < nt; ++sl) {                     // requant, conv 1x1
           wait_d(sl);
           use_slot(sl);
-          epilogue_hidden(cx, M.mode1, M.us1, M.n1, M.kd2, h1, u1, M.lo1, M.hi1, sA);
+          epilogue_hidden(cx, M.mode1, M.us1, M.n1, M.kd2, h1, u1, M.lo1, M.hi1, kBiasColumnsLo, kBiasColumnsHi, sA);
           arrive_a(sl);
         }
         for (int sl = 0; sl < nt; ++sl) {                     // requant, conv 3x3 as per-tap partials
           wait_d(sl);
           use_slot(sl);
-          epilogue_hidden(cx, M.mode2, M.us2, M.n2, M.kd3, h2, u2, M.lo2, M.hi2, sA);
+          epilogue_hidden(cx, M.mode2, M.us2, M.n2, M.kd3, h2, u2, M.lo2, M.hi2, 0u, 0u, sA);
           arrive_a(sl);
         }
         for (int sl = 0; sl < nt; ++sl) {                     // shifted sum into the accumulator

@@ -95,6 +95,34 @@ def test_zero_shift_layers_take_the_exact_path(G):
     _check_both_ways(G, model, x)
 
 
+def test_biases_around_the_folding_limit(G):
+    """The library folds a hidden layer's biases into spare rows of its GEMM while every |bias| is at
+    most 63 + 7 * 127 * 127 = 112966 and adds them in the epilogue otherwise; both routes, the exact
+    limit on either side, and layers that mix small and extreme biases must agree with the oracle.
+    (Per-channel shifts that differ within a layer take yet another route.)"""
+    limit = 63 + 7 * 127 * 127
+    model = S.make_model(23, 3, 16, 16, [True, True], 4, 48, prune=(0.5, 0.8))
+    edge = [limit, -limit, limit - 1, 1 - limit, 127 * 127, -127 * 127, 64, -64, 63, -63, 0]
+    for lv in model["levels"]:
+        for ci, cp in enumerate(lv["couplings"]):
+            for li in range(2):
+                ly = cp["layers"][li]
+                n = len(ly["bias"])
+                if ci == 0:      # all foldable, every edge value present
+                    ly["bias"][:len(edge)] = edge[:n]
+                elif ci == 1:    # one channel just past the limit: the whole layer adds in the epilogue
+                    ly["bias"][:len(edge)] = edge[:n]
+                    ly["bias"][n // 2] = limit + 1 if li == 0 else -(limit + 1)
+                elif ci == 2:    # large biases
+                    ly["bias"][::3] = 1 << 20
+                    ly["bias"][1::3] = -(1 << 20)
+                else:            # foldable biases, but shifts differ inside the layer
+                    ly["bias"][:len(edge)] = edge[:n]
+                    ly["s"][::2] += 1
+    x = S.smooth_field_images(24, 6, 16, 16, 1.5)
+    _check_both_ways(G, model, x)
+
+
 def test_zero_bias_and_no_prior(G):
     model = S.make_model(19, 3, 16, 16, [True, False], 2, 16, prune=None, prior=False, with_bias=False)
     _check_both_ways(G, model, S.smooth_field_images(20, 4, 16, 16, 1.5))
