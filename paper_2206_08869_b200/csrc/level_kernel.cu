@@ -815,49 +815,53 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
     ptx::tc_fence_after();
   };
 
-  // x_b +/-= rq(acc + bias) of the previous coupling. Work item = (pixel, group of four output
-  // channels), so that levels with few pixels per CTA still use every thread.
+  // n / pvalid for the work-item maps below (n * pvalid < 2^32)
+  const uint32_t mul_pv = pvalid > 1 ? (uint32_t)((0xFFFFFFFFull / (uint32_t)pvalid) + 1ull) : 0u;
+  // x_b +/-= rq(acc + bias) of the previous coupling. Work item = (channel, pixel), channel-major, so
+  // that levels with few pixels per CTA still use every thread and the load is even; two items at
+  // a time for independent instruction chains.
   auto apply_translation_all = [&]() {
     const uint8_t* pm = reinterpret_cast<const uint8_t*>(prevM);
     const int32_t* colB = reinterpret_cast<const int32_t*>(pm + prevM->off_colB);
     const OutRq* orq = reinterpret_cast<const OutRq*>(pm + prevM->off_out);
-    const int items = ((cb + 3) >> 2) * pvalid;
-    for (int it = cx.tid; it < items; it += kWorkers) {
-      const int cg = it / pvalid, p = it - cg * pvalid;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int c = cg * 4 + k;
-        if (c < cb) {
-          const OutRq o = orq[c];
-          const uint32_t t = (uint32_t)rq_exact(acc[c * pg + p] + o.bias, o.m0, o.s);
-          acc[c * pg + p] = 0;
-          uint32_t* vv = reinterpret_cast<uint32_t*>(&v[colB[c] * pg + p]);
-          *vv = kInv ? (*vv - t) : (*vv + t);
-        }
-      }
+    const int items = cb * pvalid;
+    auto one = [&](int it) {
+      const int c = fdiv(it, mul_pv), p = it - c * pvalid;
+      const OutRq o = orq[c];
+      int32_t* ap = acc + c * pg + p;
+      const uint32_t t = (uint32_t)rq_exact(*ap + o.bias, o.m0, o.s);
+      *ap = 0;
+      uint32_t* vv = reinterpret_cast<uint32_t*>(&v[colB[c] * pg + p]);
+      *vv = kInv ? (*vv - t) : (*vv + t);
+    };
+    int it = cx.tid;
+    for (; it + kWorkers < items; it += 2 * kWorkers) {
+      one(it);
+      one(it + kWorkers);
     }
+    if (it < items) one(it);
   };
   // network input: ca channels requantised to int8, padded to cpad bytes per pixel. Work item =
-  // (pixel, granule of eight channels).
+  // (group of four channels, pixel).
   auto requant_input_all = [&](const int32_t* cols, int32_t m0, int32_t s) {
-    const int items = (cpad >> 3) * pvalid;
+    const int items = (cpad >> 2) * pvalid;
     for (int it = cx.tid; it < items; it += kWorkers) {
-      const int g = it / pvalid, p = it - g * pvalid;
-      const int g0 = g << 3;
-      int y[8];
+      const int g = fdiv(it, mul_pv), p = it - g * pvalid;
+      const int g0 = g << 2;
+      int y[4];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < 4; ++i) {
         y[i] = 0;
         if (g0 + i < ca) y[i] = clampi(rq_exact(v[cols[g0 + i] * pg + p], m0, s), -128, 127);
       }
-      *reinterpret_cast<uint2*>(xa + (size_t)p * cpad + g0) =
-          make_uint2(pack4(y[0], y[1], y[2], y[3]), pack4(y[4], y[5], y[6], y[7]));
+      *reinterpret_cast<uint32_t*>(xa + (size_t)p * cpad + g0) = pack4(y[0], y[1], y[2], y[3]);
     }
   };
   auto worker_barrier = [&]() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); };
 
   for (int i = 0; i < st.nsteps; ++i) {
-    wait_bar(ctl, a.status, &ctl->meta_full[i & 1], (uint32_t)((i >> 1) & 1));
+    if (!ptx::mbar_test_wait(ptx::smem_u32(&ctl->meta_full[i & 1]), (uint32_t)((i >> 1) & 1)))
+      wait_bar(ctl, a.status, &ctl->meta_full[i & 1], (uint32_t)((i >> 1) & 1));
     const uint8_t* mb = smem + P.s_meta[i & 1];
     const bool prior = st.is_prior(i);
     const CouplingMeta* Mp = reinterpret_cast<const CouplingMeta*>(mb);
