@@ -343,6 +343,7 @@ bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32
       P.group = group;
       P.pg = (int)pg;
       P.tiles = tiles;
+      P.rep = tiles == 1 ? (group * P.px <= kTileM / 4 ? 4 : (group * P.px <= kTileM / 2 ? 2 : 1)) : 1;
       if (off <= limit) return true;
     }
     if (group == 1) break;

@@ -97,6 +97,10 @@ struct LevelPlan {
   int32_t n_couplings;
   int32_t split, has_prior, is_first, is_last;
   int32_t keep_c;                // channels that go on to the next level (c/2 if split else c)
+  int32_t rep;                   // row replication, 1, 2 or 4: a CTA whose pixels fill at most 128/rep rows of
+                                 // its single tile puts them in the tile rep times (rows r, r + 128/rep, ...),
+                                 // so that every TMEM lane quarter holds a copy and the epilogues split the
+                                 // accumulator columns over all 16 worker warps instead of 4 * (4 / rep)
   int32_t nslots;                // tiles in flight per CTA: 1 or 2
   int32_t tmem_cols;
   int32_t w13_alias;             // 1: W1 and W3 share a slot and are re-fetched per tile

@@ -57,8 +57,10 @@ struct Ctx {
   uint32_t* status;
   int tid, warp, lane;
   int wq;                 // TMEM lane quarter of this warp
-  int cs, ncs;            // column-split index and count
+  int cs, ncs;            // column-split index and count of the epilogues (all replicas together)
+  int bcs, bncs;          // column-split index and count of the im2col build (within one lane quarter)
   int row;                // tile row (= TMEM lane) of this thread
+  int rep, rrows;         // row replication (see LevelPlan::rep) and rows per replica (128 / rep)
   uint32_t tmem_base;     // first allocated TMEM column, lane field 0
   uint32_t tmem_slot;     // current tile slot's first column, this warp's lane quarter
 };
@@ -136,10 +138,11 @@ __device__ __forceinline__ uint32_t row_record(int p, int pvalid, int px, int h,
   return r;
 }
 
-__device__ __forceinline__ RowPos row_pos(const uint32_t* rowinfo, int tile, int row) {
+// row: the thread's tile row; prow: its row within the replica (the same unless rows are replicated)
+__device__ __forceinline__ RowPos row_pos(const uint32_t* rowinfo, int tile, int row, int prow) {
   RowPos r;
-  r.p = tile * kTileM + row;
-  const uint32_t rec = rowinfo[r.p];
+  r.p = tile * kTileM + prow;
+  const uint32_t rec = rowinfo[tile * kTileM + row];
   r.valid = (rec & 1u) != 0;
   r.gmask = (rec >> 1) & 0x1FFu;
   r.smask = (rec >> 10) & 0x1FFu;
@@ -160,7 +163,7 @@ __device__ void build_im2col(const Ctx& cx, uint8_t* __restrict__ sA, const int8
   const int gpt = cpad >> 3;                // granules per tap
   const int ngran = 9 * gpt;
   const int8_t* base = xa + (size_t)rp.p * cpad;
-  for (int jc = cx.cs; jc < nchunks; jc += cx.ncs) {
+  for (int jc = cx.bcs; jc < nchunks; jc += cx.bncs) {
     uint2 g2[2];
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
@@ -280,12 +283,21 @@ template <int kMode, int kClip>
 __device__ __forceinline__ void epilogue_hidden_t(const Ctx& cx, int n, int kd, const Requant<kMode, kClip> q,
                                                   uint32_t pad_lo, uint32_t pad_hi, uint8_t* __restrict__ sOut) {
   const int nch = n >> 4;
+  // A chunk goes to this thread's row in every replica of the tile (one replica: the row itself).
   uint8_t* out = sOut + cx.row * 16;
+  const bool replicated = cx.rep > 1;
+  auto put = [&](int chunk, const uint4 val) {
+    *reinterpret_cast<uint4*>(out + (size_t)chunk * (kTileM * 16)) = val;
+    if (replicated) {
+      uint8_t* base = sOut + (size_t)chunk * (kTileM * 16);
+      for (int k = 1; k < cx.rep; ++k)
+        *reinterpret_cast<uint4*>(base + ((cx.row + k * cx.rrows) & (kTileM - 1)) * 16) = val;
+    }
+  };
   // chunks past the data: the first one starts with the bias columns of the next GEMM (pad_lo,
   // pad_hi; zero if it has none), the others are zero
   for (int j = nch + ((cx.cs - nch) & (cx.ncs - 1)); j < (kd >> 4); j += cx.ncs)
-    *reinterpret_cast<uint4*>(out + (size_t)j * (kTileM * 16)) =
-        j == nch ? make_uint4(pad_lo, pad_hi, 0u, 0u) : make_uint4(0u, 0u, 0u, 0u);
+    put(j, j == nch ? make_uint4(pad_lo, pad_hi, 0u, 0u) : make_uint4(0u, 0u, 0u, 0u));
   int ch = cx.cs;
   for (; ch + cx.ncs < nch; ch += 2 * cx.ncs) {
     const int ch2 = ch + cx.ncs;
@@ -294,14 +306,14 @@ __device__ __forceinline__ void epilogue_hidden_t(const Ctx& cx, int n, int kd, 
     ptx::tmem_ld16(cx.tmem_slot + (uint32_t)(ch2 << 4), rb);
     ptx::tmem_ld_wait16(ra);
     ptx::tmem_ld_wait16(rb);
-    *reinterpret_cast<uint4*>(out + (size_t)ch * (kTileM * 16)) = q.chunk(ra, ch << 4);
-    *reinterpret_cast<uint4*>(out + (size_t)ch2 * (kTileM * 16)) = q.chunk(rb, ch2 << 4);
+    put(ch, q.chunk(ra, ch << 4));
+    put(ch2, q.chunk(rb, ch2 << 4));
   }
   if (ch < nch) {
     uint32_t ra[16];
     ptx::tmem_ld16(cx.tmem_slot + (uint32_t)(ch << 4), ra);
     ptx::tmem_ld_wait16(ra);
-    *reinterpret_cast<uint4*>(out + (size_t)ch * (kTileM * 16)) = q.chunk(ra, ch << 4);
+    put(ch, q.chunk(ra, ch << 4));
   }
 }
 
@@ -885,7 +897,7 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
         const int nt = min(nslots, ntv - t0);
         for (int sl = 0; sl < nt; ++sl) {
           use_slot(sl);
-          rp[sl] = row_pos(rowinfo, t0 + sl, cx.row);
+          rp[sl] = row_pos(rowinfo, t0 + sl, cx.row, cx.row & (cx.rrows - 1));
           build_im2col(cx, sA, xa, cpad, w, M.kd, recip_a, rp[sl]);
           arrive_a(sl);
         }
@@ -905,7 +917,7 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
         const int nt = min(nslots, ntv - t0);
         for (int sl = 0; sl < nt; ++sl) {                     // conv 3x3: input -> hidden 1
           use_slot(sl);
-          rp[sl] = row_pos(rowinfo, t0 + sl, cx.row);
+          rp[sl] = row_pos(rowinfo, t0 + sl, cx.row, cx.row & (cx.rrows - 1));
           build_im2col(cx, sA, xa, cpad, w, M.kd1, recip_a, rp[sl]);
           arrive_a(sl);
         }
@@ -986,8 +998,12 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
   cx.warp = warp;
   cx.lane = lane;
   cx.wq = warp & 3;
-  cx.cs = warp >> 2;
-  cx.ncs = kWorkerWarps >> 2;
+  cx.rep = P.rep;
+  cx.rrows = kTileM / P.rep;
+  cx.bcs = warp >> 2;
+  cx.bncs = kWorkerWarps >> 2;
+  cx.cs = ((cx.wq * P.rep) >> 2) * cx.bncs + cx.bcs;     // replica index * 4 + split within the quarter
+  cx.ncs = cx.bncs * P.rep;
   cx.row = cx.wq * 32 + lane;
   cx.tmem_base = tmem;
   cx.tmem_slot = tmem + ((uint32_t)(cx.wq * 32) << 16);
@@ -1005,7 +1021,7 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
     int32_t* acc = reinterpret_cast<int32_t*>(smem + P.s_acc);
     for (int idx = tid; idx < P.cb * pg; idx += kWorkers) acc[idx] = 0;
     uint32_t* rowinfo = reinterpret_cast<uint32_t*>(smem + P.s_rowinfo);
-    for (int idx = tid; idx < P.tiles * kTileM; idx += kWorkers) rowinfo[idx] = row_record(idx, pvalid, px, P.h, w, P.mul_px, P.mul_w);
+    for (int idx = tid; idx < P.tiles * kTileM; idx += kWorkers) rowinfo[idx] = row_record(P.rep > 1 ? (idx & (kTileM / P.rep - 1)) : idx, pvalid, px, P.h, w, P.mul_px, P.mul_w);
     // Everything above used only the plan; from here on the kernel reads what the previous kernel
     // in the stream wrote and writes what it may still be reading.
     ptx::grid_dependency_wait();
