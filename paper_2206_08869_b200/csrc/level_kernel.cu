@@ -155,31 +155,60 @@ __device__ __forceinline__ int tap_offset(int tap, int w) {
 }
 
 // A[row][tap*cpad + c] = xa[p + tap offset][c] (0 outside the image), as aligned 8-byte granules,
-// followed by the granule of bias columns (where K has room for it),
-// written in 16-byte chunks into the MMA operand layout [K/16][128][16].
-__device__ void build_im2col(const Ctx& cx, uint8_t* __restrict__ sA, const int8_t* __restrict__ xa, int cpad, int w,
-                             int kd, uint32_t recip_gpt, const RowPos rp) {
+// followed by the granule of bias columns (where K has room for it), written in 16-byte chunks into
+// the MMA operand layout [K/16][128][16]. kPairs: cpad is a multiple of 16, so the two granules of a
+// chunk belong to one tap and come with one 16-byte load.
+template <bool kPairs>
+__device__ __forceinline__ uint4 im2col_chunk(const int8_t* __restrict__ base, int jc, int cpad, int w, int gpt, int ngran,
+                                              uint32_t recip_gpt, uint32_t gmask) {
+  if (kPairs) {
+    const int g = 2 * jc;
+    if (g < ngran) {
+      const int tap = (int)(((uint32_t)g * recip_gpt) >> 16), i = g - tap * gpt;
+      if ((gmask >> tap) & 1u) return *reinterpret_cast<const uint4*>(base + tap_offset(tap, w) * cpad + 8 * i);
+      return make_uint4(0u, 0u, 0u, 0u);
+    }
+    return g == ngran ? make_uint4(kBiasColumnsLo, kBiasColumnsHi, 0u, 0u) : make_uint4(0u, 0u, 0u, 0u);
+  }
+  uint2 g2[2];
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    const int g = 2 * jc + half;
+    g2[half] = make_uint2(0u, 0u);
+    if (g < ngran) {
+      const int tap = (int)(((uint32_t)g * recip_gpt) >> 16), i = g - tap * gpt;
+      if ((gmask >> tap) & 1u) g2[half] = *reinterpret_cast<const uint2*>(base + tap_offset(tap, w) * cpad + 8 * i);
+    } else if (g == ngran) {
+      g2[half] = make_uint2(kBiasColumnsLo, kBiasColumnsHi);      // the bias columns
+    }
+  }
+  return make_uint4(g2[0].x, g2[0].y, g2[1].x, g2[1].y);
+}
+
+template <bool kPairs>
+__device__ __forceinline__ void build_im2col_t(const Ctx& cx, uint8_t* __restrict__ sA, const int8_t* __restrict__ xa, int cpad,
+                                               int w, int kd, uint32_t recip_gpt, const RowPos rp) {
   const int nchunks = kd >> 4;
   const int gpt = cpad >> 3;                // granules per tap
   const int ngran = 9 * gpt;
   const int8_t* base = xa + (size_t)rp.p * cpad;
-  for (int jc = cx.bcs; jc < nchunks; jc += cx.bncs) {
-    uint2 g2[2];
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      const int g = 2 * jc + half;
-      g2[half] = make_uint2(0u, 0u);
-      if (g < ngran) {
-        const int tap = (int)(((uint32_t)g * recip_gpt) >> 16), i = g - tap * gpt;
-        if ((rp.gmask >> tap) & 1u)
-          g2[half] = *reinterpret_cast<const uint2*>(base + tap_offset(tap, w) * cpad + 8 * i);
-      } else if (g == ngran) {
-        g2[half] = make_uint2(kBiasColumnsLo, kBiasColumnsHi);      // the bias columns
-      }
-    }
-    *reinterpret_cast<uint4*>(sA + (size_t)jc * (kTileM * 16) + cx.row * 16) =
-        make_uint4(g2[0].x, g2[0].y, g2[1].x, g2[1].y);
+  uint8_t* out = sA + cx.row * 16;
+  int jc = cx.bcs;
+  for (; jc + cx.bncs < nchunks; jc += 2 * cx.bncs) {          // two chunks at a time: independent loads
+    const uint4 c0 = im2col_chunk<kPairs>(base, jc, cpad, w, gpt, ngran, recip_gpt, rp.gmask);
+    const uint4 c1 = im2col_chunk<kPairs>(base, jc + cx.bncs, cpad, w, gpt, ngran, recip_gpt, rp.gmask);
+    *reinterpret_cast<uint4*>(out + (size_t)jc * (kTileM * 16)) = c0;
+    *reinterpret_cast<uint4*>(out + (size_t)(jc + cx.bncs) * (kTileM * 16)) = c1;
   }
+  if (jc < nchunks)
+    *reinterpret_cast<uint4*>(out + (size_t)jc * (kTileM * 16)) =
+        im2col_chunk<kPairs>(base, jc, cpad, w, gpt, ngran, recip_gpt, rp.gmask);
+}
+
+__device__ void build_im2col(const Ctx& cx, uint8_t* __restrict__ sA, const int8_t* __restrict__ xa, int cpad, int w,
+                             int kd, uint32_t recip_gpt, const RowPos rp) {
+  if ((cpad & 15) == 0) build_im2col_t<true>(cx, sA, xa, cpad, w, kd, recip_gpt, rp);
+  else build_im2col_t<false>(cx, sA, xa, cpad, w, kd, recip_gpt, rp);
 }
 
 // Requantisation flavours of a hidden layer (chosen per layer when the model is packed):
