@@ -158,7 +158,11 @@ void put_out_rq(OutRq* dst, const iodf_layer_desc& L, const Blobs& B) {
   const int32_t* bias = B.r + L.requant_off;
   const int32_t* m0 = bias + L.c_out;
   const int32_t* s = m0 + L.c_out;
-  for (uint32_t i = 0; i < L.c_out; ++i) dst[i] = OutRq{bias[i], m0[i], s[i], 0};
+  for (uint32_t i = 0; i < L.c_out; ++i) {
+    const long long c64 = (long long)bias[i] * (long long)m0[i] + (1ll << (30 + s[i]));
+    dst[i] = OutRq{m0[i], s[i], (uint32_t)((unsigned long long)c64 & 0xFFFFFFFFull),
+                   (uint32_t)((unsigned long long)c64 >> 32)};
+  }
 }
 
 // Weight matrix [n_pad rows][kd bytes], K-major, no swizzle: byte (n, k) at (k/16)*n_pad*16 + n*16 + k%16.
@@ -322,6 +326,7 @@ bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32
       P.s_xa = take(pg * (uint32_t)P.cpad);
       P.s_acc = take((uint32_t)P.cb * pg * 4);
       P.s_rowinfo = take((uint32_t)tiles * kTileM * 4);
+      P.s_gran = take((uint32_t)P.n_gran * 8);
       P.s_a[0] = take(a_bytes);
       P.s_a[1] = mode == 0 ? take(a_bytes) : P.s_a[0];
       P.s_meta[0] = take(meta_bytes);
@@ -507,6 +512,21 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
       n_max = std::max<uint32_t>(n_max, n);
     }
     if (n_max > 512) return IODF_EUNSUPPORTED;
+    {   // im2col granule table of the level's first convs (couplings and prior head share it)
+      const int gpt = P.cpad / 8, ndata = 9 * gpt;
+      P.n_gran = (int)up((uint32_t)(ndata + 1), 4);
+      if (P.n_gran > kMaxGran) return IODF_EUNSUPPORTED;
+      for (int g = 0; g < P.n_gran; ++g) {
+        int off = 0, sel = g == ndata ? kGranBias : kGranPad;
+        if (g < ndata) {
+          const int tap = g / gpt, i = g % gpt, u = tap / 3, v = tap % 3;
+          off = ((u - 1) * (int)w + (v - 1)) * P.cpad + 8 * i;
+          sel = tap;
+        }
+        P.gran_tab[2 * g] = off;
+        P.gran_tab[2 * g + 1] = sel;
+      }
+    }
     for (uint32_t ki = 0; ki < lv.n_couplings; ++ki) {
       append_block(hl.blob, blocks[ki], &P.coupling[ki]);
       meta = std::max(meta, P.coupling[ki].meta_bytes);

@@ -33,6 +33,9 @@ constexpr int kRingDepth = 3;        // weight K-slices in flight when weights a
 constexpr int kSlotCols = 256;       // TMEM columns per tile slot when two tiles are in flight
 constexpr uint32_t kSpinLimit = 20000u;   // bounded waits: tries of up to 100 us each
 // The eight constant A-operand bytes that multiply a layer's bias rows: 1, then seven times 127.
+// im2col granule table: validity selectors beyond the nine taps' gather-mask bits
+constexpr int kGranBias = 9, kGranPad = 10;
+constexpr int kMaxGran = 152;        // 8-byte granules of the widest first-conv K: (9 * 128 + 8) / 8, rounded up to 32 bytes
 constexpr uint32_t kBiasColumnsLo = 0x7F7F7F01u, kBiasColumnsHi = 0x7F7F7F7Fu;
 
 // Per-hidden-channel constants of the fast requantisation path (16 bytes).
@@ -43,9 +46,12 @@ struct HiddenRq {
   uint32_t c_lo, c_hi;
 };
 
-// Per-output-channel constants of the exact path (translation and prior outputs).
+// Per-output-channel constants of the translation and prior outputs (any shift 0..31):
+//   y = (acc * m0 + c64) >> (31 + s),  c64 = bias * m0 + 2^(30+s)
 struct OutRq {
-  int32_t bias, m0, s, pad;
+  int32_t m0;
+  int32_t s;
+  uint32_t c_lo, c_hi;
 };
 
 // Meta part of a coupling block, followed in memory by
@@ -108,13 +114,17 @@ struct LevelPlan {
                                  //    kRingDepth slots at s_w[0] (hidden widths above 256, one tile in flight)
   uint32_t ring_slot_bytes;
   // shared-memory byte offsets
-  uint32_t s_v, s_xa, s_acc, s_rowinfo, s_a[2], s_meta[2], s_w[3], s_total;
+  uint32_t s_v, s_xa, s_acc, s_rowinfo, s_gran, s_a[2], s_meta[2], s_w[3], s_total;
   // magic multipliers for the index maps: n / d = umulhi(n, ceil(2^32 / d)) for n * d < 2^32 (0: d = 1)
   uint32_t mul_per_img, mul_4px, mul_w2, mul_px, mul_w;
   uint32_t recip_gpa, recip_gpb; // floor(g / (cpad/8)) = (g * recip_gpa) >> 16 for g < 4096; same for cbp/8
   // global layout
   uint64_t z_off, prior_off, z_final_off, d, d_fact;
   int32_t col_out[kMaxC];        // physical column of logical channel k after the last coupling
+  // im2col granule g of the first conv's K (8 bytes): {byte offset of its source relative to the
+  // pixel's xa record, validity selector: tap 0..8 = bit of the row's gather mask, kGranBias, kGranPad}
+  int32_t n_gran;
+  int32_t gran_tab[2 * kMaxGran];
   BlockRef coupling[kMaxCouplings];
   BlockRef prior;
 };

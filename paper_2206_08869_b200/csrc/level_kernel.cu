@@ -100,6 +100,15 @@ __device__ __forceinline__ int32_t rq_exact(int32_t a, int32_t m0, int32_t s) {
   return (int32_t)(p >> 31);
 }
 
+// rq(acc + bias) with the channel's precomputed c64 = bias * m0 + 2^(30+s): one 64-bit multiply-add,
+// then the high word shifted by s - 1 (s >= 1) or the 64-bit value shifted by 31 (s = 0).
+__device__ __forceinline__ int32_t rq_out(int32_t acc, const OutRq o) {
+  const long long c64 = (long long)(((unsigned long long)o.c_hi << 32) | (unsigned long long)o.c_lo);
+  const long long p = (long long)acc * (long long)o.m0 + c64;
+  const int32_t hi = (int32_t)(p >> 32);
+  return o.s >= 1 ? (hi >> (o.s - 1)) : (int32_t)__funnelshift_r((uint32_t)p, (uint32_t)hi, 31);
+}
+
 __device__ __forceinline__ int clampi(int v, int lo, int hi) { return min(max(v, lo), hi); }
 
 // n / d with the plan's magic multiplier ceil(2^32 / d) (0 stands for d = 1); exact while n * d < 2^32
@@ -156,59 +165,52 @@ __device__ __forceinline__ int tap_offset(int tap, int w) {
 
 // A[row][tap*cpad + c] = xa[p + tap offset][c] (0 outside the image), as aligned 8-byte granules,
 // followed by the granule of bias columns (where K has room for it), written in 16-byte chunks into
-// the MMA operand layout [K/16][128][16]. kPairs: cpad is a multiple of 16, so the two granules of a
-// chunk belong to one tap and come with one 16-byte load.
+// the MMA operand layout [K/16][128][16]. Where each granule comes from is a property of the level,
+// not of the pixel: the host tabulates, per granule, the byte offset of its source relative to the
+// pixel's own xa record and the bit of the row's gather mask that validates it (9: the bias
+// granule, 10: padding), so a granule costs one table read, one mask test and one predicated load.
+// kPairs: cpad is a multiple of 16, so the two granules of a chunk belong to one tap and come with
+// one 16-byte load.
 template <bool kPairs>
-__device__ __forceinline__ uint4 im2col_chunk(const int8_t* __restrict__ base, int jc, int cpad, int w, int gpt, int ngran,
-                                              uint32_t recip_gpt, uint32_t gmask) {
+__device__ __forceinline__ uint4 im2col_chunk(const int8_t* __restrict__ base, const int2* __restrict__ tab, int jc,
+                                              uint32_t gmask) {
   if (kPairs) {
-    const int g = 2 * jc;
-    if (g < ngran) {
-      const int tap = (int)(((uint32_t)g * recip_gpt) >> 16), i = g - tap * gpt;
-      if ((gmask >> tap) & 1u) return *reinterpret_cast<const uint4*>(base + tap_offset(tap, w) * cpad + 8 * i);
-      return make_uint4(0u, 0u, 0u, 0u);
-    }
-    return g == ngran ? make_uint4(kBiasColumnsLo, kBiasColumnsHi, 0u, 0u) : make_uint4(0u, 0u, 0u, 0u);
+    const int2 e = tab[2 * jc];
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if ((gmask >> e.y) & 1u) v = *reinterpret_cast<const uint4*>(base + e.x);
+    if (e.y == kGranBias) v = make_uint4(kBiasColumnsLo, kBiasColumnsHi, 0u, 0u);
+    return v;
   }
-  uint2 g2[2];
-#pragma unroll
-  for (int half = 0; half < 2; ++half) {
-    const int g = 2 * jc + half;
-    g2[half] = make_uint2(0u, 0u);
-    if (g < ngran) {
-      const int tap = (int)(((uint32_t)g * recip_gpt) >> 16), i = g - tap * gpt;
-      if ((gmask >> tap) & 1u) g2[half] = *reinterpret_cast<const uint2*>(base + tap_offset(tap, w) * cpad + 8 * i);
-    } else if (g == ngran) {
-      g2[half] = make_uint2(kBiasColumnsLo, kBiasColumnsHi);      // the bias columns
-    }
-  }
-  return make_uint4(g2[0].x, g2[0].y, g2[1].x, g2[1].y);
+  const int4 e = *reinterpret_cast<const int4*>(tab + 2 * jc);       // both granules' entries
+  uint2 g0 = make_uint2(0u, 0u), g1 = make_uint2(0u, 0u);
+  if ((gmask >> e.y) & 1u) g0 = *reinterpret_cast<const uint2*>(base + e.x);
+  if ((gmask >> e.w) & 1u) g1 = *reinterpret_cast<const uint2*>(base + e.z);
+  if (e.y == kGranBias) g0 = make_uint2(kBiasColumnsLo, kBiasColumnsHi);
+  if (e.w == kGranBias) g1 = make_uint2(kBiasColumnsLo, kBiasColumnsHi);
+  return make_uint4(g0.x, g0.y, g1.x, g1.y);
 }
 
 template <bool kPairs>
-__device__ __forceinline__ void build_im2col_t(const Ctx& cx, uint8_t* __restrict__ sA, const int8_t* __restrict__ xa, int cpad,
-                                               int w, int kd, uint32_t recip_gpt, const RowPos rp) {
+__device__ __forceinline__ void build_im2col_t(const Ctx& cx, uint8_t* __restrict__ sA, const int8_t* __restrict__ xa,
+                                               const int2* __restrict__ tab, int cpad, int kd, const RowPos rp) {
   const int nchunks = kd >> 4;
-  const int gpt = cpad >> 3;                // granules per tap
-  const int ngran = 9 * gpt;
   const int8_t* base = xa + (size_t)rp.p * cpad;
   uint8_t* out = sA + cx.row * 16;
   int jc = cx.bcs;
   for (; jc + cx.bncs < nchunks; jc += 2 * cx.bncs) {          // two chunks at a time: independent loads
-    const uint4 c0 = im2col_chunk<kPairs>(base, jc, cpad, w, gpt, ngran, recip_gpt, rp.gmask);
-    const uint4 c1 = im2col_chunk<kPairs>(base, jc + cx.bncs, cpad, w, gpt, ngran, recip_gpt, rp.gmask);
+    const uint4 c0 = im2col_chunk<kPairs>(base, tab, jc, rp.gmask);
+    const uint4 c1 = im2col_chunk<kPairs>(base, tab, jc + cx.bncs, rp.gmask);
     *reinterpret_cast<uint4*>(out + (size_t)jc * (kTileM * 16)) = c0;
     *reinterpret_cast<uint4*>(out + (size_t)(jc + cx.bncs) * (kTileM * 16)) = c1;
   }
   if (jc < nchunks)
-    *reinterpret_cast<uint4*>(out + (size_t)jc * (kTileM * 16)) =
-        im2col_chunk<kPairs>(base, jc, cpad, w, gpt, ngran, recip_gpt, rp.gmask);
+    *reinterpret_cast<uint4*>(out + (size_t)jc * (kTileM * 16)) = im2col_chunk<kPairs>(base, tab, jc, rp.gmask);
 }
 
-__device__ void build_im2col(const Ctx& cx, uint8_t* __restrict__ sA, const int8_t* __restrict__ xa, int cpad, int w,
-                             int kd, uint32_t recip_gpt, const RowPos rp) {
-  if ((cpad & 15) == 0) build_im2col_t<true>(cx, sA, xa, cpad, w, kd, recip_gpt, rp);
-  else build_im2col_t<false>(cx, sA, xa, cpad, w, kd, recip_gpt, rp);
+__device__ __forceinline__ void build_im2col(const Ctx& cx, uint8_t* __restrict__ sA, const int8_t* __restrict__ xa,
+                                             const int2* __restrict__ tab, int cpad, int kd, const RowPos rp) {
+  if ((cpad & 15) == 0) build_im2col_t<true>(cx, sA, xa, tab, cpad, kd, rp);
+  else build_im2col_t<false>(cx, sA, xa, tab, cpad, kd, rp);
 }
 
 // Requantisation flavours of a hidden layer (chosen per layer when the model is packed):
@@ -462,7 +464,7 @@ __device__ void epilogue_prior(const Ctx& cx, const LevelPlan& P, const LevelArg
         const int col = (gi << 3) + i;
         if (col < 2 * cb) {
           const OutRq o = orq[col];
-          const int32_t y = rq_exact((int32_t)r[i] + o.bias, o.m0, o.s);
+          const int32_t y = rq_out((int32_t)r[i], o);
           if (col < cb) mu[(size_t)col * px] = y;
           else ls[(size_t)(col - cb) * px] = clampi(y, M.ls_lo, M.ls_hi);
         }
@@ -826,7 +828,7 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
   uint8_t* sA = smem + P.s_a[0];          // A-operand buffer of the current tile slot
   const uint32_t* rowinfo = reinterpret_cast<const uint32_t*>(smem + P.s_rowinfo);
   const int pg = P.pg, ca = P.ca, cb = P.cb, w = P.w, cpad = P.cpad, cbp = P.cbp;
-  const uint32_t recip_a = P.recip_gpa;
+  const int2* gtab = reinterpret_cast<const int2*>(smem + P.s_gran);
   uint32_t dpar[2] = {0u, 0u};
   const int nslots = P.nslots;
   const CouplingMeta* prevM = nullptr;       // coupling whose translation is still to be applied
@@ -870,7 +872,7 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
       const int c = fdiv(it, mul_pv), p = it - c * pvalid;
       const OutRq o = orq[c];
       int32_t* ap = acc + c * pg + p;
-      const uint32_t t = (uint32_t)rq_exact(*ap + o.bias, o.m0, o.s);
+      const uint32_t t = (uint32_t)rq_out(*ap, o);
       *ap = 0;
       uint32_t* vv = reinterpret_cast<uint32_t*>(&v[colB[c] * pg + p]);
       *vv = kInv ? (*vv - t) : (*vv + t);
@@ -927,7 +929,7 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
         for (int sl = 0; sl < nt; ++sl) {
           use_slot(sl);
           rp[sl] = row_pos(rowinfo, t0 + sl, cx.row, cx.row & (cx.rrows - 1));
-          build_im2col(cx, sA, xa, cpad, w, M.kd, recip_a, rp[sl]);
+          build_im2col(cx, sA, xa, gtab, cpad, M.kd, rp[sl]);
           arrive_a(sl);
         }
         for (int sl = 0; sl < nt; ++sl) {
@@ -947,7 +949,7 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
         for (int sl = 0; sl < nt; ++sl) {                     // conv 3x3: input -> hidden 1
           use_slot(sl);
           rp[sl] = row_pos(rowinfo, t0 + sl, cx.row, cx.row & (cx.rrows - 1));
-          build_im2col(cx, sA, xa, cpad, w, M.kd1, recip_a, rp[sl]);
+          build_im2col(cx, sA, xa, gtab, cpad, M.kd1, rp[sl]);
           arrive_a(sl);
         }
         for (int sl = 0; sl < nt; ++sl) {                     // requant, conv 1x1
@@ -1051,6 +1053,8 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
     for (int idx = tid; idx < P.cb * pg; idx += kWorkers) acc[idx] = 0;
     uint32_t* rowinfo = reinterpret_cast<uint32_t*>(smem + P.s_rowinfo);
     for (int idx = tid; idx < P.tiles * kTileM; idx += kWorkers) rowinfo[idx] = row_record(P.rep > 1 ? (idx & (kTileM / P.rep - 1)) : idx, pvalid, px, P.h, w, P.mul_px, P.mul_w);
+    int32_t* gran = reinterpret_cast<int32_t*>(smem + P.s_gran);
+    for (int idx = tid; idx < 2 * P.n_gran; idx += kWorkers) gran[idx] = P.gran_tab[idx];
     // Everything above used only the plan; from here on the kernel reads what the previous kernel
     // in the stream wrote and writes what it may still be reading.
     ptx::grid_dependency_wait();
