@@ -253,6 +253,51 @@ def main():
            "decode": latency_b1(lambda i: G.iodf_inverse(m, zs[i][:1], xo[i][:1]))}
     G.iodf_check(m)
 
+    # ---- level-stepped decode and patch-based encode of the same workload (single GPU) -----------
+    extra = {}
+    if world == 1:
+        def timed(fn, n):
+            for i in range(3):
+                fn(i)
+            t0e, t1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            stream.synchronize()
+            t0e.record(stream)
+            for i in range(n):
+                fn(i)
+            t1e.record(stream)
+            t1e.synchronize()
+            return t0e.elapsed_time(t1e) / n
+        L = int(lay.n_levels)
+        has_prior = [lv["prior"] is not None for lv in model["levels"]]
+
+        def stepped(i):
+            k = i % N_SETS
+            for lv in range(L - 1, -1, -1):
+                if has_prior[lv]:
+                    G.iodf_inverse_level(m, lv, G.IODF_LEVEL_PRIOR, zs[k], prior=ps[k])
+                G.iodf_inverse_level(m, lv, G.IODF_LEVEL_COUPLINGS, zs[k], x_u8=xo[k])
+        ms = timed(stepped, dec_steps)
+        ok = bool(all(torch.equal(xo[i], xs[i]) for i in range(min(N_SETS, dec_steps))))
+        extra["decode_level_stepped"] = {"value": B / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
+                                         "launches_per_step": L + sum(has_prior), "round_trip_exact": ok}
+        # the batch as the patch grid of one image: patches_y x patches_x patches of the model's input size
+        px_ = 1
+        while px_ * px_ < B:
+            px_ *= 2
+        py_ = B // px_
+        if px_ * py_ == B:
+            hw = model["in_h"]
+            imgs = [x.reshape(py_, px_, 3, hw, hw).permute(2, 0, 3, 1, 4).reshape(3, py_ * hw, px_ * hw).contiguous()
+                    for x in xs]
+            zp, pp = G.iodf_forward_patches(m, imgs[0])
+            same = bool(torch.equal(zp, G.iodf_forward(m, xs[0])[0]))
+            ms = timed(lambda i: G.iodf_forward_patches(m, imgs[i % N_SETS], zs[i % N_SETS], ps[i % N_SETS]),
+                       dec_steps)
+            extra["encode_patches"] = {"image": "3x%dx%d" % (py_ * hw, px_ * hw), "patches": B, "ms_per_image": ms,
+                                       "value": 3.0 * py_ * hw * px_ * hw / (ms * 1e-3) / 1e6, "unit": "MB/s",
+                                       "equals_batch_encode": same}
+        G.iodf_check(m)
+
     # ---- end to end through the host-buffer entry point --------------------------------------
     hx = [torch.from_numpy(S.config_images(cfg, batch=B, seed_offset=rank_seed_offset(rank, i))).pin_memory() for i in range(2)]
     hz = [torch.empty((B, m.d), dtype=torch.int32).pin_memory() for _ in range(2)]
@@ -288,6 +333,7 @@ def main():
                        "round_trip_exact": dec_ok},
             "latency_batch1": lat,
         }
+        out.update(extra)
         if world == 1:
             r, n, dt = oracle_rate(model, cfg, B, cores)
             out["cpu_baseline"] = {"value": r, "unit": UNIT, "cores": cores, "kind": "oracle",

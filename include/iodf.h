@@ -157,6 +157,46 @@ int iodf_inverse(iodf_model* m, const int32_t* z, int B, uint8_t* x_u8, int32_t*
                  uint32_t* out_of_range_count, void* cuda_stream);
 
 /*
+ * Level-stepped decode, for a decompressor that alternates entropy decoding and flow inversion
+ * (the multi-scale architecture of Sec. 5 / App. B.1: the prior of a level's factored-out block is
+ * conditioned on the channels that the level keeps, which a decoder only knows once every deeper
+ * level has been inverted; App. A decodes symbols with those parameters). Call order, for
+ * level = n_levels-1 down to 0:
+ *   IODF_LEVEL_PRIOR      prior parameters of the level's factored-out block (mu at
+ *                         prior[b][0][prior_off[level] ..], log-scale index at prior[b][1][..]) from the
+ *                         level's kept channels: z's final block for the deepest level, otherwise what
+ *                         the IODF_LEVEL_COUPLINGS call of level+1 left in the model's workspace. No
+ *                         other part of z is read, nothing else is written. Levels without a prior
+ *                         head return IODF_EINVAL (their block has a fixed prior).
+ *   (the caller entropy-decodes the level's block z[b][z_off[level] ..] with those parameters)
+ *   IODF_LEVEL_COUPLINGS  merges the kept channels with the level's block of z, inverts the level's
+ *                         couplings and the squeeze; the result is the kept input of level-1 (model
+ *                         workspace) or, for level 0, x_u8 (and out_of_range_count, as iodf_inverse).
+ *                         Reads only z's block of this level (and the final block at the deepest level).
+ * z, prior, x_u8: DEV, full-size buffers with the layouts of iodf_forward; x_u8 is used at level 0
+ * only and prior by IODF_LEVEL_PRIOR only (either may be NULL otherwise). The sequence over all
+ * levels gives bit for bit what iodf_inverse gives. One sequence per model at a time.
+ */
+#define IODF_LEVEL_PRIOR 1
+#define IODF_LEVEL_COUPLINGS 2
+int iodf_inverse_level(iodf_model* m, int level, int phase, const int32_t* z, int B, uint8_t* x_u8, int32_t* prior,
+                       uint32_t* out_of_range_count, void* cuda_stream);
+
+/*
+ * Patch-based coding of one high-resolution image (Sec. 5.3: a large image is cut into patches
+ * of the training resolution, which "naturally gives rise to a large batch size"). image_u8 is DEV
+ * uint8 [in_c][H][W] with H, W multiples of in_h, in_w; patch b = (b / (W/in_w), b % (W/in_w)) in
+ * row-major order is image b of a batch of B = (H/in_h)*(W/in_w) <= max_batch images. The cut is an
+ * index map of the first level's load (encode) and last store (decode): no patch batch is
+ * materialised. z is [B][d] and prior [B][2][d_fact] exactly as for iodf_forward on that batch.
+ * Errors: IODF_EINVAL if H or W is not a multiple of the patch size or B exceeds max_batch.
+ */
+int iodf_forward_patches(iodf_model* m, const uint8_t* image_u8, int H, int W, int32_t* z, int32_t* prior,
+                         void* cuda_stream);
+int iodf_inverse_patches(iodf_model* m, const int32_t* z, int H, int W, uint8_t* image_u8, int32_t* prior,
+                         uint32_t* out_of_range_count, void* cuda_stream);
+
+/*
  * The same two operations for HOST buffers (pinned memory recommended): inputs are copied to a
  * device staging area owned by the model, the flow runs, and the results are copied back, all
  * enqueued on `cuda_stream`; the host buffers are valid once the stream has been synchronised.

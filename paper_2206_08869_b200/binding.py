@@ -12,6 +12,7 @@ IODF_ABI_VERSION = 1
 IODF_MAX_LEVELS = 8
 
 DECLARED_SYMBOLS = ["iodf_create", "iodf_destroy", "iodf_get_layout", "iodf_forward", "iodf_inverse",
+                    "iodf_inverse_level", "iodf_forward_patches", "iodf_inverse_patches",
                     "iodf_forward_host", "iodf_inverse_host", "iodf_forward_timed", "iodf_inverse_timed", "iodf_forward_static",
                     "iodf_static_scratch_bytes_per_image", "iodf_check", "iodf_launches_per_call",
                     "iodf_strerror", "iodf_last_cuda_error"]
@@ -77,6 +78,12 @@ def load_library(path=None):
     L.iodf_forward.argtypes = [vp, vp, C.c_int, vp, vp, vp]
     L.iodf_inverse.restype = C.c_int
     L.iodf_inverse.argtypes = [vp, vp, C.c_int, vp, vp, vp, vp]
+    L.iodf_inverse_level.restype = C.c_int
+    L.iodf_inverse_level.argtypes = [vp, C.c_int, C.c_int, vp, C.c_int, vp, vp, vp, vp]
+    L.iodf_forward_patches.restype = C.c_int
+    L.iodf_forward_patches.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp, vp]
+    L.iodf_inverse_patches.restype = C.c_int
+    L.iodf_inverse_patches.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp, vp, vp]
     L.iodf_forward_host.restype = C.c_int
     L.iodf_forward_host.argtypes = [vp, vp, C.c_int, vp, vp, vp]
     L.iodf_inverse_host.restype = C.c_int
@@ -228,6 +235,46 @@ def iodf_inverse(model, z, x_u8=None, prior=None, out_of_range=None, stream=None
     if rc != 0:
         raise IodfError(rc, "iodf_inverse")
     return x_u8
+
+
+IODF_LEVEL_PRIOR = 1
+IODF_LEVEL_COUPLINGS = 2
+
+
+def iodf_inverse_level(model, level, phase, z, x_u8=None, prior=None, out_of_range=None, stream=None):
+    """One step of the level-stepped decode (see include/iodf.h). z: cuda int32 [B,d] (full size)."""
+    rc = load_library().iodf_inverse_level(model.handle, level, phase, _ptr(z), z.shape[0], _ptr(x_u8), _ptr(prior),
+                                           _ptr(out_of_range), _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_inverse_level")
+
+
+def iodf_forward_patches(model, image_u8, z=None, prior=None, stream=None):
+    """image_u8: cuda uint8 [C,H,W], H and W multiples of the model's input size. Returns (z, prior)
+    of the batch of patches in row-major patch order."""
+    import torch
+    _, H, W = image_u8.shape
+    B = (H // model.in_shape[1]) * (W // model.in_shape[2])
+    if z is None:
+        z = torch.empty((B, model.d), dtype=torch.int32, device=image_u8.device)
+    if prior is None and model.d_fact:
+        prior = torch.empty((B, 2, model.d_fact), dtype=torch.int32, device=image_u8.device)
+    rc = load_library().iodf_forward_patches(model.handle, _ptr(image_u8), H, W, _ptr(z), _ptr(prior), _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_forward_patches")
+    return z, prior
+
+
+def iodf_inverse_patches(model, z, H, W, image_u8=None, prior=None, out_of_range=None, stream=None):
+    """z: cuda int32 [B,d] of the patch batch. Returns the image uint8 [C,H,W]."""
+    import torch
+    if image_u8 is None:
+        image_u8 = torch.empty((model.in_shape[0], H, W), dtype=torch.uint8, device=z.device)
+    rc = load_library().iodf_inverse_patches(model.handle, _ptr(z), H, W, _ptr(image_u8), _ptr(prior),
+                                             _ptr(out_of_range), _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_inverse_patches")
+    return image_u8
 
 
 def iodf_forward_host(model, x_u8, z, prior=None, stream=None):

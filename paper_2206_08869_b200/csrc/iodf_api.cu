@@ -575,8 +575,18 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The batch as the patch grid of one image (first level's load / last store); img_w = 0: a plain batch.
+struct PatchGrid {
+  int img_h = 0, img_w = 0, patches_x = 0;
+};
+
+void set_patch_grid(LevelArgs& a, const PatchGrid& g) {
+  a.img_h = g.img_h; a.img_w = g.img_w; a.patches_x = g.patches_x;
+  a.mul_patches_x = g.patches_x > 1 ? (uint32_t)(((1ull << 32) + g.patches_x - 1) / g.patches_x) : 0u;
+}
+
 int run_forward(iodf_model* m, const uint8_t* x, int B, int32_t* z, int32_t* prior, cudaStream_t st,
-                bool timed = false) {
+                bool timed = false, PatchGrid grid = PatchGrid()) {
   const size_t L = m->levels.size();
   if (timed) CU(m, cudaEventRecord(m->ev[0], st));
   for (size_t li = 0; li < L; ++li) {
@@ -592,32 +602,56 @@ int run_forward(iodf_model* m, const uint8_t* x, int B, int32_t* z, int32_t* pri
     a.oor = nullptr;
     a.status = m->d_status;
     a.batch = B;
+    if (li == 0) set_patch_grid(a, grid);
     CU(m, launch_level(a, false, (B + P.group - 1) / P.group, P.s_total, st));
     if (timed) CU(m, cudaEventRecord(m->ev[li + 1], st));
   }
   return IODF_OK;
 }
 
+// One decode launch of level li. phase: 0 = whole level, 1 = prior head only, 2 = couplings only.
+int launch_inverse_level(iodf_model* m, int li, int phase, const int32_t* z, int B, uint8_t* x, int32_t* prior,
+                         uint32_t* oor, cudaStream_t st, const PatchGrid& grid) {
+  const int L = (int)m->levels.size();
+  const LevelPlan& P = m->levels[li].plan;
+  LevelArgs a{};
+  a.plan = m->d_plan[li];
+  a.blob = m->d_blob[li];
+  if (li == L - 1) { a.in = z + m->layout.z_final_off; a.in_stride = (long long)m->layout.d; }
+  else { a.in = m->d_keep[li]; a.in_stride = (long long)P.keep_c * P.px; }
+  a.z = const_cast<int32_t*>(z);
+  a.prior = prior;
+  a.out = li == 0 ? (void*)x : (void*)m->d_keep[li - 1];
+  a.oor = oor;
+  a.status = m->d_status;
+  a.batch = B;
+  a.phase = phase;
+  if (li == 0) set_patch_grid(a, grid);
+  CU(m, launch_level(a, true, (B + P.group - 1) / P.group, P.s_total, st));
+  return IODF_OK;
+}
+
 int run_inverse(iodf_model* m, const int32_t* z, int B, uint8_t* x, int32_t* prior, uint32_t* oor, cudaStream_t st,
-                bool timed = false) {
+                bool timed = false, PatchGrid grid = PatchGrid()) {
   const int L = (int)m->levels.size();
   if (timed) CU(m, cudaEventRecord(m->ev[L], st));
   for (int li = L - 1; li >= 0; --li) {
-    const LevelPlan& P = m->levels[li].plan;
-    LevelArgs a{};
-    a.plan = m->d_plan[li];
-    a.blob = m->d_blob[li];
-    if (li == L - 1) { a.in = z + m->layout.z_final_off; a.in_stride = (long long)m->layout.d; }
-    else { a.in = m->d_keep[li]; a.in_stride = (long long)P.keep_c * P.px; }
-    a.z = const_cast<int32_t*>(z);
-    a.prior = prior;
-    a.out = li == 0 ? (void*)x : (void*)m->d_keep[li - 1];
-    a.oor = oor;
-    a.status = m->d_status;
-    a.batch = B;
-    CU(m, launch_level(a, true, (B + P.group - 1) / P.group, P.s_total, st));
+    int rc = launch_inverse_level(m, li, 0, z, B, x, prior, oor, st, grid);
+    if (rc) return rc;
     if (timed) CU(m, cudaEventRecord(m->ev[li], st));
   }
+  return IODF_OK;
+}
+
+// H x W image as a grid of in_h x in_w patches: the batch size, or an error
+int patch_grid(const iodf_model* m, int H, int W, PatchGrid* g, int* B) {
+  if (H < 1 || W < 1 || H % (int)m->in_h || W % (int)m->in_w) return IODF_EINVAL;
+  const long long n = (long long)(H / (int)m->in_h) * (W / (int)m->in_w);
+  if (n < 1 || n > (long long)m->max_batch) return IODF_EINVAL;
+  // the patch index is split with a 32-bit magic multiplier: exact while B * patches_x < 2^32
+  if ((unsigned long long)n * (unsigned long long)(W / (int)m->in_w) >= (1ull << 32)) return IODF_EUNSUPPORTED;
+  g->img_h = H; g->img_w = W; g->patches_x = W / (int)m->in_w;
+  *B = (int)n;
   return IODF_OK;
 }
 
@@ -777,6 +811,45 @@ int iodf_inverse(iodf_model* m, const int32_t* z, int B, uint8_t* x_u8, int32_t*
   if (!aligned16(x_u8) || !aligned16(z) || !aligned16(prior)) return IODF_EINVAL;
   return run_inverse(m, z, B, x_u8, m->layout.d_fact ? prior : nullptr, out_of_range_count,
                      (cudaStream_t)cuda_stream);
+}
+
+int iodf_inverse_level(iodf_model* m, int level, int phase, const int32_t* z, int B, uint8_t* x_u8, int32_t* prior,
+                       uint32_t* out_of_range_count, void* cuda_stream) {
+  if (!m || !z || B < 1 || (uint32_t)B > m->max_batch) return IODF_EINVAL;
+  if (level < 0 || level >= (int)m->levels.size()) return IODF_EINVAL;
+  if (phase != IODF_LEVEL_PRIOR && phase != IODF_LEVEL_COUPLINGS) return IODF_EINVAL;
+  if (!aligned16(z) || !aligned16(prior) || !aligned16(x_u8)) return IODF_EINVAL;
+  const LevelPlan& P = m->levels[level].plan;
+  if (phase == IODF_LEVEL_PRIOR) {
+    if (!P.has_prior || !prior) return IODF_EINVAL;
+    return launch_inverse_level(m, level, 1, z, B, nullptr, prior, nullptr, (cudaStream_t)cuda_stream, PatchGrid());
+  }
+  if (level == 0 && !x_u8) return IODF_EINVAL;
+  return launch_inverse_level(m, level, 2, z, B, x_u8, nullptr, out_of_range_count, (cudaStream_t)cuda_stream,
+                              PatchGrid());
+}
+
+int iodf_forward_patches(iodf_model* m, const uint8_t* image_u8, int H, int W, int32_t* z, int32_t* prior,
+                         void* cuda_stream) {
+  if (!m || !image_u8 || !z) return IODF_EINVAL;
+  if (!aligned16(image_u8) || !aligned16(z) || !aligned16(prior)) return IODF_EINVAL;
+  PatchGrid g;
+  int B = 0;
+  int rc = patch_grid(m, H, W, &g, &B);
+  if (rc) return rc;
+  return run_forward(m, image_u8, B, z, m->layout.d_fact ? prior : nullptr, (cudaStream_t)cuda_stream, false, g);
+}
+
+int iodf_inverse_patches(iodf_model* m, const int32_t* z, int H, int W, uint8_t* image_u8, int32_t* prior,
+                         uint32_t* out_of_range_count, void* cuda_stream) {
+  if (!m || !image_u8 || !z) return IODF_EINVAL;
+  if (!aligned16(image_u8) || !aligned16(z) || !aligned16(prior)) return IODF_EINVAL;
+  PatchGrid g;
+  int B = 0;
+  int rc = patch_grid(m, H, W, &g, &B);
+  if (rc) return rc;
+  return run_inverse(m, z, B, image_u8, m->layout.d_fact ? prior : nullptr, out_of_range_count,
+                     (cudaStream_t)cuda_stream, false, g);
 }
 
 int iodf_forward_timed(iodf_model* m, const uint8_t* x_u8, int B, int32_t* z, int32_t* prior, void* cuda_stream,

@@ -158,11 +158,6 @@ __device__ __forceinline__ RowPos row_pos(const uint32_t* rowinfo, int tile, int
   return r;
 }
 
-__device__ __forceinline__ int tap_offset(int tap, int w) {
-  const int u = (tap * 11) >> 5;            // tap / 3 for 0..8
-  return (u - 1) * w + (tap - u * 3 - 1);
-}
-
 // A[row][tap*cpad + c] = xa[p + tap offset][c] (0 outside the image), as aligned 8-byte granules,
 // followed by the granule of bias columns (where K has room for it), written in 16-byte chunks into
 // the MMA operand layout [K/16][128][16]. Where each granule comes from is a property of the level,
@@ -1016,9 +1011,9 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
   int32_t* v = reinterpret_cast<int32_t*>(smem + P.s_v);
 
   Steps st;
-  st.n_couplings = P.n_couplings;
-  st.do_prior = P.has_prior && a.prior != nullptr;
-  st.nsteps = P.n_couplings + (st.do_prior ? 1 : 0);
+  st.n_couplings = (kInv && a.phase == 1) ? 0 : P.n_couplings;
+  st.do_prior = P.has_prior && a.prior != nullptr && !(kInv && a.phase == 2);
+  st.nsteps = st.n_couplings + (st.do_prior ? 1 : 0);
   st.inverse = kInv;
 
   Ctx cx;
@@ -1066,7 +1061,11 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
         const int g = fdiv(e, P.mul_per_img), r = e - g * per_img;
         const int ci = fdiv(r, P.mul_4px), r2 = r - ci * 4 * px;
         const int y = fdiv(r2, P.mul_w2), x = r2 - y * w2;
-        const size_t src = (size_t)(img0 + g) * per_img + r;
+        size_t src = (size_t)(img0 + g) * per_img + r;
+        if (P.is_first && a.img_w > 0) {                 // patch (by, bx) of one large image
+          const int by = fdiv(img0 + g, a.mul_patches_x), bx = img0 + g - by * a.patches_x;
+          src = ((size_t)ci * a.img_h + (size_t)(by * 2 * P.h + y)) * a.img_w + (size_t)(bx * w2 + x);
+        }
         const int32_t val = P.is_first ? (int32_t) reinterpret_cast<const uint8_t*>(a.in)[src]
                                        : reinterpret_cast<const int32_t*>(a.in)[src];
         v[(ci * 4 + (y & 1) * 2 + (x & 1)) * pg + g * px + (y >> 1) * w + (x >> 1)] = val;
@@ -1078,6 +1077,7 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
         const int g = fdiv(e, P.mul_per_img), r = e - g * per_img;
         const int k = fdiv(r, P.mul_px), q = r - k * px;
         const size_t b = (size_t)(img0 + g);
+        if (a.phase == 1 && k >= P.keep_c) continue;     // prior head only: z's block is not read
         const int32_t val =
             (k < P.keep_c) ? reinterpret_cast<const int32_t*>(a.in)[b * (size_t)a.in_stride + (size_t)k * px + q]
                            : a.z[b * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q];
@@ -1102,7 +1102,7 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
         else if (P.is_last) a.z[b * P.d + P.z_final_off + (size_t)k * px + q] = val;
         else keep_out[(b * P.keep_c + k) * (size_t)px + q] = val;
       }
-    } else {
+    } else if (a.phase != 1) {
       // depth-to-space on store
       const int w2 = 2 * w;
       uint32_t bad = 0;
@@ -1112,7 +1112,11 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
         const int ci = fdiv(r, P.mul_4px), r2 = r - ci * 4 * px;
         const int y = fdiv(r2, P.mul_w2), x = r2 - y * w2;
         const int32_t val = v[(ci * 4 + (y & 1) * 2 + (x & 1)) * pg + g * px + (y >> 1) * w + (x >> 1)];
-        const size_t dst = (size_t)(img0 + g) * per_img + r;
+        size_t dst = (size_t)(img0 + g) * per_img + r;
+        if (P.is_first && a.img_w > 0) {
+          const int by = fdiv(img0 + g, a.mul_patches_x), bx = img0 + g - by * a.patches_x;
+          dst = ((size_t)ci * a.img_h + (size_t)(by * 2 * P.h + y)) * a.img_w + (size_t)(bx * w2 + x);
+        }
         if (P.is_first) {
           reinterpret_cast<uint8_t*>(a.out)[dst] = (uint8_t)((uint32_t)val & 0xFFu);
           bad += (val < 0 || val > 255) ? 1u : 0u;

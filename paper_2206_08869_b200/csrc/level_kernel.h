@@ -25,6 +25,14 @@ struct LevelArgs {
   uint32_t* oor;           // decode, first level: count of recovered values outside 0..255, or null
   uint32_t* status;        // device status word (non-zero: a bounded wait gave up)
   int batch;
+  // decode only: 0 = the whole level; 1 = prior head only (reads the kept channels, writes prior
+  // parameters, stores nothing else); 2 = couplings only (no prior head)
+  int phase;
+  // first level only, img_w > 0: the batch is the grid of in_h x in_w patches of one image
+  // [c][img_h][img_w] (patch b = row b / patches_x, column b % patches_x), read (encode) or written
+  // (decode) in place of the [B][c][in_h][in_w] batch. mul_patches_x = ceil(2^32 / patches_x), 0 for 1.
+  int img_h, img_w, patches_x;
+  uint32_t mul_patches_x;
 };
 
 cudaError_t configure_level_kernels(uint32_t max_smem_bytes);
