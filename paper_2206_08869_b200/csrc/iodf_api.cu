@@ -86,13 +86,15 @@ int check_overflow(const iodf_layer_desc& L, const Blobs& B, int64_t amax) {
 
 struct Act { int lo, hi; };
 
-// Effective range of a hidden layer's output; must be inside the signed 8-bit range.
+// Effective range of a hidden layer's output; must be inside the signed (-128..127) or the unsigned
+// (0..255, the format of Sec. 4.1 for non-negative tensors) 8-bit range.
 int hidden_range(const iodf_layer_desc& L, Act* out) {
   if (!L.has_clamp) return IODF_EUNSUPPORTED;
   int lo = L.clamp_lo, hi = L.clamp_hi;
   if (L.relu) lo = std::max(lo, 0);
   if (lo > hi) { lo = hi; }
-  if (lo < -128 || hi > 127) return IODF_EUNSUPPORTED;
+  const bool fits_signed = lo >= -128 && hi <= 127, fits_unsigned = lo >= 0 && hi <= 255;
+  if (!fits_signed && !fits_unsigned) return IODF_EUNSUPPORTED;
   out->lo = lo;
   out->hi = hi;
   return IODF_OK;

@@ -219,15 +219,23 @@ __device__ __forceinline__ void build_im2col(const Ctx& cx, uint8_t* __restrict_
 constexpr int kModeFolded = 3, kModeUniform = 2, kModeFast = 1, kModeExact = 0;
 
 // Clip flavours: kClipS8Relu is the common ReLU + clip to [0, 127]: the saturating 32->8 bit pack
-// clips to [-128, 127] and the negative bytes are then cleared; kClipAny is max/min with the
-// layer's bounds.
-constexpr int kClipS8Relu = 1, kClipAny = 0;
+// clips to [-128, 127] and the negative bytes are then cleared; kClipU8Relu is ReLU + clip to
+// [0, 255] (unsigned activations, Sec. 4.1), which the unsigned saturating pack does by itself;
+// kClipAny is max/min with the layer's bounds.
+constexpr int kClipS8Relu = 1, kClipU8Relu = 2, kClipAny = 0;
 
 // d = {sat8(y3), sat8(y2), sat8(y1), sat8(y0)} (y0 in the lowest byte)
 __device__ __forceinline__ uint32_t pack4_sat(int y0, int y1, int y2, int y3) {
   uint32_t t, w;
   asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(y3), "r"(y2), "r"(0));
   asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(y1), "r"(y0), "r"(t));
+  return w;
+}
+// d = {satu8(y3), satu8(y2), satu8(y1), satu8(y0)}: clip(y, 0, 255) of four values
+__device__ __forceinline__ uint32_t pack4_sat_u8(int y0, int y1, int y2, int y3) {
+  uint32_t t, w;
+  asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(y3), "r"(y2), "r"(0));
+  asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(y1), "r"(y0), "r"(t));
   return w;
 }
 // clip(y, 0, 127) of four values: saturate to int8 while packing, then clear the negative bytes
@@ -259,7 +267,7 @@ struct Requant {
       if (kMode == kModeFast) y = ((int)(p >> 32)) >> r.sh;
       else y = (int)(p >> (32 + r.sh));
     }
-    return kClip == kClipS8Relu ? y : clampi(y, lo, hi);     // kClipS8Relu: clipped while packing
+    return kClip != kClipAny ? y : clampi(y, lo, hi);        // otherwise clipped while packing
   }
   // 16 accumulator columns starting at channel ch0 -> one 16-byte chunk of the next A operand
   __device__ __forceinline__ uint4 chunk(const uint32_t* r, int ch0) const {
@@ -272,7 +280,7 @@ struct Requant {
         const int4 c = q[i];
         const int y0 = uniform_one((int)r[4 * i], c.x, 0), y1 = uniform_one((int)r[4 * i + 1], c.y, 0);
         const int y2 = uniform_one((int)r[4 * i + 2], c.z, 0), y3 = uniform_one((int)r[4 * i + 3], c.w, 0);
-        wd[i] = kClip == kClipS8Relu ? pack4_relu_sat(y0, y1, y2, y3) : pack4(y0, y1, y2, y3);
+        wd[i] = pack_clipped(y0, y1, y2, y3);
       }
     } else if (kMode == kModeUniform) {
       // {m0, bias} pairs of two channels per 16-byte shared-memory load (the table is 16-byte aligned)
@@ -282,14 +290,14 @@ struct Requant {
         const int4 c01 = q[2 * i], c23 = q[2 * i + 1];
         const int y0 = uniform_one((int)r[4 * i], c01.x, c01.y), y1 = uniform_one((int)r[4 * i + 1], c01.z, c01.w);
         const int y2 = uniform_one((int)r[4 * i + 2], c23.x, c23.y), y3 = uniform_one((int)r[4 * i + 3], c23.z, c23.w);
-        wd[i] = kClip == kClipS8Relu ? pack4_relu_sat(y0, y1, y2, y3) : pack4(y0, y1, y2, y3);
+        wd[i] = pack_clipped(y0, y1, y2, y3);
       }
     } else {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int y0 = one((int)r[4 * i], ch0 + 4 * i), y1 = one((int)r[4 * i + 1], ch0 + 4 * i + 1);
         const int y2 = one((int)r[4 * i + 2], ch0 + 4 * i + 2), y3 = one((int)r[4 * i + 3], ch0 + 4 * i + 3);
-        wd[i] = kClip == kClipS8Relu ? pack4_relu_sat(y0, y1, y2, y3) : pack4(y0, y1, y2, y3);
+        wd[i] = pack_clipped(y0, y1, y2, y3);
       }
     }
     return make_uint4(wd[0], wd[1], wd[2], wd[3]);
@@ -297,7 +305,11 @@ struct Requant {
   __device__ __forceinline__ int uniform_one(int acc, int m0, int bias) const {
     const long long p = (long long)(acc + bias) * (long long)m0 + rnd64;
     const int y = ((int)(p >> 32)) >> sh;
-    return kClip == kClipS8Relu ? y : clampi(y, lo, hi);
+    return kClip != kClipAny ? y : clampi(y, lo, hi);
+  }
+  __device__ __forceinline__ uint32_t pack_clipped(int y0, int y1, int y2, int y3) const {
+    return kClip == kClipS8Relu ? pack4_relu_sat(y0, y1, y2, y3)
+                                : (kClip == kClipU8Relu ? pack4_sat_u8(y0, y1, y2, y3) : pack4(y0, y1, y2, y3));
   }
 };
 
@@ -347,11 +359,12 @@ __device__ __forceinline__ void epilogue_hidden_t(const Ctx& cx, int n, int kd, 
 __device__ __forceinline__ void epilogue_hidden(const Ctx& cx, int mode, int us, int n, int kd, const HiddenRq* rq,
                                                 const int2* mb, int lo, int hi, uint32_t pad_lo, uint32_t pad_hi,
                                                 uint8_t* sOut) {
-  const bool s8relu = lo == 0 && hi == 127;
+  const bool s8relu = lo == 0 && hi == 127, u8relu = lo == 0 && hi == 255;
   if (mode >= kModeUniform) {
     const long long rnd64 = 1ll << (30 + us);
     if (mode == kModeFolded) {
       if (s8relu) epilogue_hidden_t(cx, n, kd, Requant<kModeFolded, kClipS8Relu>{rq, mb, lo, hi, us - 1, rnd64}, pad_lo, pad_hi, sOut);
+      else if (u8relu) epilogue_hidden_t(cx, n, kd, Requant<kModeFolded, kClipU8Relu>{rq, mb, lo, hi, us - 1, rnd64}, pad_lo, pad_hi, sOut);
       else epilogue_hidden_t(cx, n, kd, Requant<kModeFolded, kClipAny>{rq, mb, lo, hi, us - 1, rnd64}, pad_lo, pad_hi, sOut);
     } else {
       if (s8relu) epilogue_hidden_t(cx, n, kd, Requant<kModeUniform, kClipS8Relu>{rq, mb, lo, hi, us - 1, rnd64}, pad_lo, pad_hi, sOut);
@@ -487,8 +500,8 @@ __device__ __forceinline__ const BlockRef& step_ref(const LevelPlan& P, const St
 // The control thread competes for issue slots with sixteen busy worker warps, so the loop body is
 // kept to the MMA and two descriptor increments (K advances by 32 bytes = two 16-byte chunks).
 __device__ __forceinline__ void issue_gemm(uint32_t d_tmem, uint32_t sa, uint32_t sb, int n_total, int n0, int n,
-                                           int kd) {
-  const uint32_t idesc = ptx::umma_idesc_s8((uint32_t)n);
+                                           int kd, bool a_unsigned) {
+  const uint32_t idesc = ptx::umma_idesc_i8((uint32_t)n, a_unsigned);
   const uint32_t lbo_b = (uint32_t)n_total * 16u;
   uint64_t da = ptx::umma_desc(sa, kTileM * 16, 128);
   uint64_t db = ptx::umma_desc(sb + (uint32_t)n0 * 16u, lbo_b, 128);
@@ -573,14 +586,14 @@ __device__ void run_control(const Ctx& cx, const LevelPlan& P, const LevelArgs& 
   __syncwarp();
   cta_barrier();                         // the workers have loaded the flow variable
   // wait for tile slot sl's A operand, then D = A * W^T into the slot's TMEM columns
-  auto mma = [&](int sl, int wslot, bool wait_w, uint32_t wpar, int n, int kd) {
+  auto mma = [&](int sl, int wslot, bool wait_w, uint32_t wpar, int n, int kd, bool au) {
     spin_then_wait(ctl, a.status, &ctl->a_ready[sl], apar[sl]);
     apar[sl] ^= 1u;
     if (wait_w) spin_then_wait(ctl, a.status, &ctl->w_full[wslot], wpar);
     ptx::tc_fence_after();
     const uint32_t sa = ptx::smem_u32(smem + P.s_a[sl]), sb = ptx::smem_u32(smem + P.s_w[wslot]);
     const uint32_t d = cx.tmem_base + (uint32_t)(sl * kSlotCols);
-    for (int n0 = 0; n0 < n; n0 += 256) issue_gemm(d + (uint32_t)n0, sa, sb, n, n0, min(256, n - n0), kd);
+    for (int n0 = 0; n0 < n; n0 += 256) issue_gemm(d + (uint32_t)n0, sa, sb, n, n0, min(256, n - n0), kd, au);
     ptx::umma_commit(ptx::smem_u32(&ctl->d_ready[sl]));
   };
   // alias mode only: wait until the MMA just issued for slot 0 has completed, then refill S0
@@ -593,6 +606,7 @@ __device__ void run_control(const Ctx& cx, const LevelPlan& P, const LevelArgs& 
   for (int i = 0; i < st.nsteps; ++i) {
     const bool prior = st.is_prior(i);
     int n[3] = {0, 0, 0}, kd[3] = {0, 0, 0};
+    bool au[3] = {false, false, false};      // A operand unsigned: hidden activations clipped above 127
     if (lead) {
       wait_bar(ctl, a.status, &ctl->meta_full[i & 1], (uint32_t)((i >> 1) & 1));
       const uint8_t* mb = smem + P.s_meta[i & 1];
@@ -603,6 +617,7 @@ __device__ void run_control(const Ctx& cx, const LevelPlan& P, const LevelArgs& 
         const CouplingMeta* M = reinterpret_cast<const CouplingMeta*>(mb);
         n[0] = M->n1; n[1] = M->n2; n[2] = M->n3;
         kd[0] = M->kd1; kd[1] = M->kd2; kd[2] = M->kd3;
+        au[1] = M->hi1 > 127; au[2] = M->hi2 > 127;
       }
     }
     cta_barrier();     // the workers have finished the pixel pass: step i-1's meta slot is free
@@ -625,7 +640,7 @@ __device__ void run_control(const Ctx& cx, const LevelPlan& P, const LevelArgs& 
 #pragma unroll
         for (int sg = 0; sg < 3; ++sg) {
           const uint32_t lbo_b = (uint32_t)n[sg] * 16u;
-          idesc[sg] = ptx::umma_idesc_s8((uint32_t)n[sg]);
+          idesc[sg] = ptx::umma_idesc_i8((uint32_t)n[sg], au[sg]);
           db_lo[sg] = ptx::umma_desc_lo(ptx::smem_u32(smem + P.s_w[sg]), lbo_b);
           db_step[sg] = (2u * lbo_b) >> 4;
           ks[sg] = kd[sg] >> 5;
@@ -670,15 +685,15 @@ __device__ void run_control(const Ctx& cx, const LevelPlan& P, const LevelArgs& 
           for (int sl = 0; sl < nt; ++sl) {
             if (!alias) {
               const int wslot = prior ? 0 : stage;
-              mma(sl, wslot, first && sl == 0, wslot == 0 ? par0 : par12, n[stage], kd[stage]);
+              mma(sl, wslot, first && sl == 0, wslot == 0 ? par0 : par12, n[stage], kd[stage], au[stage]);
               dpar[sl] ^= 1u;
             } else if (stage == 1) {
-              mma(sl, 1, first, par12, n[1], kd[1]);
+              mma(sl, 1, first, par12, n[1], kd[1], au[1]);
               dpar[sl] ^= 1u;
             } else {
               // S0 holds, in turn: W1, W3 of every tile (coupling) or the prior matrix for all tiles
               const bool ww = prior ? first : true;
-              mma(sl, 0, ww, W.s0_used & 1u, n[stage], kd[stage]);
+              mma(sl, 0, ww, W.s0_used & 1u, n[stage], kd[stage], au[stage]);
               if (ww) ++W.s0_used;
               if (prior) {
                 if (last_tile && i + 1 < st.nsteps) s0_refill(step_ref(P, st, i + 1), 0);
@@ -760,6 +775,7 @@ __device__ void run_control_streamed(const Ctx& cx, const LevelPlan& P, const Le
   for (int i = 0; i < st.nsteps; ++i) {
     const bool prior = st.is_prior(i);
     int n[3] = {0, 0, 0};
+    bool au[3] = {false, false, false};
     if (lead) {
       wait_bar(ctl, a.status, &ctl->meta_full[i & 1], (uint32_t)((i >> 1) & 1));
       const uint8_t* mb = smem + P.s_meta[i & 1];
@@ -768,6 +784,7 @@ __device__ void run_control_streamed(const Ctx& cx, const LevelPlan& P, const Le
       } else {
         const CouplingMeta* M = reinterpret_cast<const CouplingMeta*>(mb);
         n[0] = M->n1; n[1] = M->n2; n[2] = M->n3;
+        au[1] = M->hi1 > 127; au[2] = M->hi2 > 127;
       }
     }
     cta_barrier();     // the workers have finished the pixel pass: step i-1's meta slot is free
@@ -794,7 +811,7 @@ __device__ void run_control_streamed(const Ctx& cx, const LevelPlan& P, const Le
             const uint64_t da = ptx::umma_desc(sa + (uint32_t)k * 2u * (kTileM * 16), kTileM * 16, 128);
             for (int n0 = 0; n0 < nn; n0 += 256) {
               const uint64_t db = ptx::umma_desc(sb + (uint32_t)n0 * 16u, lbo_b, 128);
-              const uint32_t idesc = ptx::umma_idesc_s8((uint32_t)min(256, nn - n0));
+              const uint32_t idesc = ptx::umma_idesc_i8((uint32_t)min(256, nn - n0), au[stage]);
               if (k == 0) ptx::umma_i8_first(cx.tmem_base + (uint32_t)n0, da, db, idesc);
               else ptx::umma_i8_acc(cx.tmem_base + (uint32_t)n0, da, db, idesc);
             }

@@ -162,9 +162,10 @@ __device__ __forceinline__ uint32_t umma_desc_lo(uint32_t saddr, uint32_t lbo) {
   return ((saddr >> 4) & 0x3FFFu) | (((lbo >> 4) & 0x3FFFu) << 16);
 }
 constexpr uint32_t kUmmaDescHi = ((128u >> 4) & 0x3FFFu) | (1u << 14);   // stride offset 128 bytes, version 1
-// Instruction descriptor: D = s32, A and B signed 8-bit, both K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t umma_idesc_s8(uint32_t n) {
-  return (2u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptor: D = s32, B signed 8-bit, A signed or unsigned 8-bit (format field 1 or 0),
+// both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc_i8(uint32_t n, bool a_unsigned) {
+  return (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                         uint32_t accumulate) {

@@ -71,8 +71,11 @@ def test_bad_descriptors_fail_on_the_host():
     m["levels"][0]["couplings"][0]["layers"][2]["relu"] = True
     assert _status(m) == EINVAL                      # the translation layer must not clip
     m = _small()
-    m["levels"][0]["couplings"][0]["layers"][0]["clamp"] = (0, 255)
-    assert _status(m) == EUNSUPPORTED                # unsigned activations: not in this build
+    m["levels"][0]["couplings"][0]["layers"][0]["clamp"] = (-5, 300)
+    assert _status(m) == EUNSUPPORTED                # after the ReLU 0..300: beyond the unsigned 8-bit range
+    m = _small()
+    m["levels"][0]["couplings"][0]["layers"][1]["clamp"] = (0, 256)
+    assert _status(m) == EUNSUPPORTED
     m = _small()
     m["in_h"] = 6                                    # not divisible by 2^levels
     assert _status(m) == EINVAL

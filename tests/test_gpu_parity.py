@@ -123,6 +123,42 @@ def test_biases_around_the_folding_limit(G):
     _check_both_ways(G, model, x)
 
 
+def test_unsigned_hidden_activations(G):
+    """Hidden activations in the unsigned 8-bit format (0..255 after the ReLU, Sec. 4.1): the next
+    conv then reads an unsigned A operand. Shifts are lowered by two so that a good share of the
+    activations lies in 128..255 and some saturate at 255; couplings mix the formats (both layers
+    unsigned; only the first; a clip at 200; unsigned with biases too large to fold; unsigned with
+    per-channel shifts)."""
+    model = S.make_model(29, 3, 32, 32, [True, True, True], 5, 56, prune=(0.5, 0.9), act_hi=255)
+    for lv in model["levels"]:
+        for ci, cp in enumerate(lv["couplings"]):
+            for li in range(2):
+                ly = cp["layers"][li]
+                ly["s"][:] = np.maximum(ly["s"] - 2, 1)
+            if ci == 1:
+                cp["layers"][1]["clamp"] = (0, 127)
+                cp["layers"][1]["s"][:] += 2
+            elif ci == 2:
+                cp["layers"][0]["clamp"] = (0, 200)
+                cp["layers"][1]["clamp"] = (3, 255)
+            elif ci == 3:
+                cp["layers"][0]["bias"][::2] = 1 << 20
+                cp["layers"][1]["bias"][1::2] = -(1 << 19)
+            elif ci == 4:
+                cp["layers"][0]["s"][::2] += 1
+    x = S.smooth_field_images(30, 6, 32, 32, 2.0)
+    # activations above 127 must really occur and matter: clipping at 127 instead changes z
+    import copy
+    narrow = copy.deepcopy(model)
+    for lv in narrow["levels"]:
+        for cp in lv["couplings"]:
+            for li in range(2):
+                lo, hi = cp["layers"][li]["clamp"]
+                cp["layers"][li]["clamp"] = (lo, min(hi, 127))
+    assert not np.array_equal(O.forward(O.Packed(model), x[:1])[0], O.forward(O.Packed(narrow), x[:1])[0])
+    _check_both_ways(G, model, x)
+
+
 def test_zero_bias_and_no_prior(G):
     model = S.make_model(19, 3, 16, 16, [True, False], 2, 16, prune=None, prior=False, with_bias=False)
     _check_both_ways(G, model, S.smooth_field_images(20, 4, 16, 16, 1.5))
