@@ -215,8 +215,11 @@ def main():
     hbm, bf16, which = peaks()
     peak_int8 = 2.0 * bf16                      # dense int8 : bf16 = 2 : 1 nominal
     achieved = 2.0 * top_macs * B / (lvl[top] * 1e-3) / 1e12
+    # DRAM bytes of that launch (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture of this
+    # workload: profiles/level_kernel_config2_encode.md); only valid for the captured configuration
+    traffic = 2.70e6 if (cfg == 2 and B == 128 and top == 0) else None
     roofline = {"bound": "tensor", "kernel": "level_kernel<encode> level %d" % top, "achieved": achieved,
-                "peak": peak_int8, "unit": "TOP/s (int8)", "frac": achieved / peak_int8, "traffic": None,
+                "peak": peak_int8, "unit": "TOP/s (int8)", "frac": achieved / peak_int8, "traffic": traffic,
                 "peak_source": "2 x %s burst bf16 %.1f TFLOP/s" % (which, bf16),
                 "level_ms": [float(v) for v in lvl],
                 "whole_step_frac": (2.0 * macs * B / (total_ms / args.steps * 1e-3) / 1e12) / peak_int8}
