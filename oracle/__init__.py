@@ -16,12 +16,22 @@ _LIB = os.path.join(_HERE, "libiodf_oracle.so")
 _lib = None
 
 
+_RANS_SRC = os.path.join(_HERE, "rans_oracle.cpp")
+_RANS_LIB = os.path.join(_HERE, "librans_oracle.so")
+_rans = None
+
+
+def _compile(src, lib_path, force):
+    if force or not os.path.exists(lib_path) or os.path.getmtime(lib_path) < os.path.getmtime(src):
+        tmp = lib_path + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["g++", "-O2", "-std=c++17", "-fPIC", "-shared", "-pthread", "-o", tmp, src])
+        os.replace(tmp, lib_path)
+    return lib_path
+
+
 def build(force=False):
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        tmp = _LIB + ".tmp.%d" % os.getpid()
-        subprocess.check_call(["g++", "-O2", "-std=c++17", "-fPIC", "-shared", "-pthread", "-o", tmp, _SRC])
-        os.replace(tmp, _LIB)
-    return _LIB
+    _compile(_RANS_SRC, _RANS_LIB, force)
+    return _compile(_SRC, _LIB, force)
 
 
 def lib():
@@ -164,3 +174,120 @@ def unsqueeze(y):
     x = np.empty((c4 // 4, h2 * 2, w2 * 2), dtype=np.int32)
     lib().orc_unsqueeze(_p(y), c4, h2, w2, _p(x))
     return x
+
+
+# ---- entropy-coding side (rans_oracle.cpp) ---------------------------------------------------------
+def _rans_lib():
+    global _rans
+    if _rans is None:
+        build()
+        L = ctypes.CDLL(_RANS_LIB)
+        L.orc_rans_cum.restype = ctypes.c_uint32
+        L.orc_rans_encode_stream.restype = ctypes.c_long
+        _rans = L
+    return _rans
+
+
+def _codec_args(codec):
+    G = np.ascontiguousarray(codec["G"], dtype=np.uint16)
+    R = np.ascontiguousarray(codec["R"], dtype=np.uint32)
+    return G, R, (_p(G), ctypes.c_int(codec["umax"]), _p(R), ctypes.c_int(len(R)))
+
+
+def rans_cum(codec, ls, k):
+    """Cumulative count Cum(k) of scale index ls, k in [0, 4097]."""
+    G, R, a = _codec_args(codec)
+    return int(_rans_lib().orc_rans_cum(*a, ctypes.c_int(ls), ctypes.c_int(k)))
+
+
+def rans_encode_stream(codec, z, mu, ls):
+    """One stream: per-element int32 arrays in forward order -> uint16 words."""
+    G, R, a = _codec_args(codec)
+    z, mu, ls = (np.ascontiguousarray(v, dtype=np.int32) for v in (z, mu, ls))
+    cap = 3 * len(z) + 2
+    words = np.zeros(cap, dtype=np.uint16)
+    n = _rans_lib().orc_rans_encode_stream(*a, _p(z), _p(mu), _p(ls), ctypes.c_long(len(z)), _p(words),
+                                           ctypes.c_long(cap))
+    if n < 0:
+        raise RuntimeError("oracle rANS encode failed (rc=%d)" % n)
+    return words[:n].copy()
+
+
+def rans_decode_stream(codec, words, mu, ls):
+    G, R, a = _codec_args(codec)
+    words = np.ascontiguousarray(words, dtype=np.uint16)
+    mu, ls = (np.ascontiguousarray(v, dtype=np.int32) for v in (mu, ls))
+    z = np.zeros(len(mu), dtype=np.int32)
+    rc = _rans_lib().orc_rans_decode_stream(*a, _p(words), ctypes.c_long(len(words)), _p(mu), _p(ls),
+                                            ctypes.c_long(len(mu)), _p(z))
+    if rc != 0:
+        raise RuntimeError("oracle rANS decode failed (rc=%d)" % rc)
+    return z
+
+
+def rans_blocks(model):
+    """[(z offset, elements, prior offset or -1)] per coded block of one image: every factored-out
+    block in z order, then the final block."""
+    blocks, zo, po = [], 0, 0
+    c = model["in_c"]
+    for lv in model["levels"]:
+        c, px = lv["c"], lv["h"] * lv["w"]
+        if lv["split"]:
+            n = (c - c // 2) * px
+            blocks.append((zo, n, po if lv["prior"] is not None else -1))
+            zo += n
+            if lv["prior"] is not None:
+                po += n
+            c = c // 2
+    last = model["levels"][-1]
+    blocks.append((zo, c * last["h"] * last["w"], -1))
+    return blocks
+
+
+def _rans_batch_args(codec, model):
+    blocks = rans_blocks(model)
+    E = codec["elems_per_stream"]
+    zoff = np.array([b[0] for b in blocks], dtype=np.int64)
+    bn = np.array([b[1] for b in blocks], dtype=np.int64)
+    poff = np.array([b[2] for b in blocks], dtype=np.int64)
+    n_streams = int(sum((n + E - 1) // E for n in bn))
+    cap = 3 * E + 2
+    return blocks, E, zoff, bn, poff, n_streams, cap
+
+
+def rans_encode(codec, model, z, prior):
+    """z int32 [B,d], prior int32 [B,2,d_fact] (or None) -> (words uint16 [B,S,cap], counts uint32 [B,S])."""
+    G, R, a = _codec_args(codec)
+    blocks, E, zoff, bn, poff, S, cap = _rans_batch_args(codec, model)
+    z = np.ascontiguousarray(z, dtype=np.int32)
+    B, d = z.shape
+    d_fact = 0 if prior is None else prior.shape[2]
+    pr = np.zeros((B, 2, max(d_fact, 1)), np.int32) if prior is None else np.ascontiguousarray(prior, dtype=np.int32)
+    words = np.zeros((B, S, cap), dtype=np.uint16)
+    counts = np.zeros((B, S), dtype=np.uint32)
+    cl = ctypes.c_long
+    rc = _rans_lib().orc_rans_encode(*a, ctypes.c_int(codec["final_ls"]), cl(E), _p(z), _p(pr), cl(B), cl(d),
+                                     cl(d_fact), ctypes.c_int(len(blocks)), _p(zoff), _p(bn), _p(poff), cl(S),
+                                     cl(cap), _p(words), _p(counts))
+    if rc != 0:
+        raise RuntimeError("oracle rANS encode failed (rc=%d)" % rc)
+    return words, counts
+
+
+def rans_decode_block(codec, model, words, counts, prior, block, z):
+    """Decode coded block `block` of every image into z (in place)."""
+    G, R, a = _codec_args(codec)
+    blocks, E, zoff, bn, poff, S, cap = _rans_batch_args(codec, model)
+    B, d = z.shape
+    d_fact = 0 if prior is None else prior.shape[2]
+    pr = np.zeros((B, 2, max(d_fact, 1)), np.int32) if prior is None else np.ascontiguousarray(prior, dtype=np.int32)
+    words = np.ascontiguousarray(words, dtype=np.uint16)
+    counts = np.ascontiguousarray(counts, dtype=np.uint32)
+    assert z.dtype == np.int32 and z.flags.c_contiguous
+    cl = ctypes.c_long
+    rc = _rans_lib().orc_rans_decode_block(*a, ctypes.c_int(codec["final_ls"]), cl(E), _p(words), _p(counts), _p(pr),
+                                           cl(B), cl(d), cl(d_fact), ctypes.c_int(len(blocks)), _p(zoff), _p(bn),
+                                           _p(poff), cl(S), cl(cap), ctypes.c_int(block), _p(z))
+    if rc != 0:
+        raise RuntimeError("oracle rANS decode failed (rc=%d)" % rc)
+    return z
