@@ -45,7 +45,8 @@ typedef enum {
   IODF_ETIMEOUT = -5,     /* a bounded device-side wait gave up (reported by iodf_check)             */
   IODF_EUNSUPPORTED = -6, /* a valid model whose shape this build cannot run (see iodf_create)       */
   IODF_EOVERFLOW = -7,    /* a worst-case accumulator |sum| + |bias| would leave the int32 range     */
-  IODF_ELIMIT = -8        /* the request needs more than the fixed scratch of iodf_forward_static   */
+  IODF_ELIMIT = -8,       /* the request needs more than the fixed scratch of iodf_forward_static   */
+  IODF_EDATA = -9         /* entropy coder: a scale index outside the table or a malformed stream   */
 } iodf_status;
 
 /*
@@ -195,6 +196,72 @@ int iodf_forward_patches(iodf_model* m, const uint8_t* image_u8, int H, int W, i
                          void* cuda_stream);
 int iodf_inverse_patches(iodf_model* m, const int32_t* z, int H, int W, uint8_t* image_u8, int32_t* prior,
                          uint32_t* out_of_range_count, void* cuda_stream);
+
+/*
+ * Entropy coding of the latents on the GPU (Sec. 3: factorised discrete logistic prior; App. A:
+ * range-ANS; Sec. 5.3 leaves "an optimized GPU implementation of rANS" as future work).
+ *
+ * The prior's integer form is given by the caller (HOST arrays, copied):
+ *   sigmoid_table[u + umax], u in [-umax, umax]: a non-decreasing table of M' sigma(u / 64), M' =
+ *     2^16 - 4097, entries <= M';
+ *   inv_scale[ls] = 2^21 / s_ls for scale index ls in [0, n_scales) (the prior head's log-scale index);
+ *   final_ls: the fixed scale index (with mu = 0) of blocks that have no prior head, the final block
+ *     among them.
+ * An element with prior (mu, ls) is coded as the symbol k = clamp(z - mu, -2048, 2048) + 2048 with
+ *   Cum(k) = k + sigmoid_table[clamp(floor((2 (k - 2048) - 1) inv_scale[ls] / 2^16), -umax, umax) + umax],
+ *   Cum(0) = 0, Cum(4097) = 2^16; k = 0 and k = 4096 are escapes followed by the 32 bits of z.
+ * rANS: total mass M = 2^16, 32-bit state kept in [2^16, 2^32), 16-bit words; App. A's update
+ * X' = floor(X / F) M + C + X mod F and its inverse.
+ *
+ * Container. Per image the coded blocks are every factored-out block in z order and then the final
+ * block (a decoder needs a block's symbols before it can compute the next block's prior). Block q
+ * of n elements is cut into ceil(n / elems_per_stream) streams; stream j holds elements j, j + ns, ...
+ * words is DEV uint16 [B][n_streams][words_per_stream] and counts DEV uint32 [B][n_streams]; stream s
+ * of image b occupies words[b][s][0 .. counts[b][s]) (emitted words, then the final state, low half
+ * first); the compressed size of an image is 2 * sum of its counts bytes. iodf_codec_get_layout gives
+ * the numbers. words_per_stream = 3 * elems_per_stream + 2 is the worst case.
+ *
+ * iodf_rans_encode codes every block of z [B][d] with prior [B][2][d_fact] (as written by
+ * iodf_forward). iodf_rans_decode_block decodes one block of every image into z (the rest of z is
+ * untouched); with iodf_inverse_level the decode order is: final block, then for level = deepest
+ * .. 0: IODF_LEVEL_PRIOR, iodf_rans_decode_block(block of that level), IODF_LEVEL_COUPLINGS.
+ * Both enqueue one kernel on `cuda_stream` and allocate nothing. A scale index outside
+ * [0, n_scales) or a stream whose words do not end where they should is counted on the device and
+ * reported by iodf_codec_check (IODF_EDATA), never dereferenced.
+ */
+typedef struct {
+  uint32_t abi_version;              /* IODF_ABI_VERSION                                             */
+  const uint16_t* sigmoid_table;     /* HOST, 2 * umax + 1 entries                                   */
+  uint32_t umax;
+  const uint32_t* inv_scale;         /* HOST, n_scales entries                                       */
+  uint32_t n_scales;
+  int32_t final_ls;
+  uint32_t elems_per_stream;
+} iodf_codec_desc;
+
+typedef struct {
+  uint32_t n_blocks;                                  /* coded blocks per image                      */
+  uint32_t n_streams;                                 /* streams per image                           */
+  uint32_t words_per_stream;                          /* container stride, in 16-bit words           */
+  int32_t block_level[IODF_MAX_LEVELS + 1];           /* flow level of the block, -1: final block    */
+  uint64_t block_z_off[IODF_MAX_LEVELS + 1];
+  uint64_t block_elems[IODF_MAX_LEVELS + 1];
+  uint32_t block_first_stream[IODF_MAX_LEVELS + 1];
+  uint32_t block_streams[IODF_MAX_LEVELS + 1];
+} iodf_codec_layout;
+
+typedef struct iodf_codec iodf_codec;
+
+int iodf_codec_create(const iodf_model* m, const iodf_codec_desc* desc, iodf_codec** out);
+void iodf_codec_destroy(iodf_codec* c);
+int iodf_codec_get_layout(const iodf_codec* c, iodf_codec_layout* out);
+int iodf_rans_encode(iodf_codec* c, const int32_t* z, const int32_t* prior, int B, uint16_t* words, uint32_t* counts,
+                     void* cuda_stream);
+int iodf_rans_decode_block(iodf_codec* c, int block, const uint16_t* words, const uint32_t* counts,
+                           const int32_t* prior, int B, int32_t* z, void* cuda_stream);
+/* Synchronise the stream; IODF_EDATA if any stream was flagged since the last check (their number
+ * in *bad_streams, HOST, may be NULL). */
+int iodf_codec_check(iodf_codec* c, void* cuda_stream, uint32_t* bad_streams);
 
 /*
  * The same two operations for HOST buffers (pinned memory recommended): inputs are copied to a

@@ -13,6 +13,8 @@ IODF_MAX_LEVELS = 8
 
 DECLARED_SYMBOLS = ["iodf_create", "iodf_destroy", "iodf_get_layout", "iodf_forward", "iodf_inverse",
                     "iodf_inverse_level", "iodf_forward_patches", "iodf_inverse_patches",
+                    "iodf_codec_create", "iodf_codec_destroy", "iodf_codec_get_layout", "iodf_rans_encode",
+                    "iodf_rans_decode_block", "iodf_codec_check",
                     "iodf_forward_host", "iodf_inverse_host", "iodf_forward_timed", "iodf_inverse_timed", "iodf_forward_static",
                     "iodf_static_scratch_bytes_per_image", "iodf_check", "iodf_launches_per_call",
                     "iodf_strerror", "iodf_last_cuda_error"]
@@ -46,6 +48,20 @@ class Layout(C.Structure):
                 ("level_w", C.c_uint32 * IODF_MAX_LEVELS), ("z_off", C.c_uint64 * IODF_MAX_LEVELS),
                 ("prior_off", C.c_uint64 * IODF_MAX_LEVELS), ("z_final_off", C.c_uint64),
                 ("macs_per_image", C.c_uint64)]
+
+
+class CodecDesc(C.Structure):
+    _fields_ = [("abi_version", C.c_uint32), ("sigmoid_table", C.c_void_p), ("umax", C.c_uint32),
+                ("inv_scale", C.c_void_p), ("n_scales", C.c_uint32), ("final_ls", C.c_int32),
+                ("elems_per_stream", C.c_uint32)]
+
+
+class CodecLayout(C.Structure):
+    _fields_ = [("n_blocks", C.c_uint32), ("n_streams", C.c_uint32), ("words_per_stream", C.c_uint32),
+                ("block_level", C.c_int32 * (IODF_MAX_LEVELS + 1)), ("block_z_off", C.c_uint64 * (IODF_MAX_LEVELS + 1)),
+                ("block_elems", C.c_uint64 * (IODF_MAX_LEVELS + 1)),
+                ("block_first_stream", C.c_uint32 * (IODF_MAX_LEVELS + 1)),
+                ("block_streams", C.c_uint32 * (IODF_MAX_LEVELS + 1))]
 
 
 class IodfError(RuntimeError):
@@ -84,6 +100,18 @@ def load_library(path=None):
     L.iodf_forward_patches.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp, vp]
     L.iodf_inverse_patches.restype = C.c_int
     L.iodf_inverse_patches.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp, vp, vp]
+    L.iodf_codec_create.restype = C.c_int
+    L.iodf_codec_create.argtypes = [vp, C.POINTER(CodecDesc), C.POINTER(vp)]
+    L.iodf_codec_destroy.restype = None
+    L.iodf_codec_destroy.argtypes = [vp]
+    L.iodf_codec_get_layout.restype = C.c_int
+    L.iodf_codec_get_layout.argtypes = [vp, C.POINTER(CodecLayout)]
+    L.iodf_rans_encode.restype = C.c_int
+    L.iodf_rans_encode.argtypes = [vp, vp, vp, C.c_int, vp, vp, vp]
+    L.iodf_rans_decode_block.restype = C.c_int
+    L.iodf_rans_decode_block.argtypes = [vp, C.c_int, vp, vp, vp, C.c_int, vp, vp]
+    L.iodf_codec_check.restype = C.c_int
+    L.iodf_codec_check.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
     L.iodf_forward_host.restype = C.c_int
     L.iodf_forward_host.argtypes = [vp, vp, C.c_int, vp, vp, vp]
     L.iodf_inverse_host.restype = C.c_int
@@ -275,6 +303,64 @@ def iodf_inverse_patches(model, z, H, W, image_u8=None, prior=None, out_of_range
     if rc != 0:
         raise IodfError(rc, "iodf_inverse_patches")
     return image_u8
+
+
+class Codec:
+    """Handle of an iodf_codec; destroyed when garbage collected."""
+
+    def __init__(self, handle, layout, model):
+        self.handle, self.layout, self.model = handle, layout, model
+        self.n_blocks, self.n_streams = int(layout.n_blocks), int(layout.n_streams)
+        self.words_per_stream = int(layout.words_per_stream)
+
+    def __del__(self):
+        h, self.handle = getattr(self, "handle", None), None
+        if h and _lib is not None:
+            _lib.iodf_codec_destroy(h)
+
+
+def iodf_codec_create(model, codec):
+    """codec: dict with the tables G (uint16), R (uint32), umax, final_ls, elems_per_stream."""
+    L = load_library()
+    G = np.ascontiguousarray(codec["G"], dtype=np.uint16)
+    R = np.ascontiguousarray(codec["R"], dtype=np.uint32)
+    desc = CodecDesc(IODF_ABI_VERSION, G.ctypes.data, int(codec["umax"]), R.ctypes.data, len(R),
+                     int(codec["final_ls"]), int(codec["elems_per_stream"]))
+    out = C.c_void_p()
+    rc = L.iodf_codec_create(model.handle, C.byref(desc), C.byref(out))
+    if rc != 0:
+        raise IodfError(rc, "iodf_codec_create")
+    lay = CodecLayout()
+    L.iodf_codec_get_layout(out, C.byref(lay))
+    return Codec(out, lay, model)
+
+
+def iodf_rans_encode(codec, z, prior, words=None, counts=None, stream=None):
+    """z cuda int32 [B,d], prior cuda int32 [B,2,d_fact] -> (words uint16 [B,S,cap], counts uint32-as-int32 [B,S])."""
+    import torch
+    B = z.shape[0]
+    if words is None:
+        words = torch.empty((B, codec.n_streams, codec.words_per_stream), dtype=torch.int16, device=z.device)
+    if counts is None:
+        counts = torch.empty((B, codec.n_streams), dtype=torch.int32, device=z.device)
+    rc = load_library().iodf_rans_encode(codec.handle, _ptr(z), _ptr(prior), B, _ptr(words), _ptr(counts), _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_rans_encode")
+    return words, counts
+
+
+def iodf_rans_decode_block(codec, block, words, counts, prior, z, stream=None):
+    rc = load_library().iodf_rans_decode_block(codec.handle, int(block), _ptr(words), _ptr(counts), _ptr(prior),
+                                               z.shape[0], _ptr(z), _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_rans_decode_block")
+
+
+def iodf_codec_check(codec, stream=None):
+    n = C.c_uint32(0)
+    rc = load_library().iodf_codec_check(codec.handle, _stream(stream), C.byref(n))
+    if rc != 0:
+        raise IodfError(rc, "iodf_codec_check (%d streams)" % n.value)
 
 
 def iodf_forward_host(model, x_u8, z, prior=None, stream=None):

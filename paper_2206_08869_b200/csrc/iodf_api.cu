@@ -12,6 +12,7 @@
 
 #include "../../include/iodf.h"
 #include "iodf_dev.h"
+#include "rans_kernel.h"
 #include "level_kernel.h"
 
 using namespace iodf;
@@ -46,6 +47,17 @@ struct iodf_model {
   uint8_t* d_x = nullptr;
   int32_t* d_z = nullptr;
   int32_t* d_prior = nullptr;
+};
+
+struct iodf_codec {
+  int device = 0;
+  int last_cuda = 0;
+  uint32_t max_batch = 0;
+  uint32_t elems_per_stream = 0;
+  uint8_t* d_tables = nullptr;      // R then G
+  uint32_t* d_errors = nullptr;
+  iodf::RansArgs args{};
+  iodf_codec_layout layout{};
 };
 
 namespace {
@@ -854,6 +866,130 @@ int iodf_inverse_patches(iodf_model* m, const int32_t* z, int H, int W, uint8_t*
                      (cudaStream_t)cuda_stream, false, g);
 }
 
+// ---- entropy coding ---------------------------------------------------------------------------------
+#define CUC(c, x)                                                      \
+  do {                                                                 \
+    cudaError_t e__ = (x);                                             \
+    if (e__ != cudaSuccess) {                                          \
+      (c)->last_cuda = (int)e__;                                       \
+      return e__ == cudaErrorMemoryAllocation ? IODF_ENOMEM : IODF_ECUDA; \
+    }                                                                  \
+  } while (0)
+
+int iodf_codec_create(const iodf_model* m, const iodf_codec_desc* desc, iodf_codec** out) {
+  if (!m || !desc || !out) return IODF_EINVAL;
+  *out = nullptr;
+  if (desc->abi_version != IODF_ABI_VERSION) return IODF_EVERSION;
+  if (!desc->sigmoid_table || !desc->inv_scale || desc->umax < 1 || desc->umax > 16384 || desc->n_scales < 1 ||
+      desc->n_scales > 1024 || desc->elems_per_stream < 1 || desc->elems_per_stream > 65536)
+    return IODF_EINVAL;
+  if (desc->final_ls < 0 || desc->final_ls >= (int32_t)desc->n_scales) return IODF_EINVAL;
+  const uint32_t top = (1u << 16) - (2u * 2048u + 1u);
+  for (uint32_t i = 0; i < 2 * desc->umax + 1; ++i) {
+    if (desc->sigmoid_table[i] > top) return IODF_EINVAL;
+    if (i && desc->sigmoid_table[i] < desc->sigmoid_table[i - 1]) return IODF_EINVAL;   // must not decrease
+  }
+  for (uint32_t i = 0; i < desc->n_scales; ++i)
+    if (desc->inv_scale[i] < 1) return IODF_EINVAL;
+  iodf_codec* c = new (std::nothrow) iodf_codec();
+  if (!c) return IODF_ENOMEM;
+  c->device = m->device;
+  c->max_batch = m->max_batch;
+  c->elems_per_stream = desc->elems_per_stream;
+  RansArgs& a = c->args;
+  a.umax = (int)desc->umax; a.n_scales = (int)desc->n_scales; a.final_ls = desc->final_ls;
+  a.d = (long long)m->layout.d; a.d_fact = (long long)m->layout.d_fact;
+  a.cap = (int)(3 * desc->elems_per_stream + 2);
+  // coded blocks: every factored-out block in z order, then the final block
+  int nb = 0, first = 0;
+  const uint32_t E = desc->elems_per_stream;
+  auto add_block = [&](uint64_t z_off, uint64_t n, long long prior_off) {
+    RansBlock& b = a.blocks[nb];
+    b.z_off = (long long)z_off; b.n = (long long)n; b.prior_off = prior_off;
+    b.first_stream = first; b.n_streams = (int)((n + E - 1) / E);
+    c->layout.block_z_off[nb] = z_off; c->layout.block_elems[nb] = n;
+    c->layout.block_first_stream[nb] = (uint32_t)first; c->layout.block_streams[nb] = (uint32_t)b.n_streams;
+    c->layout.block_level[nb] = -1;
+    first += b.n_streams;
+    ++nb;
+  };
+  for (size_t li = 0; li < m->levels.size(); ++li) {
+    const LevelPlan& P = m->levels[li].plan;
+    if (!P.split) continue;
+    // the scale indices a prior head can emit must be table entries
+    add_block(P.z_off, (uint64_t)P.cb * P.px, P.has_prior ? (long long)P.prior_off : -1);
+    c->layout.block_level[nb - 1] = (int32_t)li;
+  }
+  add_block(m->layout.z_final_off, m->layout.d - m->layout.z_final_off, -1);
+  a.n_blocks = nb; a.n_streams = first;
+  c->layout.n_blocks = (uint32_t)nb; c->layout.n_streams = (uint32_t)first; c->layout.words_per_stream = (uint32_t)a.cap;
+  int prev = -1;
+  CUC(c, cudaGetDevice(&prev));
+  CUC(c, cudaSetDevice(c->device));
+  const size_t rbytes = 4 * (size_t)desc->n_scales, gbytes = 2 * (size_t)(2 * desc->umax + 1);
+  cudaError_t e = cudaMalloc(&c->d_tables, rbytes + gbytes);
+  if (e == cudaSuccess) e = cudaMemcpy(c->d_tables, desc->inv_scale, rbytes, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(c->d_tables + rbytes, desc->sigmoid_table, gbytes, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMalloc(&c->d_errors, sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMemset(c->d_errors, 0, sizeof(uint32_t));
+  cudaSetDevice(prev);
+  if (e != cudaSuccess) {
+    const int rc = e == cudaErrorMemoryAllocation ? IODF_ENOMEM : IODF_ECUDA;
+    iodf_codec_destroy(c);
+    return rc;
+  }
+  a.R = reinterpret_cast<const uint32_t*>(c->d_tables);
+  a.G = reinterpret_cast<const uint16_t*>(c->d_tables + rbytes);
+  a.errors = c->d_errors;
+  *out = c;
+  return IODF_OK;
+}
+
+void iodf_codec_destroy(iodf_codec* c) {
+  if (!c) return;
+  cudaSetDevice(c->device);
+  if (c->d_tables) cudaFree(c->d_tables);
+  if (c->d_errors) cudaFree(c->d_errors);
+  delete c;
+}
+
+int iodf_codec_get_layout(const iodf_codec* c, iodf_codec_layout* out) {
+  if (!c || !out) return IODF_EINVAL;
+  *out = c->layout;
+  return IODF_OK;
+}
+
+int iodf_rans_encode(iodf_codec* c, const int32_t* z, const int32_t* prior, int B, uint16_t* words, uint32_t* counts,
+                     void* cuda_stream) {
+  if (!c || !z || !words || !counts || B < 1 || (uint32_t)B > c->max_batch) return IODF_EINVAL;
+  if (c->args.d_fact && !prior) return IODF_EINVAL;
+  RansArgs a = c->args;
+  a.batch = B;
+  CUC(c, launch_rans_encode(a, z, prior, words, counts, (cudaStream_t)cuda_stream));
+  return IODF_OK;
+}
+
+int iodf_rans_decode_block(iodf_codec* c, int block, const uint16_t* words, const uint32_t* counts,
+                           const int32_t* prior, int B, int32_t* z, void* cuda_stream) {
+  if (!c || !z || !words || !counts || B < 1 || (uint32_t)B > c->max_batch) return IODF_EINVAL;
+  if (block < 0 || block >= c->args.n_blocks) return IODF_EINVAL;
+  if (c->args.blocks[block].prior_off >= 0 && !prior) return IODF_EINVAL;
+  RansArgs a = c->args;
+  a.batch = B;
+  CUC(c, launch_rans_decode(a, block, words, counts, prior, z, (cudaStream_t)cuda_stream));
+  return IODF_OK;
+}
+
+int iodf_codec_check(iodf_codec* c, void* cuda_stream, uint32_t* bad_streams) {
+  if (!c) return IODF_EINVAL;
+  uint32_t n = 0;
+  CUC(c, cudaMemcpyAsync(&n, c->d_errors, sizeof(n), cudaMemcpyDeviceToHost, (cudaStream_t)cuda_stream));
+  CUC(c, cudaStreamSynchronize((cudaStream_t)cuda_stream));
+  if (n) CUC(c, cudaMemsetAsync(c->d_errors, 0, sizeof(n), (cudaStream_t)cuda_stream));
+  if (bad_streams) *bad_streams = n;
+  return n ? IODF_EDATA : IODF_OK;
+}
+
 int iodf_forward_timed(iodf_model* m, const uint8_t* x_u8, int B, int32_t* z, int32_t* prior, void* cuda_stream,
                        float* level_ms) {
   if (!m || !x_u8 || !z || !level_ms || B < 1 || (uint32_t)B > m->max_batch) return IODF_EINVAL;
@@ -926,6 +1062,7 @@ const char* iodf_strerror(int status) {
     case IODF_EUNSUPPORTED: return "model shape not supported by this build";
     case IODF_EOVERFLOW: return "worst-case accumulator leaves the int32 range";
     case IODF_ELIMIT: return "request exceeds the fixed scratch of iodf_forward_static";
+    case IODF_EDATA: return "entropy coder: scale index outside the table or malformed stream";
     default: return "unknown status";
   }
 }

@@ -1,0 +1,188 @@
+// Entropy coding of the flow's latents on the GPU: the discrete logistic prior of Sec. 3 in integer
+// table form and range-ANS (App. A) with a 32-bit state renormalised in 16-bit words, one thread
+// per stream. The streams are independent (an image's coded blocks are cut into streams of about
+// `elems_per_stream` interleaved elements), so a batch of 128 ImageNet64-sized latents is 6 144
+// streams: the paper's "optimized GPU implementation of rANS" left as future work (Sec. 5.3).
+//
+//   symbol of an element   k = clamp(z - mu, -2048, 2048) + 2048          (0 and 4096: escapes, then
+//                                                                          z follows as 2 x 16 raw bits)
+//   cumulative counts      Cum(k) = k + G[clamp(floor((2(k-2048)-1) R[ls] / 2^16), -umax, umax) + umax]
+//                          Cum(0) = 0, Cum(4097) = M = 2^16
+//   encode step            if x >= F * 2^16: move the low 16 bits of x out;  x = (x / F) * M + (x mod F) + C
+//   decode step            slot = x mod M; k: Cum(k) <= slot < Cum(k+1);  x = F * (x / M) + slot - C;
+//                          if x < 2^16: x = x * 2^16 + next word
+//
+// The encoder walks a stream's elements last to first and appends words, then the state (low half,
+// high half); the decoder starts at the end of the words and walks back, producing the elements
+// first to last. Consecutive threads own consecutive streams of a block, whose i-th elements are
+// consecutive in memory: the loads of z and of the prior parameters are coalesced.
+#include "rans_kernel.h"
+
+namespace iodf {
+
+namespace {
+
+constexpr int kWin = 2048;
+constexpr uint32_t kM = 1u << 16;
+constexpr int kThreadsPerBlock = 128;
+
+struct Tables {
+  const uint16_t* G;       // shared memory
+  const uint32_t* R;       // shared memory
+  int umax, n_scales;
+};
+
+__device__ __forceinline__ uint32_t cum(const Tables& t, int ls, int k) {
+  if (k <= 0) return 0u;
+  if (k >= 2 * kWin + 1) return kM;
+  const long long edge2 = 2ll * (k - kWin) - 1;
+  long long u = (edge2 * (long long)t.R[ls]) >> 16;          // arithmetic shift: floor
+  u = u < -t.umax ? -t.umax : (u > t.umax ? t.umax : u);
+  return (uint32_t)k + t.G[(int)u + t.umax];
+}
+
+__device__ __forceinline__ void load_tables(const RansArgs& a, uint16_t* sG, uint32_t* sR) {
+  for (int i = threadIdx.x; i < 2 * a.umax + 1; i += blockDim.x) sG[i] = a.G[i];
+  for (int i = threadIdx.x; i < a.n_scales; i += blockDim.x) sR[i] = a.R[i];
+  __syncthreads();
+}
+
+// the element's prior parameters; a block without a prior head has mu = 0 and the fixed scale index
+__device__ __forceinline__ void prior_of(const RansArgs& a, const RansBlock& blk, const int32_t* prior_img, long e,
+                                         int32_t* mu, int* ls, uint32_t* bad) {
+  if (blk.prior_off < 0) { *mu = 0; *ls = a.final_ls; return; }
+  *mu = prior_img[blk.prior_off + e];
+  int l = prior_img[a.d_fact + blk.prior_off + e];
+  if (l < 0 || l >= a.n_scales) { *bad = 1u; l = l < 0 ? 0 : a.n_scales - 1; }
+  *ls = l;
+}
+
+__global__ void __launch_bounds__(kThreadsPerBlock) rans_encode_kernel(const RansArgs a, const int32_t* __restrict__ z,
+                                                                       const int32_t* __restrict__ prior,
+                                                                       uint16_t* __restrict__ words,
+                                                                       uint32_t* __restrict__ counts) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  uint32_t* sR = reinterpret_cast<uint32_t*>(smem);
+  uint16_t* sG = reinterpret_cast<uint16_t*>(smem + 4 * a.n_scales);
+  load_tables(a, sG, sR);
+  const Tables t{sG, sR, a.umax, a.n_scales};
+  const long gid = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= (long)a.batch * a.n_streams) return;
+  const int b = (int)(gid / a.n_streams), s = (int)(gid - (long)b * a.n_streams);
+  int q = 0;
+  while (q + 1 < a.n_blocks && s >= a.blocks[q + 1].first_stream) ++q;
+  const RansBlock blk = a.blocks[q];
+  const int j = s - blk.first_stream, ns = blk.n_streams;
+  const long n_el = (blk.n - j + ns - 1) / ns;
+  const int32_t* zb = z + (long)b * a.d + blk.z_off;
+  const int32_t* pb = prior + (long)b * 2 * a.d_fact;
+  uint16_t* out = words + gid * a.cap;
+  uint32_t pos = 0, x = 1u << 16, bad = 0;
+  auto push = [&](uint32_t F, uint32_t C) {
+    if ((unsigned long long)x >= ((unsigned long long)F << 16)) {
+      out[pos++] = (uint16_t)(x & 0xFFFFu);
+      x >>= 16;
+    }
+    x = ((x / F) << 16) + (x % F) + C;
+  };
+  for (long i = n_el - 1; i >= 0; --i) {
+    const long e = j + i * ns;
+    const int32_t zv = zb[e];
+    int32_t mu; int ls;
+    prior_of(a, blk, pb, e, &mu, &ls, &bad);
+    long long r = (long long)zv - (long long)mu;
+    r = r < -kWin ? -kWin : (r > kWin ? kWin : r);
+    const int k = (int)r + kWin;
+    if (k == 0 || k == 2 * kWin) {
+      push(1u, (uint32_t)zv & 0xFFFFu);
+      push(1u, ((uint32_t)zv >> 16) & 0xFFFFu);
+    }
+    const uint32_t C = cum(t, ls, k), F = cum(t, ls, k + 1) - C;
+    push(F, C);
+  }
+  out[pos++] = (uint16_t)(x & 0xFFFFu);
+  out[pos++] = (uint16_t)(x >> 16);
+  counts[gid] = pos;
+  if (bad && a.errors) atomicAdd(a.errors, 1u);
+}
+
+__global__ void __launch_bounds__(kThreadsPerBlock) rans_decode_kernel(const RansArgs a, int q,
+                                                                       const uint16_t* __restrict__ words,
+                                                                       const uint32_t* __restrict__ counts,
+                                                                       const int32_t* __restrict__ prior,
+                                                                       int32_t* __restrict__ z) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  uint32_t* sR = reinterpret_cast<uint32_t*>(smem);
+  uint16_t* sG = reinterpret_cast<uint16_t*>(smem + 4 * a.n_scales);
+  load_tables(a, sG, sR);
+  const Tables t{sG, sR, a.umax, a.n_scales};
+  const RansBlock blk = a.blocks[q];
+  const long tid = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (tid >= (long)a.batch * blk.n_streams) return;
+  const int b = (int)(tid / blk.n_streams), j = (int)(tid - (long)b * blk.n_streams), ns = blk.n_streams;
+  const long sid = (long)b * a.n_streams + blk.first_stream + j;
+  const long n_el = (blk.n - j + ns - 1) / ns;
+  const uint16_t* in = words + sid * a.cap;
+  long pos = min((long)counts[sid], (long)a.cap);
+  uint32_t bad = 0;
+  auto next = [&]() -> uint32_t {               // never reads before the stream's first word
+    if (pos <= 0) { bad = 1u; return 0u; }
+    return in[--pos];
+  };
+  uint32_t x = next() << 16;
+  x |= next();
+  int32_t* zb = z + (long)b * a.d + blk.z_off;
+  const int32_t* pb = prior + (long)b * 2 * a.d_fact;
+  for (long i = 0; i < n_el; ++i) {
+    const long e = j + i * ns;
+    int32_t mu; int ls;
+    prior_of(a, blk, pb, e, &mu, &ls, &bad);
+    const uint32_t slot = x & 0xFFFFu;
+    int lo = 0, hi = 2 * kWin;                  // largest k with Cum(k) <= slot
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (cum(t, ls, mid) <= slot) lo = mid; else hi = mid - 1;
+    }
+    const int k = lo;
+    const uint32_t C = cum(t, ls, k), F = cum(t, ls, k + 1) - C;
+    x = F * (x >> 16) + slot - C;
+    if (x < (1u << 16)) x = (x << 16) | next();
+    int32_t zv;
+    if (k == 0 || k == 2 * kWin) {
+      const uint32_t h = x & 0xFFFFu;
+      x >>= 16;                                  // F = 1, C = slot: x = x / M
+      if (x < (1u << 16)) x = (x << 16) | next();
+      const uint32_t l = x & 0xFFFFu;
+      x >>= 16;
+      if (x < (1u << 16)) x = (x << 16) | next();
+      zv = (int32_t)((h << 16) | l);
+    } else {
+      zv = (int32_t)((long long)mu + (k - kWin));
+    }
+    zb[e] = zv;
+  }
+  if (pos != 0 || x != (1u << 16)) bad = 1u;     // every word used and the state back at its start
+  if (bad && a.errors) atomicAdd(a.errors, 1u);
+}
+
+}  // namespace
+
+static size_t table_smem(const RansArgs& a) { return 4 * (size_t)a.n_scales + 2 * (size_t)(2 * a.umax + 1) + 16; }
+
+cudaError_t launch_rans_encode(const RansArgs& a, const int32_t* z, const int32_t* prior, uint16_t* words,
+                               uint32_t* counts, cudaStream_t stream) {
+  const long total = (long)a.batch * a.n_streams;
+  const unsigned grid = (unsigned)((total + kThreadsPerBlock - 1) / kThreadsPerBlock);
+  rans_encode_kernel<<<grid, kThreadsPerBlock, table_smem(a), stream>>>(a, z, prior, words, counts);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rans_decode(const RansArgs& a, int block, const uint16_t* words, const uint32_t* counts,
+                               const int32_t* prior, int32_t* z, cudaStream_t stream) {
+  const long total = (long)a.batch * a.blocks[block].n_streams;
+  const unsigned grid = (unsigned)((total + kThreadsPerBlock - 1) / kThreadsPerBlock);
+  rans_decode_kernel<<<grid, kThreadsPerBlock, table_smem(a), stream>>>(a, block, words, counts, prior, z);
+  return cudaGetLastError();
+}
+
+}  // namespace iodf
