@@ -299,6 +299,54 @@ def main():
             extra["encode_patches"] = {"image": "3x%dx%d" % (py_ * hw, px_ * hw), "patches": B, "ms_per_image": ms,
                                        "value": 3.0 * py_ * hw * px_ * hw / (ms * 1e-3) / 1e6, "unit": "MB/s",
                                        "equals_batch_encode": same}
+        # entropy coding of the latents (rANS, one thread per stream) and the whole compressor /
+        # decompressor: flow + coder, latents and prior parameters never leave the GPU
+        codec = S.logistic_codec()
+        cd = G.iodf_codec_create(m, codec)
+        wbuf = [torch.empty((B, cd.n_streams, cd.words_per_stream), dtype=torch.int16, device=dev) for _ in range(2)]
+        cbuf = [torch.empty((B, cd.n_streams), dtype=torch.int32, device=dev) for _ in range(2)]
+        G.iodf_forward(m, xs[0], zs[0], ps[0])
+        enc_ms = timed(lambda i: G.iodf_rans_encode(cd, zs[0], ps[0], wbuf[i % 2], cbuf[i % 2]), dec_steps)
+        blk_of = {int(cd.layout.block_level[q]): q for q in range(cd.n_blocks - 1)}
+
+        def compress(i):
+            k = i % N_SETS
+            G.iodf_forward(m, xs[k], zs[k], ps[k])
+            G.iodf_rans_encode(cd, zs[k], ps[k], wbuf[0], cbuf[0])
+
+        def decompress(i):
+            k = 0
+            G.iodf_rans_decode_block(cd, cd.n_blocks - 1, wbuf[1], cbuf[1], ps[k], zs[k])
+            for lv in range(L - 1, -1, -1):
+                if lv in blk_of:
+                    G.iodf_inverse_level(m, lv, G.IODF_LEVEL_PRIOR, zs[k], prior=ps[k])
+                    G.iodf_rans_decode_block(cd, blk_of[lv], wbuf[1], cbuf[1], ps[k], zs[k])
+                G.iodf_inverse_level(m, lv, G.IODF_LEVEL_COUPLINGS, zs[k], x_u8=xo[k])
+        G.iodf_forward(m, xs[0], zs[0], ps[0])
+        G.iodf_rans_encode(cd, zs[0], ps[0], wbuf[1], cbuf[1])
+        coded_bytes = 2.0 * float(cbuf[1].to(torch.int64).sum().item())
+        zs[0].fill_(0x7A7A7A7A)
+        dms = timed(decompress, dec_steps)
+        rt = bool(torch.equal(xo[0], xs[0]))
+        cms = timed(compress, dec_steps)
+        G.iodf_codec_check(cd)
+        raw = float(B * m.d)
+        # the oracle's coder on a few images of the same latents, for the CPU figure beside it
+        import oracle as O
+        nz = min(B, 8)
+        zc, pc = zs[0][:nz].cpu().numpy(), ps[0][:nz].cpu().numpy()
+        G.iodf_forward(m, xs[0], zs[0], ps[0])
+        zc, pc = zs[0][:nz].cpu().numpy(), ps[0][:nz].cpu().numpy()
+        t0 = time.perf_counter()
+        O.rans_encode(codec, model, zc, pc)
+        cpu_s = time.perf_counter() - t0
+        extra["entropy_coding"] = {
+            "rans_encode_ms": enc_ms, "rans_encode_msym_per_s": B * m.d / (enc_ms * 1e-3) / 1e6,
+            "streams": B * cd.n_streams, "bits_per_dim": 8.0 * coded_bytes / raw,
+            "note": "random (untrained) weights: the bit rate says nothing about the model, only that the coder is exact",
+            "compress_ms": cms, "compress_MB_per_s": raw / (cms * 1e-3) / 1e6,
+            "decompress_ms": dms, "decompress_MB_per_s": raw / (dms * 1e-3) / 1e6, "round_trip_exact": rt,
+            "cpu_oracle_rans_msym_per_s": nz * m.d / cpu_s / 1e6}
         G.iodf_check(m)
 
     # ---- end to end through the host-buffer entry point --------------------------------------

@@ -889,8 +889,8 @@ int iodf_codec_create(const iodf_model* m, const iodf_codec_desc* desc, iodf_cod
     if (desc->sigmoid_table[i] > top) return IODF_EINVAL;
     if (i && desc->sigmoid_table[i] < desc->sigmoid_table[i - 1]) return IODF_EINVAL;   // must not decrease
   }
-  for (uint32_t i = 0; i < desc->n_scales; ++i)
-    if (desc->inv_scale[i] < 1) return IODF_EINVAL;
+  for (uint32_t i = 0; i < desc->n_scales; ++i)   // 2^21 / s with s >= 2^-9: the kernels multiply in 32 bits
+    if (desc->inv_scale[i] < 1 || desc->inv_scale[i] >= (1u << 30)) return IODF_EINVAL;
   iodf_codec* c = new (std::nothrow) iodf_codec();
   if (!c) return IODF_ENOMEM;
   c->device = m->device;

@@ -35,10 +35,13 @@ struct Tables {
 __device__ __forceinline__ uint32_t cum(const Tables& t, int ls, int k) {
   if (k <= 0) return 0u;
   if (k >= 2 * kWin + 1) return kM;
-  const long long edge2 = 2ll * (k - kWin) - 1;
-  long long u = (edge2 * (long long)t.R[ls]) >> 16;          // arithmetic shift: floor
-  u = u < -t.umax ? -t.umax : (u > t.umax ? t.umax : u);
-  return (uint32_t)k + t.G[(int)u + t.umax];
+  // floor(edge2 * R / 2^16) in 32-bit pieces: with R = Rh 2^16 + Rl it is edge2 * Rh + floor(edge2 * Rl /
+  // 2^16) exactly (|edge2| < 2^13, Rl < 2^16, Rh < 2^15 for the scales a codec accepts)
+  const int edge2 = 2 * (k - kWin) - 1;
+  const uint32_t R = t.R[ls];
+  int u = edge2 * (int)(R >> 16) + ((edge2 * (int)(R & 0xFFFFu)) >> 16);      // arithmetic shift: floor
+  u = max(-t.umax, min(t.umax, u));
+  return (uint32_t)k + t.G[u + t.umax];
 }
 
 __device__ __forceinline__ void load_tables(const RansArgs& a, uint16_t* sG, uint32_t* sR) {
@@ -106,6 +109,12 @@ __global__ void __launch_bounds__(kThreadsPerBlock) rans_encode_kernel(const Ran
   if (bad && a.errors) atomicAdd(a.errors, 1u);
 }
 
+// Decode: one WARP per stream. The state, the word pointer and every step are the same in all 32
+// lanes; only the symbol search is shared out: instead of 13 dependent bisection steps, three rounds
+// in which lane L tests one candidate k each (steps of 129, 5 and 1) and a ballot picks the largest
+// k with Cum(k) <= slot. A stream's latency, which bounds the decompressor (a block's streams are
+// few and long), drops about threefold; the redundant lanes are free because the kernel is
+// latency-bound.
 __global__ void __launch_bounds__(kThreadsPerBlock) rans_decode_kernel(const RansArgs a, int q,
                                                                        const uint16_t* __restrict__ words,
                                                                        const uint32_t* __restrict__ counts,
@@ -117,9 +126,10 @@ __global__ void __launch_bounds__(kThreadsPerBlock) rans_decode_kernel(const Ran
   load_tables(a, sG, sR);
   const Tables t{sG, sR, a.umax, a.n_scales};
   const RansBlock blk = a.blocks[q];
-  const long tid = (long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (tid >= (long)a.batch * blk.n_streams) return;
-  const int b = (int)(tid / blk.n_streams), j = (int)(tid - (long)b * blk.n_streams), ns = blk.n_streams;
+  const int lane = threadIdx.x & 31;
+  const long wid = ((long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;       // one stream per warp
+  if (wid >= (long)a.batch * blk.n_streams) return;
+  const int b = (int)(wid / blk.n_streams), j = (int)(wid - (long)b * blk.n_streams), ns = blk.n_streams;
   const long sid = (long)b * a.n_streams + blk.first_stream + j;
   const long n_el = (blk.n - j + ns - 1) / ns;
   const uint16_t* in = words + sid * a.cap;
@@ -138,12 +148,15 @@ __global__ void __launch_bounds__(kThreadsPerBlock) rans_decode_kernel(const Ran
     int32_t mu; int ls;
     prior_of(a, blk, pb, e, &mu, &ls, &bad);
     const uint32_t slot = x & 0xFFFFu;
-    int lo = 0, hi = 2 * kWin;                  // largest k with Cum(k) <= slot
-    while (lo < hi) {
-      const int mid = (lo + hi + 1) >> 1;
-      if (cum(t, ls, mid) <= slot) lo = mid; else hi = mid - 1;
+    // largest k in [0, 4096] with Cum(k) <= slot (Cum(0) = 0 <= slot always; Cum(k > 4096) = M > slot)
+    int k = 0;
+#pragma unroll
+    for (int round = 0; round < 3; ++round) {
+      const int step = round == 0 ? 129 : (round == 1 ? 5 : 1);
+      const int cand = k + lane * step;
+      const unsigned ok = __ballot_sync(0xFFFFFFFFu, cum(t, ls, cand) <= slot);   // a prefix of the lanes (Cum is monotone)
+      k += (31 - __clz((int)ok)) * step;
     }
-    const int k = lo;
     const uint32_t C = cum(t, ls, k), F = cum(t, ls, k + 1) - C;
     x = F * (x >> 16) + slot - C;
     if (x < (1u << 16)) x = (x << 16) | next();
@@ -159,10 +172,10 @@ __global__ void __launch_bounds__(kThreadsPerBlock) rans_decode_kernel(const Ran
     } else {
       zv = (int32_t)((long long)mu + (k - kWin));
     }
-    zb[e] = zv;
+    if (lane == 0) zb[e] = zv;
   }
   if (pos != 0 || x != (1u << 16)) bad = 1u;     // every word used and the state back at its start
-  if (bad && a.errors) atomicAdd(a.errors, 1u);
+  if (bad && lane == 0 && a.errors) atomicAdd(a.errors, 1u);
 }
 
 }  // namespace
@@ -179,7 +192,7 @@ cudaError_t launch_rans_encode(const RansArgs& a, const int32_t* z, const int32_
 
 cudaError_t launch_rans_decode(const RansArgs& a, int block, const uint16_t* words, const uint32_t* counts,
                                const int32_t* prior, int32_t* z, cudaStream_t stream) {
-  const long total = (long)a.batch * a.blocks[block].n_streams;
+  const long total = (long)a.batch * a.blocks[block].n_streams * 32;        // a warp per stream
   const unsigned grid = (unsigned)((total + kThreadsPerBlock - 1) / kThreadsPerBlock);
   rans_decode_kernel<<<grid, kThreadsPerBlock, table_smem(a), stream>>>(a, block, words, counts, prior, z);
   return cudaGetLastError();
