@@ -102,6 +102,31 @@ def test_escapes_and_extreme_values(G):
     np.testing.assert_array_equal(out.cpu().numpy(), z)
 
 
+def test_model_without_prior_heads(G):
+    """Every block then has the fixed prior (mu = 0, one scale index); no prior buffer is passed."""
+    import torch
+    model = S.make_model(0xAE00, 3, 16, 16, [True, True], 2, 16, prior=False)
+    codec = S.logistic_codec(elems_per_stream=50, final_ls=50)
+    x = S.smooth_field_images(0xAE01, 3, 16, 16, 2.0)
+    z_ref, p_ref = O.forward(O.Packed(model), x)
+    assert p_ref is None
+    w_ref, c_ref = O.rans_encode(codec, model, z_ref, None)
+    m = G.iodf_create(model, 3)
+    cd = G.iodf_codec_create(m, codec)
+    z, p = G.iodf_forward(m, _t(x))
+    assert p is None
+    words, counts = G.iodf_rans_encode(cd, z, None)
+    G.iodf_codec_check(cd)
+    cc = counts.cpu().numpy().view(np.uint32)
+    np.testing.assert_array_equal(cc, c_ref)
+    np.testing.assert_array_equal(_valid(words.cpu().numpy().view(np.uint16), cc), _valid(w_ref, c_ref))
+    out = torch.zeros_like(z)
+    for q in range(cd.n_blocks):
+        G.iodf_rans_decode_block(cd, q, words, counts, None, out)
+    G.iodf_codec_check(cd)
+    assert torch.equal(out, z)
+
+
 def test_bad_scale_index_and_damaged_stream_are_reported(G):
     import torch
     model = S.make_model(0xAD00, 3, 8, 8, [True], 1, 8)
