@@ -259,6 +259,37 @@ int iodf_rans_encode(iodf_codec* c, const int32_t* z, const int32_t* prior, int 
                      void* cuda_stream);
 int iodf_rans_decode_block(iodf_codec* c, int block, const uint16_t* words, const uint32_t* counts,
                            const int32_t* prior, int B, int32_t* z, void* cuda_stream);
+/*
+ * Compact byte stream of a batch (what a file or a network message would hold; little endian):
+ *   uint32 offset[B + 1]   byte offset of image b's record from the start of the payload;
+ *                          offset[B] = payload bytes
+ *   payload, per image:    uint16 count[n_streams], then the words of stream 0, 1, ... back to back
+ * iodf_rans_pack writes it from a container (packed: DEV, 4-byte aligned, at least
+ * iodf_rans_packed_capacity(c, B) bytes; the total is 4 (B + 1) + offset[B]); iodf_rans_unpack
+ * restores the container from packed_bytes bytes, checking every record against the payload size
+ * and its own counts (a bad record gets zero counts and is reported by iodf_codec_check). Both need
+ * words_per_stream <= 65535.
+ */
+size_t iodf_rans_packed_capacity(const iodf_codec* c, int B);
+int iodf_rans_pack(iodf_codec* c, const uint16_t* words, const uint32_t* counts, int B, uint8_t* packed,
+                   void* cuda_stream);
+int iodf_rans_unpack(iodf_codec* c, const uint8_t* packed, size_t packed_bytes, int B, uint16_t* words,
+                     uint32_t* counts, void* cuda_stream);
+
+/*
+ * Whole compressor and decompressor for HOST buffers (pinned memory recommended): images in, compact
+ * byte stream out, and back. The latents and prior parameters stay on the device. The first call
+ * allocates the codec's staging buffers for the model's max_batch (do it before any stream capture).
+ * iodf_compress_host synchronises the stream (the size of the byte stream is data dependent) and
+ * returns it in *out_bytes; IODF_ELIMIT if out_capacity is too small (*out_bytes then says how much
+ * is needed). iodf_decompress_host enqueues everything and returns; x_u8_host is valid after the
+ * stream has been synchronised, and iodf_codec_check / iodf_check report damaged input.
+ */
+int iodf_compress_host(iodf_model* m, iodf_codec* c, const uint8_t* x_u8_host, int B, uint8_t* out_host,
+                       size_t out_capacity, size_t* out_bytes, void* cuda_stream);
+int iodf_decompress_host(iodf_model* m, iodf_codec* c, const uint8_t* in_host, size_t in_bytes, int B,
+                         uint8_t* x_u8_host, void* cuda_stream);
+
 /* Synchronise the stream; IODF_EDATA if any stream was flagged since the last check (their number
  * in *bad_streams, HOST, may be NULL). */
 int iodf_codec_check(iodf_codec* c, void* cuda_stream, uint32_t* bad_streams);

@@ -14,7 +14,8 @@ IODF_MAX_LEVELS = 8
 DECLARED_SYMBOLS = ["iodf_create", "iodf_destroy", "iodf_get_layout", "iodf_forward", "iodf_inverse",
                     "iodf_inverse_level", "iodf_forward_patches", "iodf_inverse_patches",
                     "iodf_codec_create", "iodf_codec_destroy", "iodf_codec_get_layout", "iodf_rans_encode",
-                    "iodf_rans_decode_block", "iodf_codec_check",
+                    "iodf_rans_decode_block", "iodf_codec_check", "iodf_rans_packed_capacity", "iodf_rans_pack",
+                    "iodf_rans_unpack", "iodf_compress_host", "iodf_decompress_host",
                     "iodf_forward_host", "iodf_inverse_host", "iodf_forward_timed", "iodf_inverse_timed", "iodf_forward_static",
                     "iodf_static_scratch_bytes_per_image", "iodf_check", "iodf_launches_per_call",
                     "iodf_strerror", "iodf_last_cuda_error"]
@@ -112,6 +113,16 @@ def load_library(path=None):
     L.iodf_rans_decode_block.argtypes = [vp, C.c_int, vp, vp, vp, C.c_int, vp, vp]
     L.iodf_codec_check.restype = C.c_int
     L.iodf_codec_check.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
+    L.iodf_rans_packed_capacity.restype = C.c_size_t
+    L.iodf_rans_packed_capacity.argtypes = [vp, C.c_int]
+    L.iodf_rans_pack.restype = C.c_int
+    L.iodf_rans_pack.argtypes = [vp, vp, vp, C.c_int, vp, vp]
+    L.iodf_rans_unpack.restype = C.c_int
+    L.iodf_rans_unpack.argtypes = [vp, vp, C.c_size_t, C.c_int, vp, vp, vp]
+    L.iodf_compress_host.restype = C.c_int
+    L.iodf_compress_host.argtypes = [vp, vp, vp, C.c_int, vp, C.c_size_t, C.POINTER(C.c_size_t), vp]
+    L.iodf_decompress_host.restype = C.c_int
+    L.iodf_decompress_host.argtypes = [vp, vp, vp, C.c_size_t, C.c_int, vp, vp]
     L.iodf_forward_host.restype = C.c_int
     L.iodf_forward_host.argtypes = [vp, vp, C.c_int, vp, vp, vp]
     L.iodf_inverse_host.restype = C.c_int
@@ -354,6 +365,63 @@ def iodf_rans_decode_block(codec, block, words, counts, prior, z, stream=None):
                                                z.shape[0], _ptr(z), _stream(stream))
     if rc != 0:
         raise IodfError(rc, "iodf_rans_decode_block")
+
+
+def iodf_rans_packed_capacity(codec, B):
+    return int(load_library().iodf_rans_packed_capacity(codec.handle, int(B)))
+
+
+def iodf_rans_pack(codec, words, counts, packed=None, stream=None):
+    """Container -> compact byte stream. Returns (packed cuda uint8 tensor of full capacity, total bytes);
+    reading the total synchronises."""
+    import torch
+    B = counts.shape[0]
+    if packed is None:
+        packed = torch.empty(iodf_rans_packed_capacity(codec, B), dtype=torch.uint8, device=counts.device)
+    rc = load_library().iodf_rans_pack(codec.handle, _ptr(words), _ptr(counts), B, _ptr(packed), _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_rans_pack")
+    payload = int(packed[4 * B:4 * B + 4].cpu().numpy().view(np.uint32)[0])
+    return packed, 4 * (B + 1) + payload
+
+
+def iodf_rans_unpack(codec, packed, nbytes, B, words=None, counts=None, stream=None):
+    import torch
+    if words is None:
+        words = torch.zeros((B, codec.n_streams, codec.words_per_stream), dtype=torch.int16, device=packed.device)
+    if counts is None:
+        counts = torch.zeros((B, codec.n_streams), dtype=torch.int32, device=packed.device)
+    rc = load_library().iodf_rans_unpack(codec.handle, _ptr(packed), int(nbytes), int(B), _ptr(words), _ptr(counts),
+                                         _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_rans_unpack")
+    return words, counts
+
+
+def iodf_compress_host(model, codec, x_u8_host, out_host=None, stream=None):
+    """Host uint8 images [B,C,H,W] -> (host uint8 buffer, number of valid bytes). Synchronises."""
+    import torch
+    B = x_u8_host.shape[0]
+    if out_host is None:
+        out_host = torch.empty(iodf_rans_packed_capacity(codec, B), dtype=torch.uint8).pin_memory()
+    n = C.c_size_t(0)
+    rc = load_library().iodf_compress_host(model.handle, codec.handle, _ptr(x_u8_host), B, _ptr(out_host),
+                                           out_host.numel(), C.byref(n), _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_compress_host")
+    return out_host, int(n.value)
+
+
+def iodf_decompress_host(model, codec, in_host, nbytes, B, x_u8_host=None, stream=None):
+    """Compact byte stream (host) -> host uint8 images; valid after the stream is synchronised."""
+    import torch
+    if x_u8_host is None:
+        x_u8_host = torch.empty((B,) + tuple(model.in_shape), dtype=torch.uint8).pin_memory()
+    rc = load_library().iodf_decompress_host(model.handle, codec.handle, _ptr(in_host), int(nbytes), int(B),
+                                             _ptr(x_u8_host), _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_decompress_host")
+    return x_u8_host
 
 
 def iodf_codec_check(codec, stream=None):

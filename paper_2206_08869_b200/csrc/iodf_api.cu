@@ -56,6 +56,12 @@ struct iodf_codec {
   uint32_t elems_per_stream = 0;
   uint8_t* d_tables = nullptr;      // R then G
   uint32_t* d_errors = nullptr;
+  uint32_t* d_sizes = nullptr;      // max_batch record sizes (packing scratch)
+  // staging of the host-buffer entry points, allocated by their first call
+  uint16_t* d_words = nullptr;
+  uint32_t* d_counts = nullptr;
+  uint8_t* d_packed = nullptr;
+  size_t packed_capacity = 0;
   iodf::RansArgs args{};
   iodf_codec_layout layout{};
 };
@@ -931,6 +937,7 @@ int iodf_codec_create(const iodf_model* m, const iodf_codec_desc* desc, iodf_cod
   if (e == cudaSuccess) e = cudaMemcpy(c->d_tables, desc->inv_scale, rbytes, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemcpy(c->d_tables + rbytes, desc->sigmoid_table, gbytes, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMalloc(&c->d_errors, sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&c->d_sizes, sizeof(uint32_t) * (size_t)c->max_batch);
   if (e == cudaSuccess) e = cudaMemset(c->d_errors, 0, sizeof(uint32_t));
   cudaSetDevice(prev);
   if (e != cudaSuccess) {
@@ -950,6 +957,10 @@ void iodf_codec_destroy(iodf_codec* c) {
   cudaSetDevice(c->device);
   if (c->d_tables) cudaFree(c->d_tables);
   if (c->d_errors) cudaFree(c->d_errors);
+  if (c->d_sizes) cudaFree(c->d_sizes);
+  if (c->d_words) cudaFree(c->d_words);
+  if (c->d_counts) cudaFree(c->d_counts);
+  if (c->d_packed) cudaFree(c->d_packed);
   delete c;
 }
 
@@ -977,6 +988,119 @@ int iodf_rans_decode_block(iodf_codec* c, int block, const uint16_t* words, cons
   RansArgs a = c->args;
   a.batch = B;
   CUC(c, launch_rans_decode(a, block, words, counts, prior, z, (cudaStream_t)cuda_stream));
+  return IODF_OK;
+}
+
+size_t iodf_rans_packed_capacity(const iodf_codec* c, int B) {
+  if (!c || B < 1) return 0;
+  const size_t S = (size_t)c->args.n_streams, cap = (size_t)c->args.cap;
+  return 4 * ((size_t)B + 1) + (size_t)B * 2 * (S + S * cap);
+}
+
+int iodf_rans_pack(iodf_codec* c, const uint16_t* words, const uint32_t* counts, int B, uint8_t* packed,
+                   void* cuda_stream) {
+  if (!c || !words || !counts || !packed || B < 1 || (uint32_t)B > c->max_batch) return IODF_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(packed) & 3u) || c->args.cap > 65535) return IODF_EINVAL;
+  RansArgs a = c->args;
+  a.batch = B;
+  CUC(c, launch_rans_pack(a, words, counts, c->d_sizes, packed, (cudaStream_t)cuda_stream));
+  return IODF_OK;
+}
+
+int iodf_rans_unpack(iodf_codec* c, const uint8_t* packed, size_t packed_bytes, int B, uint16_t* words,
+                     uint32_t* counts, void* cuda_stream) {
+  if (!c || !words || !counts || !packed || B < 1 || (uint32_t)B > c->max_batch) return IODF_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(packed) & 3u) || c->args.cap > 65535) return IODF_EINVAL;
+  if (packed_bytes < 4 * ((size_t)B + 1)) return IODF_EINVAL;
+  RansArgs a = c->args;
+  a.batch = B;
+  CUC(c, launch_rans_unpack(a, packed, (unsigned long long)(packed_bytes - 4 * ((size_t)B + 1)), words, counts,
+                            (cudaStream_t)cuda_stream));
+  return IODF_OK;
+}
+
+namespace {
+int codec_staging(iodf_codec* c) {
+  if (c->d_packed) return IODF_OK;
+  int prev = -1;
+  CUC(c, cudaGetDevice(&prev));
+  CUC(c, cudaSetDevice(c->device));
+  const size_t S = (size_t)c->args.n_streams, cap = (size_t)c->args.cap, B = c->max_batch;
+  c->packed_capacity = iodf_rans_packed_capacity(c, (int)B);
+  cudaError_t e = cudaMalloc(&c->d_words, B * S * cap * sizeof(uint16_t));
+  if (e == cudaSuccess) e = cudaMalloc(&c->d_counts, B * S * sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&c->d_packed, c->packed_capacity);
+  cudaSetDevice(prev);
+  if (e != cudaSuccess) {
+    c->last_cuda = (int)e;
+    return e == cudaErrorMemoryAllocation ? IODF_ENOMEM : IODF_ECUDA;
+  }
+  return IODF_OK;
+}
+}  // namespace
+
+int iodf_compress_host(iodf_model* m, iodf_codec* c, const uint8_t* x_u8_host, int B, uint8_t* out_host,
+                       size_t out_capacity, size_t* out_bytes, void* cuda_stream) {
+  if (!m || !c || !x_u8_host || !out_host || !out_bytes || B < 1 || (uint32_t)B > m->max_batch ||
+      (uint32_t)B > c->max_batch || c->args.d != (long long)m->layout.d || c->args.cap > 65535)
+    return IODF_EINVAL;
+  int rc = codec_staging(c);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t d = m->layout.d;
+  int32_t* prior = m->layout.d_fact ? m->d_prior : nullptr;
+  CU(m, cudaMemcpyAsync(m->d_x, x_u8_host, (size_t)B * d, cudaMemcpyHostToDevice, st));
+  rc = run_forward(m, m->d_x, B, m->d_z, prior, st);
+  if (rc) return rc;
+  RansArgs a = c->args;
+  a.batch = B;
+  CUC(c, launch_rans_encode(a, m->d_z, prior, c->d_words, c->d_counts, st));
+  CUC(c, launch_rans_pack(a, c->d_words, c->d_counts, c->d_sizes, c->d_packed, st));
+  // the payload size is only known now: read it, then copy exactly header + payload
+  uint32_t payload = 0;
+  CUC(c, cudaMemcpyAsync(&payload, c->d_packed + 4 * (size_t)B, sizeof(payload), cudaMemcpyDeviceToHost, st));
+  CUC(c, cudaStreamSynchronize(st));
+  const size_t total = 4 * ((size_t)B + 1) + payload;
+  *out_bytes = total;
+  if (total > out_capacity) return IODF_ELIMIT;
+  CUC(c, cudaMemcpyAsync(out_host, c->d_packed, total, cudaMemcpyDeviceToHost, st));
+  CUC(c, cudaStreamSynchronize(st));
+  return IODF_OK;
+}
+
+int iodf_decompress_host(iodf_model* m, iodf_codec* c, const uint8_t* in_host, size_t in_bytes, int B,
+                         uint8_t* x_u8_host, void* cuda_stream) {
+  if (!m || !c || !in_host || !x_u8_host || B < 1 || (uint32_t)B > m->max_batch || (uint32_t)B > c->max_batch ||
+      c->args.d != (long long)m->layout.d || c->args.cap > 65535)
+    return IODF_EINVAL;
+  int rc = codec_staging(c);
+  if (rc) return rc;
+  if (in_bytes < 4 * ((size_t)B + 1) || in_bytes > c->packed_capacity) return IODF_EINVAL;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CU(m, cudaMemcpyAsync(c->d_packed, in_host, in_bytes, cudaMemcpyHostToDevice, st));
+  RansArgs a = c->args;
+  a.batch = B;
+  CUC(c, launch_rans_unpack(a, c->d_packed, (unsigned long long)(in_bytes - 4 * ((size_t)B + 1)), c->d_words,
+                            c->d_counts, st));
+  int32_t* prior = m->layout.d_fact ? m->d_prior : nullptr;
+  // decoder order: the final block, then per level: prior parameters, the level's block, inverse couplings
+  CUC(c, launch_rans_decode(a, a.n_blocks - 1, c->d_words, c->d_counts, prior, m->d_z, st));
+  const int L = (int)m->levels.size();
+  for (int li = L - 1; li >= 0; --li) {
+    int q = -1;
+    for (int k = 0; k + 1 < a.n_blocks; ++k)
+      if (c->layout.block_level[k] == li) q = k;
+    if (q >= 0) {
+      if (m->levels[li].plan.has_prior) {
+        rc = launch_inverse_level(m, li, 1, m->d_z, B, nullptr, prior, nullptr, st, PatchGrid());
+        if (rc) return rc;
+      }
+      CUC(c, launch_rans_decode(a, q, c->d_words, c->d_counts, prior, m->d_z, st));
+    }
+    rc = launch_inverse_level(m, li, 2, m->d_z, B, m->d_x, nullptr, nullptr, st, PatchGrid());
+    if (rc) return rc;
+  }
+  CU(m, cudaMemcpyAsync(x_u8_host, m->d_x, (size_t)B * m->layout.d, cudaMemcpyDeviceToHost, st));
   return IODF_OK;
 }
 

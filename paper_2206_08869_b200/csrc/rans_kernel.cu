@@ -178,7 +178,124 @@ __global__ void __launch_bounds__(kThreadsPerBlock) rans_decode_kernel(const Ran
   if (bad && lane == 0 && a.errors) atomicAdd(a.errors, 1u);
 }
 
+// ---- compact byte stream -----------------------------------------------------------------------------
+// Packed form of a batch's container (little endian):
+//   uint32 offset[B + 1]      byte offset of image b's record from the start of the payload; offset[B] =
+//                             payload bytes
+//   payload, per image:       uint16 count[n_streams], then the words of stream 0, 1, ... back to back
+// so an image's record is 2 * (n_streams + sum of its counts) bytes.
+
+// exclusive scan of n values by one warp, 32 at a time; returns the total (in every lane)
+template <typename Load, typename Store>
+__device__ __forceinline__ uint32_t warp_scan(int n, int lane, Load load, Store store) {
+  uint32_t run = 0;
+  for (int base = 0; base < n; base += 32) {
+    const int i = base + lane;
+    const uint32_t v = i < n ? load(i) : 0u;
+    uint32_t inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+      if (lane >= d) inc += o;
+    }
+    if (i < n) store(i, run + inc - v);
+    run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+  }
+  return run;
+}
+
+// record size of every image, in bytes
+__global__ void pack_sizes_kernel(const uint32_t* __restrict__ counts, int n_streams, int cap, uint32_t* __restrict__ sizes) {
+  __shared__ uint32_t part[8];
+  const int b = blockIdx.x;
+  uint32_t sum = 0;
+  for (int s = threadIdx.x; s < n_streams; s += blockDim.x) sum += min(counts[(long)b * n_streams + s], (uint32_t)cap);
+  sum = __reduce_add_sync(0xFFFFFFFFu, sum);
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t t = 0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += part[w];
+    sizes[b] = 2u * ((uint32_t)n_streams + t);
+  }
+}
+
+// offset[0 .. B] from the sizes (one warp)
+__global__ void pack_offsets_kernel(const uint32_t* __restrict__ sizes, int B, uint32_t* __restrict__ offset) {
+  const int lane = threadIdx.x;
+  const uint32_t total = warp_scan(B, lane, [&](int i) { return sizes[i]; }, [&](int i, uint32_t v) { offset[i] = v; });
+  if (lane == 0) offset[B] = total;
+}
+
+// kPack: container -> records; !kPack: records -> container. One CTA per image.
+template <bool kPack>
+__global__ void __launch_bounds__(256) pack_copy_kernel(uint16_t* __restrict__ words, uint32_t* __restrict__ counts,
+                                                        int n_streams, int cap, uint8_t* __restrict__ packed,
+                                                        int B, unsigned long long payload_bytes, uint32_t* errors) {
+  extern __shared__ uint32_t start[];       // word offset of every stream inside the record, after the counts
+  __shared__ uint32_t bad;
+  const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const uint32_t* offset = reinterpret_cast<const uint32_t*>(packed);
+  uint8_t* payload = packed + 4 * (size_t)(B + 1);
+  if (threadIdx.x == 0) bad = 0;
+  __syncthreads();
+  const uint32_t off = offset[b], end = offset[b + 1];
+  // a record that does not fit the payload, or that cannot even hold its counts, is skipped
+  const bool fits = kPack || (off <= end && end <= payload_bytes && (end - off) >= 2u * (uint32_t)n_streams && (off & 1u) == 0);
+  uint16_t* rec = reinterpret_cast<uint16_t*>(payload + off);
+  uint32_t* cnt = counts + (long)b * n_streams;
+  if (!fits) {
+    for (int s = threadIdx.x; s < n_streams; s += blockDim.x) cnt[s] = 0;
+    if (threadIdx.x == 0 && errors) atomicAdd(errors, 1u);
+    return;
+  }
+  if (warp == 0) {
+    const uint32_t total = warp_scan(n_streams, lane,
+        [&](int s) { return min(kPack ? cnt[s] : (uint32_t)rec[s], (uint32_t)cap); },
+        [&](int s, uint32_t v) { start[s] = v; });
+    if (lane == 0) {
+      start[n_streams] = total;
+      if (!kPack && 2u * ((uint32_t)n_streams + total) != end - off) bad = 1;    // counts disagree with the record size
+    }
+  }
+  __syncthreads();
+  if (bad) {
+    for (int s = threadIdx.x; s < n_streams; s += blockDim.x) cnt[s] = 0;
+    if (threadIdx.x == 0 && errors) atomicAdd(errors, 1u);
+    return;
+  }
+  for (int s = threadIdx.x; s < n_streams; s += blockDim.x) {
+    if (kPack) rec[s] = (uint16_t)min(cnt[s], (uint32_t)cap);
+    else cnt[s] = min((uint32_t)rec[s], (uint32_t)cap);
+  }
+  uint16_t* body = rec + n_streams;
+  for (int s = warp; s < n_streams; s += nwarps) {
+    const uint32_t n = start[s + 1] - start[s];
+    uint16_t* w = words + ((long)b * n_streams + s) * cap;
+    uint16_t* r = body + start[s];
+    for (uint32_t i = lane; i < n; i += 32) {
+      if (kPack) r[i] = w[i]; else w[i] = r[i];
+    }
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_rans_pack(const RansArgs& a, const uint16_t* words, const uint32_t* counts, uint32_t* sizes,
+                             uint8_t* packed, cudaStream_t stream) {
+  pack_sizes_kernel<<<a.batch, 256, 0, stream>>>(counts, a.n_streams, a.cap, sizes);
+  pack_offsets_kernel<<<1, 32, 0, stream>>>(sizes, a.batch, reinterpret_cast<uint32_t*>(packed));
+  pack_copy_kernel<true><<<a.batch, 256, 4 * (a.n_streams + 1), stream>>>(
+      const_cast<uint16_t*>(words), const_cast<uint32_t*>(counts), a.n_streams, a.cap, packed, a.batch, 0ull, a.errors);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rans_unpack(const RansArgs& a, const uint8_t* packed, unsigned long long payload_bytes,
+                               uint16_t* words, uint32_t* counts, cudaStream_t stream) {
+  pack_copy_kernel<false><<<a.batch, 256, 4 * (a.n_streams + 1), stream>>>(
+      words, counts, a.n_streams, a.cap, const_cast<uint8_t*>(packed), a.batch, payload_bytes, a.errors);
+  return cudaGetLastError();
+}
 
 static size_t table_smem(const RansArgs& a) { return 4 * (size_t)a.n_scales + 2 * (size_t)(2 * a.umax + 1) + 16; }
 

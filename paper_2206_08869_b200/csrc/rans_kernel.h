@@ -33,4 +33,13 @@ cudaError_t launch_rans_encode(const RansArgs& a, const int32_t* z, const int32_
 cudaError_t launch_rans_decode(const RansArgs& a, int block, const uint16_t* words, const uint32_t* counts,
                                const int32_t* prior, int32_t* z, cudaStream_t stream);
 
+// Container <-> compact byte stream ([B + 1] uint32 record offsets, then per image uint16 counts and the
+// streams' words back to back). `sizes` is a scratch array of batch uint32. Unpacking checks every
+// record against `payload_bytes` and its own counts; a bad record gives zero counts and is counted in
+// a.errors.
+cudaError_t launch_rans_pack(const RansArgs& a, const uint16_t* words, const uint32_t* counts, uint32_t* sizes,
+                             uint8_t* packed, cudaStream_t stream);
+cudaError_t launch_rans_unpack(const RansArgs& a, const uint8_t* packed, unsigned long long payload_bytes,
+                               uint16_t* words, uint32_t* counts, cudaStream_t stream);
+
 }  // namespace iodf

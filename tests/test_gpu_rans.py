@@ -154,3 +154,56 @@ def test_bad_scale_index_and_damaged_stream_are_reported(G):
     with pytest.raises(G.IodfError) as e:
         G.iodf_codec_create(m, bad)
     assert e.value.status == -1
+
+
+def _packed_reference(words, counts):
+    """The compact byte stream written out with numpy: offsets, then per image counts and words."""
+    B, S, _ = words.shape
+    recs = []
+    for b in range(B):
+        parts = [counts[b].astype("<u2").tobytes()]
+        parts += [words[b, s, :counts[b, s]].astype("<u2").tobytes() for s in range(S)]
+        recs.append(b"".join(parts))
+    off = np.zeros(B + 1, dtype="<u4")
+    off[1:] = np.cumsum([len(r) for r in recs])
+    return off.tobytes() + b"".join(recs)
+
+
+@pytest.mark.parametrize("hw,splits,batch,eps", [(32, [True, True, True], 7, 256), (16, [True, False], 33, 40)])
+def test_compact_stream_and_host_round_trip(G, hw, splits, batch, eps):
+    import torch
+    model = S.make_model(0xAF00 + hw, 3, hw, hw, splits, 2, 24, prune=(0.4, 0.7))
+    codec = S.logistic_codec(elems_per_stream=eps)
+    x = S.smooth_field_images(0xAF10 + hw, batch, hw, hw, 2.0)
+    z_ref, p_ref = O.forward(O.Packed(model), x)
+    w_ref, c_ref = O.rans_encode(codec, model, z_ref, p_ref)
+    want = _packed_reference(w_ref, c_ref)
+
+    m = G.iodf_create(model, batch + 3)
+    cd = G.iodf_codec_create(m, codec)
+    z, p = G.iodf_forward(m, _t(x))
+    words, counts = G.iodf_rans_encode(cd, z, p)
+    packed, n = G.iodf_rans_pack(cd, words, counts)
+    assert n == len(want) and n <= G.iodf_rans_packed_capacity(cd, batch)
+    assert packed[:n].cpu().numpy().tobytes() == want
+    w2, c2 = G.iodf_rans_unpack(cd, packed, n, batch)
+    G.iodf_codec_check(cd)
+    assert torch.equal(c2, counts)
+    cc = counts.cpu().numpy().view(np.uint32)
+    np.testing.assert_array_equal(_valid(w2.cpu().numpy().view(np.uint16), cc), _valid(w_ref, c_ref))
+
+    # images -> bytes -> images through the host-buffer calls
+    xh = torch.from_numpy(x).pin_memory()
+    out, nb = G.iodf_compress_host(m, cd, xh)
+    assert out[:nb].numpy().tobytes() == want
+    back = G.iodf_decompress_host(m, cd, out, nb, batch)
+    torch.cuda.synchronize()
+    G.iodf_check(m)
+    G.iodf_codec_check(cd)
+    np.testing.assert_array_equal(back.numpy(), x)
+    # a byte stream cut short is reported, not read past its end
+    G.iodf_decompress_host(m, cd, out, nb - 10, batch)
+    with pytest.raises(G.IodfError):
+        G.iodf_codec_check(cd)
+    with pytest.raises(G.IodfError):                          # too small an output buffer
+        G.iodf_compress_host(m, cd, xh, out_host=torch.empty(64, dtype=torch.uint8).pin_memory())
