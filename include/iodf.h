@@ -202,9 +202,10 @@ int iodf_inverse_patches(iodf_model* m, const int32_t* z, int H, int W, uint8_t*
  * range-ANS; Sec. 5.3 leaves "an optimized GPU implementation of rANS" as future work).
  *
  * The prior's integer form is given by the caller (HOST arrays, copied):
- *   sigmoid_table[u + umax], u in [-umax, umax]: a non-decreasing table of M' sigma(u / 64), M' =
- *     2^16 - 4097, entries <= M';
- *   inv_scale[ls] = 2^21 / s_ls for scale index ls in [0, n_scales) (the prior head's log-scale index);
+ *   sigmoid_table[u + umax], u in [-umax, umax], umax <= 8192: a non-decreasing table of
+ *     M' sigma(u / 64), M' = 2^16 - 4097, entries <= M';
+ *   inv_scale[ls] = 2^21 / s_ls, in [1, 2^30), for scale index ls in [0, n_scales), n_scales <= 1024
+ *     (the prior head's log-scale index);
  *   final_ls: the fixed scale index (with mu = 0) of blocks that have no prior head, the final block
  *     among them.
  * An element with prior (mu, ls) is coded as the symbol k = clamp(z - mu, -2048, 2048) + 2048 with
@@ -268,7 +269,8 @@ int iodf_rans_decode_block(iodf_codec* c, int block, const uint16_t* words, cons
  * iodf_rans_packed_capacity(c, B) bytes; the total is 4 (B + 1) + offset[B]); iodf_rans_unpack
  * restores the container from packed_bytes bytes, checking every record against the payload size
  * and its own counts (a bad record gets zero counts and is reported by iodf_codec_check). Both need
- * words_per_stream <= 65535.
+ * words_per_stream <= 65535 (IODF_EINVAL otherwise), at most 8192 streams per image and a byte stream
+ * below 4 GiB (IODF_EUNSUPPORTED otherwise).
  */
 size_t iodf_rans_packed_capacity(const iodf_codec* c, int B);
 int iodf_rans_pack(iodf_codec* c, const uint16_t* words, const uint32_t* counts, int B, uint8_t* packed,

@@ -886,7 +886,7 @@ int iodf_codec_create(const iodf_model* m, const iodf_codec_desc* desc, iodf_cod
   if (!m || !desc || !out) return IODF_EINVAL;
   *out = nullptr;
   if (desc->abi_version != IODF_ABI_VERSION) return IODF_EVERSION;
-  if (!desc->sigmoid_table || !desc->inv_scale || desc->umax < 1 || desc->umax > 16384 || desc->n_scales < 1 ||
+  if (!desc->sigmoid_table || !desc->inv_scale || desc->umax < 1 || desc->umax > 8192 || desc->n_scales < 1 ||
       desc->n_scales > 1024 || desc->elems_per_stream < 1 || desc->elems_per_stream > 65536)
     return IODF_EINVAL;
   if (desc->final_ls < 0 || desc->final_ls >= (int32_t)desc->n_scales) return IODF_EINVAL;
@@ -1001,6 +1001,8 @@ int iodf_rans_pack(iodf_codec* c, const uint16_t* words, const uint32_t* counts,
                    void* cuda_stream) {
   if (!c || !words || !counts || !packed || B < 1 || (uint32_t)B > c->max_batch) return IODF_EINVAL;
   if ((reinterpret_cast<uintptr_t>(packed) & 3u) || c->args.cap > 65535) return IODF_EINVAL;
+  // record offsets are 32-bit and the per-stream offsets of an image live in shared memory
+  if (iodf_rans_packed_capacity(c, B) >= (1ull << 32) || c->args.n_streams > 8192) return IODF_EUNSUPPORTED;
   RansArgs a = c->args;
   a.batch = B;
   CUC(c, launch_rans_pack(a, words, counts, c->d_sizes, packed, (cudaStream_t)cuda_stream));
@@ -1012,6 +1014,7 @@ int iodf_rans_unpack(iodf_codec* c, const uint8_t* packed, size_t packed_bytes, 
   if (!c || !words || !counts || !packed || B < 1 || (uint32_t)B > c->max_batch) return IODF_EINVAL;
   if ((reinterpret_cast<uintptr_t>(packed) & 3u) || c->args.cap > 65535) return IODF_EINVAL;
   if (packed_bytes < 4 * ((size_t)B + 1)) return IODF_EINVAL;
+  if (packed_bytes >= (1ull << 32) || c->args.n_streams > 8192) return IODF_EUNSUPPORTED;
   RansArgs a = c->args;
   a.batch = B;
   CUC(c, launch_rans_unpack(a, packed, (unsigned long long)(packed_bytes - 4 * ((size_t)B + 1)), words, counts,
@@ -1044,6 +1047,7 @@ int iodf_compress_host(iodf_model* m, iodf_codec* c, const uint8_t* x_u8_host, i
   if (!m || !c || !x_u8_host || !out_host || !out_bytes || B < 1 || (uint32_t)B > m->max_batch ||
       (uint32_t)B > c->max_batch || c->args.d != (long long)m->layout.d || c->args.cap > 65535)
     return IODF_EINVAL;
+  if (iodf_rans_packed_capacity(c, B) >= (1ull << 32) || c->args.n_streams > 8192) return IODF_EUNSUPPORTED;
   int rc = codec_staging(c);
   if (rc) return rc;
   cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -1076,6 +1080,7 @@ int iodf_decompress_host(iodf_model* m, iodf_codec* c, const uint8_t* in_host, s
   int rc = codec_staging(c);
   if (rc) return rc;
   if (in_bytes < 4 * ((size_t)B + 1) || in_bytes > c->packed_capacity) return IODF_EINVAL;
+  if (in_bytes >= (1ull << 32) || c->args.n_streams > 8192) return IODF_EUNSUPPORTED;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   CU(m, cudaMemcpyAsync(c->d_packed, in_host, in_bytes, cudaMemcpyHostToDevice, st));
   RansArgs a = c->args;
