@@ -8,9 +8,9 @@ library each marshal the arrays produced here into their own formats.
 from .rng import Stream
 from .images import smooth_field_images
 from .codec import logistic_codec
-from .model import (make_model, CONFIGS, config_model, config_images, model_macs, level_shapes,
+from .model import (make_model, make_residual_model, CONFIGS, config_model, config_images, model_macs, level_shapes,
                     latent_sizes, masked_dense_model, zero_padded_model)
 
-__all__ = ["Stream", "smooth_field_images", "make_model", "CONFIGS", "config_model",
+__all__ = ["Stream", "smooth_field_images", "make_model", "make_residual_model", "CONFIGS", "config_model",
            "config_images", "model_macs", "level_shapes", "latent_sizes", "masked_dense_model",
            "zero_padded_model", "logistic_codec"]

@@ -97,6 +97,46 @@ def make_model(seed, in_c, in_h, in_w, splits, n_couplings, hidden, prune=None, 
     return {"in_c": in_c, "in_h": in_h, "in_w": in_w, "levels": levels}
 
 
+def make_residual_model(seed, in_c, in_h, in_w, splits, n_couplings, hidden, n_blocks, prune=None, prior=True):
+    """The flow with the paper's coupling network: conv3x3 (C/2 -> hidden), n_blocks residual blocks
+    [conv3x3 (hidden -> K), ReLU, conv3x3 (K -> K'), scatter add onto the hidden-wide shortcut, ReLU],
+    conv3x3 (hidden -> C/2). K, K' are the kept (odd) widths when `prune` = (lo, hi) keep fractions.
+    A coupling carries "blocks": per block the shortcut requantisation pair, the clip after the ReLU
+    and the index list that places the second conv's K' outputs among the hidden channels.
+    Hidden activations use the unsigned 8-bit range 0..255."""
+    shapes = level_shapes(in_c, in_h, in_w, splits)
+    levels = []
+    for li, ((c, h, w), sp) in enumerate(zip(shapes, splits)):
+        ca, cb = c // 2, c - c // 2
+        couplings = []
+        for ki in range(n_couplings):
+            st = Stream(seed, "R%d/K%d" % (li, ki))
+            p = st.permutation(c)
+            layers = [_layer(st, 3, ca, hidden, 48.0, True, (0, 255), True)]
+            blocks = []
+            for b in range(n_blocks):
+                if prune is None:
+                    k1 = k2 = hidden
+                else:
+                    f = prune[0] + (prune[1] - prune[0]) * st.uniform(2)
+                    k1, k2 = (min(hidden, int(math.floor(hidden * x + 0.5)) | 1) for x in f)
+                layers.append(_layer(st, 3, hidden, k1, 23.0, True, (0, 255), True))
+                layers.append(_layer(st, 3, k1, k2, 23.0, False, None, True))
+                idx = np.sort(st.permutation(hidden)[:k2]).astype(np.int32)
+                blocks.append({"short_m0": int(st.integers(1 << 30, 1 << 31, 1)[0]), "short_s": 0,
+                               "clamp": (0, 255), "idx": idx})
+            layers.append(_layer(st, 3, hidden, cb, 30.0, False, None, True))
+            couplings.append({"perm": p.astype(np.int32), "in_m0": int(st.integers(1 << 30, 1 << 31, 1)[0]),
+                              "in_s": 1, "layers": layers, "blocks": blocks})
+        head = None
+        if sp and prior:
+            st = Stream(seed, "R%d/prior" % li)
+            head = {"in_m0": int(st.integers(1 << 30, 1 << 31, 1)[0]), "in_s": 1,
+                    "layer": _layer(st, 3, ca, 2 * cb, 48.0, False, None, True), "ls_lo": 0, "ls_hi": 63}
+        levels.append({"c": c, "h": h, "w": w, "couplings": couplings, "split": bool(sp), "prior": head})
+    return {"in_c": in_c, "in_h": in_h, "in_w": in_w, "levels": levels}
+
+
 def latent_sizes(model):
     """(d, d_fact, blocks): blocks = [(level, channels, h, w, has_prior)] in z order."""
     blocks = []

@@ -76,9 +76,13 @@ class Packed:
             for cp in lv["couplings"]:
                 desc.append(len(cp["perm"]))
                 desc.extend(int(v) for v in cp["perm"])
-                desc.extend([cp["in_m0"], cp["in_s"], len(cp["layers"])])
+                blocks = cp.get("blocks") or []
+                desc.extend([cp["in_m0"], cp["in_s"], len(cp["layers"]), len(blocks)])
                 for ly in cp["layers"]:
                     layer(ly)
+                for rb in blocks:
+                    desc.extend([rb["short_m0"], rb["short_s"], rb["clamp"][0], rb["clamp"][1], len(rb["idx"])])
+                    desc.extend(int(v) for v in rb["idx"])
             if lv["prior"] is not None:
                 hd = lv["prior"]
                 desc.extend([hd["in_m0"], hd["in_s"]])

@@ -14,6 +14,13 @@
 //                 (k-1)/2 so the map keeps its shape (App. B.1), int32 accumulator + int32 bias.
 //   hidden layers Sec. 4.1 "Integer-Only ReLU": max(0, .) on the integer part, then the 8-bit clip.
 //   gate          Eq. 8 (Sec. 4.4): a filter whose binary gate is 0 outputs an all-zero map.
+//   residual t    Eq. 3 (Sec. 4.1) and the scatter add of Sec. 4.5: a coupling whose network is
+//                 conv -> L x [ ReLU(SAdd(Q(x), GConv(ReLU(GConv(Q(x)))))) ] -> conv (App. B.1: eight
+//                 blocks, 3x3 convs, 128 hidden channels). In integers (a reading, the paper
+//                 requantises in floating point): the block input x is an 8-bit tensor of D channels
+//                 and feeds the first conv as it is; the second conv's requantised outputs (kept
+//                 channels only) are added, through their index list, to the requantised shortcut
+//                 rq(x; M_r, s_r) of all D channels; then max(0, .) and the block's clip.
 //   coupling      Eq. 2 (Sec. 3): z_a = x_a, z_b = x_b + round(t(x_a)); inverse subtracts.
 //   levels        Sec. 5 / App. B.1: L levels of D couplings; 2x2 space-to-depth before a level;
 //                 half of the channels factored out after it; the prior head gives (mu, log-scale
@@ -49,10 +56,16 @@ struct Layer {
   const int32_t* s;      // [c_out]
   const int32_t* gate;   // [c_out] or null
 };
+struct ResBlock {                  // block l uses layers[1 + 2l] and layers[2 + 2l] of its coupling
+  int32_t short_m0, short_s;       // shortcut requantisation Q(x), per tensor
+  int32_t clamp_lo, clamp_hi;      // clip after the block's ReLU
+  std::vector<int32_t> idx;        // channel of the block's D-wide tensor that receives output j of the second conv
+};
 struct Coupling {
   std::vector<int32_t> perm;
   int32_t in_m0, in_s;
   std::vector<Layer> layers;
+  std::vector<ResBlock> blocks;    // empty: plain chain of layers; else [conv_in, (conv_a, conv_b) per block, conv_out]
 };
 struct Head {
   int32_t in_m0, in_s, ls_lo, ls_hi;
@@ -127,6 +140,30 @@ bool translation(const Coupling& cp, const int32_t* xa, int ca, int h, int w, st
   for (size_t i = 0; i < a.size(); ++i) a[i] = (int32_t)clampi(rq(xa[i], cp.in_m0, cp.in_s), -128, 127);
   bool ok = true;
   std::vector<int64_t> y;
+  if (!cp.blocks.empty()) {
+    const size_t px = (size_t)h * w;
+    ok = run_layer(cp.layers[0], a, h, w, y) && ok;                      // conv_in -> x of the first block
+    T32 x(y.begin(), y.end());
+    const int D = cp.layers[0].c_out;
+    for (size_t b = 0; b < cp.blocks.size(); ++b) {
+      const ResBlock& rb = cp.blocks[b];
+      std::vector<int64_t> mid, br;
+      ok = run_layer(cp.layers[1 + 2 * b], x, h, w, mid) && ok;          // ReLU(GConv(Q(x)))
+      T32 m32(mid.begin(), mid.end());
+      ok = run_layer(cp.layers[2 + 2 * b], m32, h, w, br) && ok;         // GConv(.), kept channels only
+      std::vector<int64_t> sum((size_t)D * px);
+      for (size_t i = 0; i < sum.size(); ++i) sum[i] = rq(x[i], rb.short_m0, rb.short_s);   // Q(x), all D channels
+      for (size_t j = 0; j < rb.idx.size(); ++j)                          // scatter add
+        for (size_t q = 0; q < px; ++q) sum[(size_t)rb.idx[j] * px + q] += br[j * px + q];
+      for (size_t i = 0; i < sum.size(); ++i)
+        x[i] = (int32_t)clampi(std::max<int64_t>(sum[i], 0), rb.clamp_lo, rb.clamp_hi);
+    }
+    ok = run_layer(cp.layers.back(), x, h, w, y) && ok;                  // conv_out -> translation
+    t.swap(y);
+    for (size_t i = 0; i < t.size(); ++i)
+      if (t[i] > INT32_MAX || t[i] < INT32_MIN) ok = false;
+    return ok;
+  }
   for (size_t li = 0; li < cp.layers.size(); ++li) {
     ok = run_layer(cp.layers[li], a, h, w, y) && ok;
     if (li + 1 < cp.layers.size()) {
@@ -318,15 +355,36 @@ bool parse(const int32_t* desc, long n, const int8_t* wts, const int32_t* par, M
       }
       cp.in_m0 = cu.next(); cp.in_s = cu.next();
       int nlay = cu.next();
-      if (!cu.ok || nlay < 1 || cp.in_m0 < (1 << 30) || cp.in_s < 0 || cp.in_s > 31) return false;
-      int cin = c / 2;
+      int nblk = cu.next();
+      if (!cu.ok || nlay < 1 || nblk < 0 || cp.in_m0 < (1 << 30) || cp.in_s < 0 || cp.in_s > 31) return false;
+      if (nblk > 0 && nlay != 2 + 2 * nblk) return false;
+      int cin = c / 2, D = 0;
       for (int q = 0; q < nlay; ++q) {
         Layer L;
         if (!parse_layer(cu, wts, par, L) || L.c_in != cin) return false;
         cin = L.c_out;
+        if (q == 0) D = L.c_out;
+        // after a block's second conv the tensor is D wide again, whatever that conv keeps
+        if (nblk > 0 && q >= 2 && q % 2 == 0 && q < nlay - 1) cin = D;
         cp.layers.push_back(L);
       }
       if (cin != c - c / 2) return false;
+      for (int b = 0; b < nblk; ++b) {
+        ResBlock rb;
+        rb.short_m0 = cu.next(); rb.short_s = cu.next(); rb.clamp_lo = cu.next(); rb.clamp_hi = cu.next();
+        int nidx = cu.next();
+        if (!cu.ok || rb.short_m0 < (1 << 30) || rb.short_s < 0 || rb.short_s > 31 || rb.clamp_lo > rb.clamp_hi)
+          return false;
+        const Layer& second = cp.layers[2 + 2 * b];
+        if (nidx != second.c_out || second.relu || second.has_clamp) return false;
+        std::vector<int> used(D, 0);
+        for (int j = 0; j < nidx; ++j) {
+          int ch = cu.next();
+          if (!cu.ok || ch < 0 || ch >= D || used[ch]) return false;
+          used[ch] = 1; rb.idx.push_back(ch);
+        }
+        cp.blocks.push_back(rb);
+      }
       lv.couplings.push_back(cp);
     }
     if (lv.has_prior) {

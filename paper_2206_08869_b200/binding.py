@@ -178,6 +178,10 @@ class _Marshalled:
         for li, lv in enumerate(model["levels"]):
             cps = (CouplingDesc * max(1, len(lv["couplings"])))()
             for ki, cp in enumerate(lv["couplings"]):
+                if cp.get("blocks"):
+                    # the C descriptor has no residual blocks: refuse here rather than pass a layer
+                    # list whose meaning would be lost
+                    raise IodfError(-6, "iodf_create (couplings with residual blocks)")
                 perm = np.ascontiguousarray(cp["perm"], dtype=np.int32)
                 lays = (LayerDesc * len(cp["layers"]))(*[layer(ly) for ly in cp["layers"]])
                 self.keep += [perm, lays]

@@ -100,3 +100,12 @@ def test_gated_models_must_be_compacted():
     dense = S.masked_dense_model(_small(), 9, 12)
     with pytest.raises(ValueError):
         G.iodf_create(dense, 4)
+
+
+def test_residual_block_couplings_are_refused_not_misread():
+    """The oracle knows the residual-block coupling network; the CUDA library does not yet: creating
+    such a model must fail with IODF_EUNSUPPORTED instead of running something else."""
+    m = S.make_residual_model(3, 3, 8, 8, [True], 1, 8, 1)
+    with pytest.raises(G.IodfError) as e:
+        G.iodf_create(m, 2)
+    assert e.value.status == -6
