@@ -34,7 +34,7 @@
 extern "C" {
 #endif
 
-#define IODF_ABI_VERSION 1u
+#define IODF_ABI_VERSION 2u
 
 typedef enum {
   IODF_OK = 0,
@@ -73,10 +73,30 @@ typedef struct {
  * The last layer must have relu = 0 and has_clamp = 0 (its rq output is the integer translation).
  */
 typedef struct {
+  int32_t short_m0, short_s;      /* shortcut requantisation Q(x) of the block, per tensor           */
+  int32_t clamp_lo, clamp_hi;     /* clip after the block's ReLU                                     */
+  uint32_t n_idx;                 /* = c_out of the block's second conv                              */
+  const int32_t* idx;             /* HOST: channel of the D-wide block tensor that output j adds to  */
+} iodf_resblock_desc;
+
+/*
+ * With n_blocks > 0 the network is the residual form of Eq. 3 (Sec. 4.1) with the scatter add of
+ * Sec. 4.5 (App. B.1: eight blocks, 3x3 convs, 128 hidden channels): layers = [conv_in,
+ * (conv_a, conv_b) per block, conv_out], n_layers = 2 + 2 n_blocks. conv_in maps the requantised
+ * x_a to the D-channel block tensor x (ReLU + clip); per block
+ *   m = clip(ReLU(rq(conv_a(x))));  b = rq(conv_b(m))   (conv_b: relu = 0, has_clamp = 0, K' kept outputs)
+ *   x = clip(max(rq(x; short_m0, short_s) [all D channels]  +  scatter of b through idx, 0), clamp_lo, clamp_hi)
+ * and conv_out maps x to the integer translation. This build runs it for 3x3 convs with D and every
+ * kept width <= 128, hidden activations in 0..255, and levels of at most 256 pixels per image;
+ * all couplings of a level must then be of this form.
+ */
+typedef struct {
   const int32_t* perm;            /* HOST, C entries, a permutation of 0..C-1                        */
   int32_t in_m0, in_s;
   uint32_t n_layers;
   const iodf_layer_desc* layers;  /* HOST                                                            */
+  uint32_t n_blocks;              /* 0: the layers are a plain chain                                 */
+  const iodf_resblock_desc* blocks; /* HOST, n_blocks entries                                        */
 } iodf_coupling_desc;
 
 /*

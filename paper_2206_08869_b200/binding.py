@@ -8,7 +8,7 @@ import numpy as np
 
 from . import build as _build
 
-IODF_ABI_VERSION = 1
+IODF_ABI_VERSION = 2
 IODF_MAX_LEVELS = 8
 
 DECLARED_SYMBOLS = ["iodf_create", "iodf_destroy", "iodf_get_layout", "iodf_forward", "iodf_inverse",
@@ -27,9 +27,15 @@ class LayerDesc(C.Structure):
                 ("weight_off", C.c_uint64), ("requant_off", C.c_uint64)]
 
 
+class ResBlockDesc(C.Structure):
+    _fields_ = [("short_m0", C.c_int32), ("short_s", C.c_int32), ("clamp_lo", C.c_int32), ("clamp_hi", C.c_int32),
+                ("n_idx", C.c_uint32), ("idx", C.POINTER(C.c_int32))]
+
+
 class CouplingDesc(C.Structure):
     _fields_ = [("perm", C.POINTER(C.c_int32)), ("in_m0", C.c_int32), ("in_s", C.c_int32),
-                ("n_layers", C.c_uint32), ("layers", C.POINTER(LayerDesc))]
+                ("n_layers", C.c_uint32), ("layers", C.POINTER(LayerDesc)),
+                ("n_blocks", C.c_uint32), ("blocks", C.POINTER(ResBlockDesc))]
 
 
 class LevelDesc(C.Structure):
@@ -178,15 +184,19 @@ class _Marshalled:
         for li, lv in enumerate(model["levels"]):
             cps = (CouplingDesc * max(1, len(lv["couplings"])))()
             for ki, cp in enumerate(lv["couplings"]):
-                if cp.get("blocks"):
-                    # the C descriptor has no residual blocks: refuse here rather than pass a layer
-                    # list whose meaning would be lost
-                    raise IodfError(-6, "iodf_create (couplings with residual blocks)")
                 perm = np.ascontiguousarray(cp["perm"], dtype=np.int32)
                 lays = (LayerDesc * len(cp["layers"]))(*[layer(ly) for ly in cp["layers"]])
                 self.keep += [perm, lays]
+                rblocks = cp.get("blocks") or []
+                rbs = (ResBlockDesc * max(1, len(rblocks)))()
+                for bi, rb in enumerate(rblocks):
+                    idx = np.ascontiguousarray(rb["idx"], dtype=np.int32)
+                    self.keep.append(idx)
+                    rbs[bi] = ResBlockDesc(rb["short_m0"], rb["short_s"], rb["clamp"][0], rb["clamp"][1], len(idx),
+                                           idx.ctypes.data_as(C.POINTER(C.c_int32)))
+                self.keep.append(rbs)
                 cps[ki] = CouplingDesc(perm.ctypes.data_as(C.POINTER(C.c_int32)), cp["in_m0"], cp["in_s"],
-                                       len(cp["layers"]), lays)
+                                       len(cp["layers"]), lays, len(rblocks), rbs)
             self.keep.append(cps)
             levels[li].n_couplings = len(lv["couplings"])
             levels[li].couplings = cps

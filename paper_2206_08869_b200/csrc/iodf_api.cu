@@ -13,6 +13,7 @@
 #include "../../include/iodf.h"
 #include "iodf_dev.h"
 #include "rans_kernel.h"
+#include "res_level.h"
 #include "level_kernel.h"
 
 using namespace iodf;
@@ -387,6 +388,150 @@ int cuda_fail(iodf_model* m, cudaError_t e) {
     if (e__ != cudaSuccess) return cuda_fail(m, e__); \
   } while (0)
 
+// A coupling with residual blocks (layers already checked one by one): shapes, ranges and what this
+// build runs.
+int check_residual(const iodf_coupling_desc& cp, const Blobs& B, uint32_t ca, uint32_t cb, uint32_t px) {
+  if (!cp.blocks || cp.n_layers != 2 + 2 * cp.n_blocks) return IODF_EINVAL;
+  const iodf_layer_desc& cin = cp.layers[0];
+  const iodf_layer_desc& cout = cp.layers[cp.n_layers - 1];
+  const uint32_t D = cin.c_out;
+  if (cin.c_in != ca || cout.c_in != D || cout.c_out != cb || cout.relu || cout.has_clamp) return IODF_EINVAL;
+  for (uint32_t b = 0; b < cp.n_blocks; ++b) {
+    const iodf_layer_desc& la = cp.layers[1 + 2 * b];
+    const iodf_layer_desc& lb = cp.layers[2 + 2 * b];
+    const iodf_resblock_desc& rb = cp.blocks[b];
+    if (la.c_in != D || lb.c_in != la.c_out || lb.relu || lb.has_clamp) return IODF_EINVAL;
+    if (!rb.idx || rb.n_idx != lb.c_out || rb.short_m0 < (1 << 30) || rb.short_s < 0 || rb.short_s > 31 ||
+        rb.clamp_lo > rb.clamp_hi)
+      return IODF_EINVAL;
+    std::vector<char> used(D, 0);
+    for (uint32_t j = 0; j < rb.n_idx; ++j) {
+      if (rb.idx[j] < 0 || rb.idx[j] >= (int32_t)D || used[rb.idx[j]]) return IODF_EINVAL;
+      used[rb.idx[j]] = 1;
+    }
+  }
+  // what the residual kernel runs
+  if (px > (uint32_t)kResMaxPixels) return IODF_EUNSUPPORTED;
+  for (uint32_t q = 0; q < cp.n_layers; ++q) {
+    const iodf_layer_desc& L = cp.layers[q];
+    if (L.k != 3 || L.c_out > (uint32_t)kResMaxWidth || L.c_in > (uint32_t)kResMaxWidth) return IODF_EUNSUPPORTED;
+    const bool hidden = q == 0 || (q + 1 < cp.n_layers && q % 2 == 1);      // conv_in and every conv_a
+    if (hidden) {
+      Act a;
+      int rc = hidden_range(L, &a);
+      if (rc) return rc;
+      if (a.lo != 0 || a.hi != 255) return IODF_EUNSUPPORTED;
+    }
+    int rc = check_overflow(L, B, q == 0 ? 128 : 255);
+    if (rc) return rc;
+  }
+  for (uint32_t b = 0; b < cp.n_blocks; ++b)
+    if (cp.blocks[b].clamp_lo != 0 || cp.blocks[b].clamp_hi != 255) return IODF_EUNSUPPORTED;
+  return IODF_OK;
+}
+
+// Level blob of a residual level: ResHead, coupling records, conv records, then tables and weights.
+int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P, std::vector<uint8_t>& blob,
+                        const std::vector<std::vector<int>>& cols, uint32_t smem_limit) {
+  const int ca = P.ca, cb = P.cb, px = P.px;
+  std::vector<ResCouplingRec> cps(lv.n_couplings);
+  std::vector<ResConv> convs;
+  int maxD = 32, maxK = 32, kmax = 32, nmax = 16;
+  struct Src { const iodf_layer_desc* L; };
+  std::vector<const iodf_layer_desc*> conv_layer;
+  auto add_conv = [&](const iodf_layer_desc& L, int kind, int src, int dst, bool a_unsigned) {
+    ResConv c{};
+    c.n = (int)L.c_out; c.n_pad = (int)up(L.c_out, 16); c.kpad = (int)up(L.c_in, 32);
+    c.a_unsigned = a_unsigned; c.kind = kind; c.src = src; c.dst = dst;
+    c.slice_bytes = (uint32_t)c.n_pad * (uint32_t)c.kpad;
+    kmax = std::max(kmax, c.kpad); nmax = std::max(nmax, c.n_pad);
+    convs.push_back(c);
+    conv_layer.push_back(&L);
+    return (int)convs.size() - 1;
+  };
+  for (uint32_t ki = 0; ki < lv.n_couplings; ++ki) {
+    const iodf_coupling_desc& cp = lv.couplings[ki];
+    cps[ki].in_m0 = cp.in_m0; cps[ki].in_s = cp.in_s;
+    cps[ki].conv0 = (int)convs.size(); cps[ki].n_convs = (int)cp.n_layers;
+    maxD = std::max(maxD, (int)up(cp.layers[0].c_out, 32));
+    add_conv(cp.layers[0], kResHidden, 0, 1, false);
+    for (uint32_t b = 0; b < cp.n_blocks; ++b) {
+      maxK = std::max(maxK, (int)up(cp.layers[1 + 2 * b].c_out, 32));
+      add_conv(cp.layers[1 + 2 * b], kResHidden, 1, 2, true);
+      const int j = add_conv(cp.layers[2 + 2 * b], kResBranch, 2, 1, true);
+      convs[j].short_m0 = cp.blocks[b].short_m0; convs[j].short_s = cp.blocks[b].short_s;
+    }
+    add_conv(cp.layers[cp.n_layers - 1], kResOut, 1, 1, true);
+  }
+  int prior_conv = -1;
+  if (lv.has_prior) prior_conv = add_conv(lv.prior_layer, kResPrior, 0, 0, false);
+
+  ResHead H{};
+  H.n_couplings = (int)lv.n_couplings; H.n_convs = (int)convs.size(); H.prior_conv = prior_conv;
+  H.prior_in_m0 = lv.prior_in_m0; H.prior_in_s = lv.prior_in_s; H.ls_lo = lv.ls_lo; H.ls_hi = lv.ls_hi;
+  H.xa_pitch = (int)up(ca, 32); H.x_pitch = maxD; H.mid_pitch = maxK;
+  auto place = [&](size_t bytes) { blob.resize(up((uint32_t)blob.size(), kAlign), 0); uint32_t o = (uint32_t)blob.size(); blob.resize(o + bytes, 0); return o; };
+  blob.clear();
+  place(sizeof(ResHead));
+  H.coupling_off = place(sizeof(ResCouplingRec) * cps.size());
+  H.conv_off = place(sizeof(ResConv) * convs.size());
+  for (uint32_t ki = 0; ki < lv.n_couplings; ++ki) {
+    cps[ki].colA_off = place(4 * (size_t)ca);
+    std::memcpy(blob.data() + cps[ki].colA_off, cols[ki].data(), 4 * (size_t)ca);
+    cps[ki].colB_off = place(4 * (size_t)cb);
+    std::memcpy(blob.data() + cps[ki].colB_off, cols[ki].data() + ca, 4 * (size_t)cb);
+  }
+  // per conv: requantisation constants, index list, nine weight slices
+  size_t block_of_branch = 0;
+  std::vector<const iodf_resblock_desc*> branch_block;
+  for (uint32_t ki = 0; ki < lv.n_couplings; ++ki)
+    for (uint32_t b = 0; b < lv.couplings[ki].n_blocks; ++b) branch_block.push_back(&lv.couplings[ki].blocks[b]);
+  for (size_t ci = 0; ci < convs.size(); ++ci) {
+    ResConv& c = convs[ci];
+    const iodf_layer_desc& L = *conv_layer[ci];
+    c.rq_off = place(sizeof(OutRq) * (size_t)c.n_pad);
+    std::vector<OutRq> rq(c.n_pad, OutRq{1 << 30, 0, 1u << 30, 0u});          // padding: 0 -> 0
+    put_out_rq(rq.data(), L, B);
+    std::memcpy(blob.data() + c.rq_off, rq.data(), sizeof(OutRq) * rq.size());
+    if (c.kind == kResBranch) {
+      const iodf_resblock_desc& rb = *branch_block[block_of_branch++];
+      c.idx_off = place(4 * (size_t)c.n);
+      std::memcpy(blob.data() + c.idx_off, rb.idx, 4 * (size_t)c.n);
+    }
+    c.w_off = place(9 * (size_t)c.slice_bytes);
+    const int8_t* w = B.w + L.weight_off;
+    for (int tap = 0; tap < 9; ++tap) {
+      uint8_t* sl = blob.data() + c.w_off + (size_t)tap * c.slice_bytes;
+      for (int n = 0; n < c.n; ++n)
+        for (uint32_t k = 0; k < L.c_in; ++k)
+          sl[wpos(c.n_pad, n, (int)k)] = (uint8_t)w[((size_t)n * 9 + tap) * L.c_in + k];
+    }
+  }
+  // shared memory: flow variable, the three activation buffers (cleared together at kernel start),
+  // row masks, two A slices, two weight slices
+  const uint32_t pg = up((uint32_t)px, 32);
+  const int ntiles = (px + kTileM - 1) / kTileM;
+  uint32_t off = 0;
+  auto take = [&](uint32_t bytes) { uint32_t o = off; off = up(off + bytes, kAlign); return o; };
+  H.s_v = take((uint32_t)P.c * pg * 4);
+  H.s_xa = take((uint32_t)px * H.xa_pitch);
+  H.s_x = take((uint32_t)px * H.x_pitch);
+  H.s_mid = take((uint32_t)px * H.mid_pitch);
+  H.s_rowinfo = take((uint32_t)ntiles * kTileM * 4);
+  for (int i = 0; i < 2; ++i) H.s_abuf[i] = take((uint32_t)kTileM * kmax);
+  for (int i = 0; i < 2; ++i) H.s_wbuf[i] = take((uint32_t)nmax * kmax);
+  H.s_total = off;
+  H.tmem_cols = ntiles > 1 ? 2 * kResMaxWidth : kResMaxWidth;
+  if (off > smem_limit || ntiles > 2) return IODF_EUNSUPPORTED;
+  std::memcpy(blob.data(), &H, sizeof(H));
+  std::memcpy(blob.data() + H.coupling_off, cps.data(), sizeof(ResCouplingRec) * cps.size());
+  std::memcpy(blob.data() + H.conv_off, convs.data(), sizeof(ResConv) * convs.size());
+  P.residual = 1;
+  P.group = 1; P.pg = (int)pg; P.tiles = ntiles; P.rep = 1; P.nslots = 1;
+  P.s_total = H.s_total;
+  return IODF_OK;
+}
+
 int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_model* m) {
   if (desc->abi_version != IODF_ABI_VERSION) return IODF_EVERSION;
   if (!desc->levels || desc->n_levels < 1 || desc->n_levels > IODF_MAX_LEVELS || desc->max_batch < 1 ||
@@ -429,9 +574,18 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
       for (uint32_t q = 0; q < cp.n_layers; ++q) {
         int rc = check_layer(cp.layers[q], B);
         if (rc) return rc;
-        if (cp.layers[q].c_in != cin) return IODF_EINVAL;
+        if (cp.n_blocks == 0 && cp.layers[q].c_in != cin) return IODF_EINVAL;
         cin = cp.layers[q].c_out;
       }
+      if (cp.n_blocks > 0) {
+        int rc = check_residual(cp, B, ca, cb, px);
+        if (rc) return rc;
+        if (ki > 0 && lv.couplings[0].n_blocks == 0) return IODF_EUNSUPPORTED;    // one kind per level
+        for (uint32_t q = 0; q < cp.n_layers; ++q)
+          lay.macs_per_image += (uint64_t)px * 9 * cp.layers[q].c_in * cp.layers[q].c_out;
+        continue;
+      }
+      if (lv.couplings[0].n_blocks > 0) return IODF_EUNSUPPORTED;
       if (cin != cb) return IODF_EINVAL;
       const iodf_layer_desc& last = cp.layers[cp.n_layers - 1];
       if (last.relu || last.has_clamp) return IODF_EINVAL;
@@ -507,6 +661,22 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
     P.recip_gpb = 65536u / (uint32_t)(P.cbp / 8) + 1u;
     std::vector<int> pi(c);
     for (uint32_t k = 0; k < c; ++k) pi[k] = (int)k;
+    if (lv.n_couplings > 0 && lv.couplings[0].n_blocks > 0) {
+      std::vector<std::vector<int>> cols;
+      for (uint32_t ki = 0; ki < lv.n_couplings; ++ki) {
+        const iodf_coupling_desc& cp = lv.couplings[ki];
+        std::vector<int> nxt(c);
+        for (uint32_t k = 0; k < c; ++k) nxt[k] = pi[cp.perm[k]];
+        pi.swap(nxt);
+        cols.push_back(pi);
+      }
+      for (int k = 0; k < (int)c; ++k) P.col_out[k] = pi[k];
+      int rc = pack_residual_level(lv, B, P, hl.blob, cols, (uint32_t)smem_limit);
+      if (rc) return rc;
+      if ((uint64_t)c * h * w * ((uint64_t)c * h * w) >= (1ull << 32)) return IODF_EUNSUPPORTED;
+      if (lv.split) c = (uint32_t)ca;
+      continue;
+    }
     uint32_t a_bytes = 16, meta = 16, wmax[3] = {16, 16, 16};
     uint32_t n_max = 32;
     std::vector<PackedBlock> blocks;
@@ -571,6 +741,7 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
   // that creating a second, smaller model cannot lower it under a first model's needs.
   (void)max_smem;
   CU(m, configure_level_kernels((uint32_t)smem_limit));
+  CU(m, configure_res_kernels((uint32_t)smem_limit));
   const size_t L = desc->n_levels;
   m->d_plan.assign(L, nullptr); m->d_blob.assign(L, nullptr); m->d_keep.assign(L, nullptr);
   for (size_t li = 0; li < L; ++li) {
@@ -623,7 +794,8 @@ int run_forward(iodf_model* m, const uint8_t* x, int B, int32_t* z, int32_t* pri
     a.status = m->d_status;
     a.batch = B;
     if (li == 0) set_patch_grid(a, grid);
-    CU(m, launch_level(a, false, (B + P.group - 1) / P.group, P.s_total, st));
+    CU(m, P.residual ? launch_res_level(a, false, (B + P.group - 1) / P.group, P.s_total, st)
+                      : launch_level(a, false, (B + P.group - 1) / P.group, P.s_total, st));
     if (timed) CU(m, cudaEventRecord(m->ev[li + 1], st));
   }
   return IODF_OK;
@@ -647,7 +819,8 @@ int launch_inverse_level(iodf_model* m, int li, int phase, const int32_t* z, int
   a.batch = B;
   a.phase = phase;
   if (li == 0) set_patch_grid(a, grid);
-  CU(m, launch_level(a, true, (B + P.group - 1) / P.group, P.s_total, st));
+  CU(m, P.residual ? launch_res_level(a, true, (B + P.group - 1) / P.group, P.s_total, st)
+                    : launch_level(a, true, (B + P.group - 1) / P.group, P.s_total, st));
   return IODF_OK;
 }
 
@@ -769,7 +942,8 @@ int iodf_forward_static(iodf_model* m, const uint8_t* x_u8, int B, int32_t* z, i
     a.oor = nullptr;
     a.status = m->d_status;
     a.batch = B;
-    CU(m, launch_level(a, false, (B + P.group - 1) / P.group, P.s_total, st));
+    CU(m, P.residual ? launch_res_level(a, false, (B + P.group - 1) / P.group, P.s_total, st)
+                      : launch_level(a, false, (B + P.group - 1) / P.group, P.s_total, st));
   }
   return IODF_OK;
 }

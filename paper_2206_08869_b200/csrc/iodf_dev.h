@@ -107,6 +107,9 @@ struct LevelPlan {
                                  // its single tile puts them in the tile rep times (rows r, r + 128/rep, ...),
                                  // so that every TMEM lane quarter holds a copy and the epilogues split the
                                  // accumulator columns over all 16 worker warps instead of 4 * (4 / rep)
+  int32_t residual;              // 1: the level's couplings are residual-block networks (its own kernel; the
+                                 //    level blob then starts with a ResHead and the fields on tiles, slots and
+                                 //    the shared-memory layout below are unused)
   int32_t nslots;                // tiles in flight per CTA: 1 or 2
   int32_t tmem_cols;
   int32_t w13_alias;             // 1: W1 and W3 share a slot and are re-fetched per tile

@@ -1,0 +1,64 @@
+// Flow levels whose couplings use the residual-block network (Eq. 3, Sec. 4.1; scatter add, Sec. 4.5;
+// App. B.1): device-side records and the launch interface. The level's shape, index maps and
+// latent layout are the LevelPlan's; everything about the networks sits in the level blob, headed
+// by a ResHead.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "iodf_dev.h"
+#include "level_kernel.h"
+
+namespace iodf {
+
+constexpr int kResThreads = 512;
+constexpr int kResMaxWidth = 128;      // hidden channels of a residual network (conv outputs), padded to 16
+constexpr int kResMaxPixels = 256;     // pixels per image at a residual level (two 128-row tiles)
+
+// what a conv's epilogue does with its requantised outputs
+enum ResKind : int32_t {
+  kResHidden = 0,     // ReLU + clip to 0..255, written as bytes to the conv's destination buffer
+  kResBranch = 1,     // second conv of a block: added through idx[] to the (already requantised) shortcut in X
+  kResOut = 2,        // last conv: the translation, added to / subtracted from the flow variable
+  kResPrior = 3       // prior head: mu and clipped log-scale index to global memory
+};
+
+// One 3x3 conv. Its nine weight slices (one per tap) are [kpad/16][n_pad][16 bytes] each, back to back.
+struct ResConv {
+  uint32_t w_off;          // blob offset of slice 0
+  uint32_t slice_bytes;    // n_pad * kpad
+  uint32_t rq_off;         // blob offset of OutRq[n_pad] (padding channels requantise 0 to 0)
+  uint32_t idx_off;        // kResBranch: blob offset of int32 idx[n]
+  int32_t n, n_pad;        // outputs, and padded to 16
+  int32_t kpad;            // input bytes per pixel and tap, a multiple of 32 (<= the source's pitch)
+  int32_t a_unsigned;      // input is unsigned 8-bit (hidden activations) or signed (network / head input)
+  int32_t kind;
+  int32_t src, dst;        // buffers: 0 = network input (int8), 1 = X, 2 = MID
+  int32_t short_m0, short_s;   // kResBranch: the block's shortcut requantisation
+  int32_t pad[3];
+};
+static_assert(sizeof(ResConv) == 64, "64-byte records");
+
+struct ResCouplingRec {
+  int32_t in_m0, in_s;
+  uint32_t colA_off, colB_off;   // blob offsets of the physical columns of the coupling's logical channels
+  int32_t conv0, n_convs;        // its convs in the conv array
+  int32_t pad[2];
+};
+
+struct ResHead {
+  int32_t n_couplings, n_convs;
+  int32_t prior_conv;            // index of the prior head's conv, or -1
+  int32_t prior_in_m0, prior_in_s, ls_lo, ls_hi;
+  int32_t xa_pitch, x_pitch, mid_pitch;      // bytes per pixel of the three activation buffers (multiples of 32)
+  uint32_t coupling_off, conv_off;           // blob offsets of ResCouplingRec[] and ResConv[]
+  uint32_t s_v, s_xa, s_x, s_mid, s_rowinfo, s_abuf[2], s_wbuf[2], s_total;   // shared-memory layout
+  int32_t tmem_cols;
+  int32_t pad[9];
+};
+static_assert(sizeof(ResHead) == 128, "128-byte header");
+
+cudaError_t configure_res_kernels(uint32_t max_smem_bytes);
+cudaError_t launch_res_level(const LevelArgs& args, bool inverse, int grid, uint32_t smem_bytes, cudaStream_t stream);
+
+}  // namespace iodf

@@ -102,10 +102,13 @@ def test_gated_models_must_be_compacted():
         G.iodf_create(dense, 4)
 
 
-def test_residual_block_couplings_are_refused_not_misread():
-    """The oracle knows the residual-block coupling network; the CUDA library does not yet: creating
-    such a model must fail with IODF_EUNSUPPORTED instead of running something else."""
+def test_residual_couplings_beyond_the_kernels_limits_are_refused():
+    """Residual-block couplings run for levels of at most 256 pixels per image and widths up to 128;
+    anything else must be refused on the host (IODF_EUNSUPPORTED), a malformed index list is EINVAL."""
+    m = S.make_residual_model(3, 3, 64, 64, [True], 1, 8, 1)          # 1024 pixels at the level
+    assert _status(m) == -6
+    m = S.make_residual_model(3, 3, 8, 8, [True], 1, 136, 1)          # hidden width above 128
+    assert _status(m) == -6
     m = S.make_residual_model(3, 3, 8, 8, [True], 1, 8, 1)
-    with pytest.raises(G.IodfError) as e:
-        G.iodf_create(m, 2)
-    assert e.value.status == -6
+    m["levels"][0]["couplings"][0]["blocks"][0]["idx"][:] = 0
+    assert _status(m) == -1

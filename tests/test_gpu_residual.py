@@ -1,0 +1,79 @@
+"""Couplings with the paper's residual-block network (Eq. 3, scatter add of Sec. 4.5) on the GPU
+against the CPU oracle, bit for bit, through the C ABI: encode, decode, prior parameters and the
+level-stepped decode."""
+import numpy as np
+import pytest
+
+import iodf_synth as S
+import oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def G():
+    import paper_2206_08869_b200 as g
+    g.load_library()
+    return g
+
+
+def _t(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _both_ways(G, model, x):
+    import torch
+    z_ref, p_ref = O.forward(O.Packed(model), x)
+    m = G.iodf_create(model, x.shape[0])
+    z, p = G.iodf_forward(m, _t(x))
+    G.iodf_check(m)
+    np.testing.assert_array_equal(z.cpu().numpy(), z_ref)
+    if p_ref is not None:
+        np.testing.assert_array_equal(p.cpu().numpy(), p_ref)
+    oor = torch.zeros(1, dtype=torch.int32, device="cuda")
+    p2 = torch.empty_like(p) if p is not None else None
+    xr = G.iodf_inverse(m, _t(z_ref), prior=p2, out_of_range=oor)
+    G.iodf_check(m)
+    np.testing.assert_array_equal(xr.cpu().numpy(), x)
+    assert int(oor.item()) == 0
+    if p is not None:
+        assert torch.equal(p, p2)
+    return m, z_ref, p_ref
+
+
+@pytest.mark.parametrize("hw,splits,couplings,hidden,blocks,prune,batch", [
+    (8, [True], 1, 16, 1, None, 2),                       # 16 pixels, one block, nothing pruned
+    (16, [True, True], 2, 24, 2, (0.4, 0.8), 5),          # 64- and 16-pixel levels, odd kept widths
+    (32, [True, True, True], 2, 40, 2, (0.4, 0.7), 3),    # 256 pixels: two tiles per image
+    (16, [True, False], 1, 128, 8, (0.4, 0.7), 2),        # the paper's width and depth: 128 channels, 8 blocks
+])
+def test_residual_models_bit_exact(G, hw, splits, couplings, hidden, blocks, prune, batch):
+    model = S.make_residual_model(0xE500 + hw + hidden, 3, hw, hw, splits, couplings, hidden, blocks, prune=prune)
+    x = S.smooth_field_images(0xE600 + hw, batch, hw, hw, 2.0)
+    _both_ways(G, model, x)
+
+
+def test_residual_and_plain_levels_in_one_model_and_stepped_decode(G):
+    """A model whose first level uses residual couplings and whose second the three-conv couplings;
+    decoded level by level with the blocks that are not decoded yet poisoned."""
+    import torch
+    res = S.make_residual_model(0xE700, 3, 16, 16, [True, True], 2, 32, 2, prune=(0.4, 0.7))
+    plain = S.make_model(0xE701, 3, 16, 16, [True, True], 2, 24, prune=(0.4, 0.7))
+    model = {"in_c": 3, "in_h": 16, "in_w": 16, "levels": [res["levels"][0], plain["levels"][1]]}
+    x = S.smooth_field_images(0xE702, 4, 16, 16, 2.0)
+    m, z_ref, p_ref = _both_ways(G, model, x)
+    lay = G.iodf_get_layout(m)
+    z = torch.full((4, int(lay.d)), 0x7A7A7A7A, dtype=torch.int32, device="cuda")
+    zf = int(lay.z_final_off)
+    z[:, zf:] = _t(z_ref[:, zf:])
+    prior = torch.full((4, 2, int(lay.d_fact)), -1, dtype=torch.int32, device="cuda")
+    xr = torch.zeros((4, 3, 16, 16), dtype=torch.uint8, device="cuda")
+    for lv in (1, 0):
+        G.iodf_inverse_level(m, lv, G.IODF_LEVEL_PRIOR, z, prior=prior)
+        zo, n = int(lay.z_off[lv]), (int(lay.level_c[lv]) // 2) * int(lay.level_h[lv]) * int(lay.level_w[lv])
+        z[:, zo:zo + n] = _t(z_ref[:, zo:zo + n])
+        G.iodf_inverse_level(m, lv, G.IODF_LEVEL_COUPLINGS, z, x_u8=xr if lv == 0 else None)
+    G.iodf_check(m)
+    np.testing.assert_array_equal(prior.cpu().numpy(), p_ref)
+    np.testing.assert_array_equal(xr.cpu().numpy(), x)
