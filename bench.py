@@ -129,9 +129,10 @@ def rank_seed_offset(rank, i):
 
 def workload(args):
     c = S.CONFIGS[args.config]
+    net = ", %d residual blocks per coupling" % c["n_blocks"] if c.get("n_blocks") else ""
     return {"workload": "config %s: ImageNet%d-shaped pruned IODF encode, batch %d of uint8 3x%dx%d, %d levels x %d "
-                        "couplings, hidden %d" % (args.config, c["hw"], args.batch, c["hw"], c["hw"],
-                                                   len(c["splits"]), c["n_couplings"], c["hidden"]),
+                        "couplings, hidden %d%s" % (args.config, c["hw"], args.batch, c["hw"], c["hw"],
+                                                     len(c["splits"]), c["n_couplings"], c["hidden"], net),
             "batch_per_gpu": args.batch, "l2_policy": "rotating %d input/output sets (> L2)" % N_SETS,
             "parallelism": "independent batches per GPU, no collective"}
 
@@ -218,7 +219,7 @@ def main():
     # DRAM bytes of that launch (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture of this
     # workload: profiles/level_kernel_config2_encode.md); only valid for the captured configuration
     traffic = 2.70e6 if (cfg == 2 and B == 128 and top == 0) else None
-    roofline = {"bound": "tensor", "kernel": "level_kernel<encode> level %d" % top, "achieved": achieved,
+    roofline = {"bound": "tensor", "kernel": "%s<encode> level %d" % ("res_level_kernel" if model["levels"][top]["couplings"][0].get("blocks") else "level_kernel", top), "achieved": achieved,
                 "peak": peak_int8, "unit": "TOP/s (int8)", "frac": achieved / peak_int8, "traffic": traffic,
                 "peak_source": "2 x %s burst bf16 %.1f TFLOP/s" % (which, bf16),
                 "level_ms": [float(v) for v in lvl],

@@ -256,11 +256,18 @@ CONFIGS = {
             hidden=256, prune=(0.40, 0.70), prior=True, perm="random"),
     "4s": dict(seed=0x10DF0004, batch=64, hw=64, sigma=4.0, splits=[True] * 4, n_couplings=8,
                hidden=512, prune=None, prior=True, perm="random"),
+    # the paper's own coupling network (App. B.1) on the ImageNet32 geometry: 3 levels x 8 couplings,
+    # each conv3x3 -> 8 gated residual blocks -> conv3x3 on 128 hidden channels, about half pruned
+    "R32": dict(seed=0x10DF0032, batch=64, hw=32, sigma=2.0, splits=[True] * 3, n_couplings=8,
+                hidden=128, prune=(0.40, 0.70), prior=True, perm="random", n_blocks=8),
 }
 
 
 def config_model(idx):
     c = CONFIGS[idx]
+    if c.get("n_blocks"):
+        return make_residual_model(c["seed"], 3, c["hw"], c["hw"], c["splits"], c["n_couplings"], c["hidden"],
+                                   c["n_blocks"], prune=c["prune"], prior=c["prior"])
     return make_model(c["seed"], 3, c["hw"], c["hw"], c["splits"], c["n_couplings"], c["hidden"],
                       prune=c["prune"], prior=c["prior"], perm=c["perm"])
 

@@ -518,8 +518,13 @@ int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P,
   H.s_x = take((uint32_t)px * H.x_pitch);
   H.s_mid = take((uint32_t)px * H.mid_pitch);
   H.s_rowinfo = take((uint32_t)ntiles * kTileM * 4);
+  H.s_tab = take((uint32_t)kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t)));
   for (int i = 0; i < 2; ++i) H.s_abuf[i] = take((uint32_t)kTileM * kmax);
-  for (int i = 0; i < 2; ++i) H.s_wbuf[i] = take((uint32_t)nmax * kmax);
+  // as deep a weight ring as fits (at least two slots)
+  H.w_slot_bytes = up((uint32_t)nmax * kmax, kAlign);
+  H.n_wslots = kResMaxWSlots;
+  while (H.n_wslots > 2 && off + (uint32_t)H.n_wslots * H.w_slot_bytes > smem_limit) --H.n_wslots;
+  H.s_wring = take((uint32_t)H.n_wslots * H.w_slot_bytes);
   H.s_total = off;
   H.tmem_cols = ntiles > 1 ? 2 * kResMaxWidth : kResMaxWidth;
   if (off > smem_limit || ntiles > 2) return IODF_EUNSUPPORTED;

@@ -13,16 +13,18 @@
 //     D[tile] (+)= A * W^T    tcgen05.mma kind::i8, K = kpad, accumulators of all tiles in TMEM
 //   epilogue: TMEM -> exact 64-bit requantisation -> what the conv's kind says (see ResKind)
 //
-// Slices are double-buffered: while the tensor core works on slice g, all threads build slice g+1 and
-// the elected thread has already requested its weights. A block is
+// Slices are double-buffered: while the tensor core works on slice g the builders write slice g+1,
+// and the weights travel through a ring several slices ahead. A block is
 //   MID = clip(ReLU(rq(conv_a(X))))                        kResHidden
 //   X   = rq(X; M_r, s_r)      for all D channels          the shortcut Q(x), in place
 //   X[idx[j]] = clip(max(X[idx[j]] + rq(conv_b(MID))[j], 0), 0, 255)   kResBranch: scatter add + ReLU
 // which equals Eq. 3 with the scatter add because rq(X) of an 8-bit X with a multiplier below one
 // is again in 0..255, and channels that the second conv does not keep only get the shortcut.
 //
-// This is the first, plain version of the path: one thread issues copies and MMAs, phases are
-// separated by CTA barriers, nothing overlaps across convs.
+// Sixteen builder warps write the operand slices and requantise; one more warp's elected lane
+// requests the weight slices and issues the MMAs, so building slice g+1 overlaps issuing slice g.
+// This is a first version of the path: convs run one after another, a conv's epilogue does not
+// overlap the next conv's MMAs.
 #include "res_level.h"
 #include "ptx.cuh"
 
@@ -31,8 +33,9 @@ namespace iodf {
 namespace {
 
 struct __align__(16) ResCtl {
-  uint64_t w_full[2];       // bulk copy -> issuer: weight slice buffer filled
+  uint64_t w_full[kResMaxWSlots];   // bulk copy -> issuer: weight ring slot filled
   uint64_t slice_done[2];   // tensor core -> everyone: the MMAs that read A/W buffer b have completed
+  uint64_t a_full[2];       // builders -> issuer: A slice buffer b written (one arrival per builder warp)
   uint32_t tmem_base;
   uint32_t abort;
 };
@@ -49,6 +52,14 @@ __device__ __noinline__ bool res_wait(ResCtl* ctl, uint32_t* status, uint64_t* b
   *ab = 1;
   atomicExch(status, 1u);
   return false;
+}
+
+// usually the phase has completed already: probe inline before the bounded blocking wait
+__device__ __forceinline__ void res_wait_fast(ResCtl* ctl, uint32_t* status, uint64_t* bar, uint32_t parity) {
+  const uint32_t b = ptx::smem_u32(bar);
+  for (int it = 0; it < 64; ++it)
+    if (ptx::mbar_test_wait(b, parity)) return;
+  res_wait(ctl, status, bar, parity);
 }
 
 __device__ __forceinline__ int rdiv(int n, uint32_t mul) { return mul ? (int)__umulhi((uint32_t)n, mul) : n; }
@@ -95,6 +106,7 @@ struct Run {
   int ntiles;
   uint32_t tmem;
   uint32_t gslice;          // slices issued so far (buffer = gslice & 1, use count = gslice >> 1)
+  uint32_t gload;           // weight slices requested so far (ring slot = gload % n_wslots), issuing thread only
   int32_t* v;
   const uint32_t* rowinfo;
 };
@@ -112,19 +124,78 @@ __device__ void conv_mma(Run& r, const ResConv& c) {
   const int pitch = pitch_of(r, c.src);
   const int nchunks = c.kpad >> 4;
   const uint32_t idesc = ptx::umma_idesc_i8((uint32_t)c.n_pad, c.a_unsigned != 0);
+  // Weight slices travel through a ring of n_wslots slots, requested n_wslots - 2 slices ahead of
+  // their use so that the L2 latency of the copies is off the slice loop. Slice number `g` of the
+  // kernel uses ring slot g % n_wslots; a slot is free once the MMAs of the slice that used it last
+  // have completed, which the wait at the top of a slice guarantees for every slice up to g - 2.
+  const int nslices = r.ntiles * 9;
+  const uint32_t nws = (uint32_t)r.H->n_wslots, ahead = nws - 2u;
+  const uint32_t g0 = r.gslice;
+  if (r.warp == kResBuilderWarps) {
+    // ---- issuing warp: weight copies and MMAs; the builders run one slice ahead of it ----
+    if (r.lane == 0) {
+      auto request = [&](int sidx) {                // weights of the conv's slice sidx
+        const uint32_t slot = r.gload % nws;
+        const uint32_t bar = ptx::smem_u32(&r.ctl->w_full[slot]);
+        ptx::mbar_expect_tx(bar, c.slice_bytes);
+        ptx::bulk_g2s(ptx::smem_u32(r.smem + r.H->s_wring + slot * r.H->w_slot_bytes),
+                      r.blob + c.w_off + (size_t)(sidx % 9) * c.slice_bytes, c.slice_bytes, bar);
+        ++r.gload;
+      };
+      // every earlier slice has completed (the previous conv ended with a CTA barrier): the ring is free
+      for (int sidx = 0; sidx < nslices && sidx < (int)ahead; ++sidx) request(sidx);
+      for (int tile = 0; tile < r.ntiles; ++tile)
+        for (int tap = 0; tap < 9; ++tap) {
+          const uint32_t g = r.gslice++;
+          const int b = (int)(g & 1u);
+          const uint32_t use = g >> 1;
+          const int sidx = (int)(g - g0);
+          if (sidx + (int)ahead < nslices) {
+            // its ring slot was last read by slice g - 2
+            if (use > 0) res_wait_fast(r.ctl, r.status, &r.ctl->slice_done[b], (use - 1u) & 1u);
+            request(sidx + (int)ahead);
+          }
+          res_wait_fast(r.ctl, r.status, &r.ctl->a_full[b], use & 1u);
+          const uint32_t wslot = g % nws;
+          res_wait_fast(r.ctl, r.status, &r.ctl->w_full[wslot], (g / nws) & 1u);
+          ptx::tc_fence_after();
+          const uint32_t sa = ptx::smem_u32(r.smem + r.H->s_abuf[b]);
+          const uint32_t sb = ptx::smem_u32(r.smem + r.H->s_wring + wslot * r.H->w_slot_bytes);
+          const uint32_t lbo_b = (uint32_t)c.n_pad * 16u;
+          const uint32_t d = r.tmem + (uint32_t)(tile * kResMaxWidth);
+          for (int k = 0; k < (c.kpad >> 5); ++k) {
+            const uint64_t da = ptx::umma_desc(sa + (uint32_t)k * 2u * (kTileM * 16), kTileM * 16, 128);
+            const uint64_t db = ptx::umma_desc(sb + (uint32_t)k * 2u * lbo_b, lbo_b, 128);
+            ptx::umma_i8(d, da, db, idesc, (tap > 0 || k > 0) ? 1u : 0u);
+          }
+          ptx::umma_commit(ptx::smem_u32(&r.ctl->slice_done[b]));
+        }
+    } else {
+      r.gslice += (uint32_t)nslices;
+    }
+    __syncwarp();
+    return;
+  }
+  // ---- builders ----
+  // the conv's requantisation constants and index list move to shared memory while the slices run
+  // (the previous conv's epilogue, their last reader, ended with a CTA barrier)
+  {
+    uint4* tab = reinterpret_cast<uint4*>(r.smem + r.H->s_tab);
+    const uint4* src_rq = reinterpret_cast<const uint4*>(r.blob + c.rq_off);
+    for (int i = r.tid; i < c.n_pad; i += kResThreads) tab[i] = src_rq[i];
+    if (c.kind == kResBranch) {
+      int32_t* ti = reinterpret_cast<int32_t*>(tab + kResMaxWidth);
+      const int32_t* si = reinterpret_cast<const int32_t*>(r.blob + c.idx_off);
+      for (int i = r.tid; i < c.n; i += kResThreads) ti[i] = si[i];
+    }
+  }
   for (int tile = 0; tile < r.ntiles; ++tile) {
     for (int tap = 0; tap < 9; ++tap) {
       const uint32_t g = r.gslice++;
       const int b = (int)(g & 1u);
       const uint32_t use = g >> 1;                      // how often buffer b has been used before
       // the MMAs that last read buffer b must have completed before it is overwritten
-      if (use > 0) res_wait(r.ctl, r.status, &r.ctl->slice_done[b], (use - 1u) & 1u);
-      if (r.tid == 0) {
-        const uint32_t bar = ptx::smem_u32(&r.ctl->w_full[b]);
-        ptx::mbar_expect_tx(bar, c.slice_bytes);
-        ptx::bulk_g2s(ptx::smem_u32(r.smem + r.H->s_wbuf[b]), r.blob + c.w_off + (size_t)tap * c.slice_bytes,
-                      c.slice_bytes, bar);
-      }
+      if (use > 0) res_wait_fast(r.ctl, r.status, &r.ctl->slice_done[b], (use - 1u) & 1u);
       uint8_t* abuf = r.smem + r.H->s_abuf[b];
       const int off = ((tap * 11) >> 5) - 1;            // u - 1
       const int shift = off * r.g.w + (tap - (off + 1) * 3 - 1);
@@ -137,27 +208,17 @@ __device__ void conv_mma(Run& r, const ResConv& c) {
         *reinterpret_cast<uint4*>(abuf + (size_t)ch * (kTileM * 16) + row * 16) = val;
       }
       ptx::fence_async_smem();
-      __syncthreads();
-      if (r.tid == 0) {
-        res_wait(r.ctl, r.status, &r.ctl->w_full[b], use & 1u);
-        ptx::tc_fence_after();
-        const uint32_t sa = ptx::smem_u32(abuf), sb = ptx::smem_u32(r.smem + r.H->s_wbuf[b]);
-        const uint32_t lbo_b = (uint32_t)c.n_pad * 16u;
-        const uint32_t d = r.tmem + (uint32_t)(tile * kResMaxWidth);
-        for (int k = 0; k < (c.kpad >> 5); ++k) {
-          const uint64_t da = ptx::umma_desc(sa + (uint32_t)k * 2u * (kTileM * 16), kTileM * 16, 128);
-          const uint64_t db = ptx::umma_desc(sb + (uint32_t)k * 2u * lbo_b, lbo_b, 128);
-          ptx::umma_i8(d, da, db, idesc, (tap > 0 || k > 0) ? 1u : 0u);
-        }
-        ptx::umma_commit(ptx::smem_u32(&r.ctl->slice_done[b]));
-      }
+      __syncwarp();
+      if (r.lane == 0)
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ptx::smem_u32(&r.ctl->a_full[b])) : "memory");
     }
   }
   // the last two slices (one per buffer) close the conv
   const uint32_t g = r.gslice;
-  if (g >= 1) res_wait(r.ctl, r.status, &r.ctl->slice_done[(g - 1) & 1u], (((g - 1) >> 1)) & 1u);
-  if (g >= 2) res_wait(r.ctl, r.status, &r.ctl->slice_done[(g - 2) & 1u], (((g - 2) >> 1)) & 1u);
+  if (g >= 1) res_wait_fast(r.ctl, r.status, &r.ctl->slice_done[(g - 1) & 1u], (((g - 1) >> 1)) & 1u);
+  if (g >= 2) res_wait_fast(r.ctl, r.status, &r.ctl->slice_done[(g - 2) & 1u], (((g - 2) >> 1)) & 1u);
   ptx::tc_fence_after();
+  asm volatile("bar.sync 1, %0;" ::"n"(kResThreads) : "memory");      // builders only: the staged tables are complete
 }
 
 struct StepIo {            // what the epilogue of the last conv / the prior head needs
@@ -169,13 +230,13 @@ struct StepIo {            // what the epilogue of the last conv / the prior hea
 };
 
 __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
-  const OutRq* orq = reinterpret_cast<const OutRq*>(r.blob + c.rq_off);
-  const int32_t* idx = reinterpret_cast<const int32_t*>(r.blob + c.idx_off);
+  const OutRq* orq = reinterpret_cast<const OutRq*>(r.smem + r.H->s_tab);          // staged by conv_mma
+  const int32_t* idx = reinterpret_cast<const int32_t*>(r.smem + r.H->s_tab + kResMaxWidth * sizeof(OutRq));
   const int q = r.warp & 3, split = r.warp >> 2, nsplit = kResThreads / 128;
   const int nch = c.n_pad >> 4;
   uint8_t* dst = buf_of(r, c.dst);
   const int dpitch = pitch_of(r, c.dst);
-  for (int tile = 0; tile < r.ntiles; ++tile) {
+  for (int tile = 0; tile < (r.warp < kResBuilderWarps ? r.ntiles : 0); ++tile) {
     const int p = tile * kTileM + q * 32 + r.lane;
     const bool valid = p < r.g.px;
     for (int ch = split; ch < nch; ch += nsplit) {
@@ -228,7 +289,7 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
 __device__ void requant_input(Run& r, const int32_t* cols, int n, int32_t m0, int32_t s) {
   int8_t* xa = reinterpret_cast<int8_t*>(r.smem + r.H->s_xa);
   const int pitch = r.H->xa_pitch;
-  for (int it = r.tid; it < n * r.g.px; it += kResThreads) {
+  for (int it = r.tid; it < (r.warp < kResBuilderWarps ? n * r.g.px : 0); it += kResThreads) {
     const int c = it / r.g.px, p = it - c * r.g.px;
     xa[(size_t)p * pitch + c] = (int8_t)clampi(rq64(r.v[cols[c] * r.g.pg + p], m0, s), -128, 127);
   }
@@ -236,7 +297,7 @@ __device__ void requant_input(Run& r, const int32_t* cols, int n, int32_t m0, in
 }
 
 template <bool kInv>
-__global__ void __launch_bounds__(kResThreads, 1) res_level_kernel(const LevelArgs a) {
+__global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const LevelArgs a) {
   extern __shared__ __align__(1024) uint8_t smem[];
   __shared__ ResCtl ctl;
   const LevelPlan& P = *a.plan;
@@ -244,9 +305,10 @@ __global__ void __launch_bounds__(kResThreads, 1) res_level_kernel(const LevelAr
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
+    for (int s = 0; s < kResMaxWSlots; ++s) ptx::mbar_init(ptx::smem_u32(&ctl.w_full[s]), 1);
     for (int s = 0; s < 2; ++s) {
-      ptx::mbar_init(ptx::smem_u32(&ctl.w_full[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&ctl.slice_done[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl.a_full[s]), (uint32_t)kResBuilderWarps);
     }
     ptx::mbar_init_fence();
     ctl.abort = 0;
@@ -263,18 +325,20 @@ __global__ void __launch_bounds__(kResThreads, 1) res_level_kernel(const LevelAr
   r.ntiles = (P.px + kTileM - 1) / kTileM;
   r.tmem = ctl.tmem_base;
   r.gslice = 0;
+  r.gload = 0;
   r.v = reinterpret_cast<int32_t*>(smem + H->s_v);
   uint32_t* rowinfo = reinterpret_cast<uint32_t*>(smem + H->s_rowinfo);
   r.rowinfo = rowinfo;
 
   const int c = P.c, px = P.px, pg = P.pg, w = P.w;
   const int b = blockIdx.x;                       // one image per CTA
-  const int per_img = c * px;
+  const bool builder = warp < kResBuilderWarps;
+  const int per_img = builder ? c * px : 0;       // the issuing warp takes no part in the element loops
   int32_t* v = r.v;
-  for (int i = tid; i < r.ntiles * kTileM; i += kResThreads) rowinfo[i] = gather_mask(i, r.g);
+  for (int i = tid; i < (builder ? r.ntiles * kTileM : 0); i += kResThreads) rowinfo[i] = gather_mask(i, r.g);
   // activation buffers start at zero: padding channels and bytes beyond a conv's outputs stay zero
   // or meet zero weights
-  for (uint32_t i = H->s_xa + tid * 16; i < H->s_rowinfo; i += kResThreads * 16)
+  for (uint32_t i = H->s_xa + tid * 16; builder && i < H->s_rowinfo; i += kResThreads * 16)
     *reinterpret_cast<uint4*>(smem + i) = make_uint4(0u, 0u, 0u, 0u);
 
   if (!kInv) {
@@ -333,7 +397,7 @@ __global__ void __launch_bounds__(kResThreads, 1) res_level_kernel(const LevelAr
         // the shortcut Q(x) of all channels, in place (the first conv of the block has read X already)
         uint8_t* X = smem + H->s_x;
         const int words = H->x_pitch >> 2;
-        for (int it = tid; it < px * words; it += kResThreads) {
+        for (int it = tid; it < (builder ? px * words : 0); it += kResThreads) {
           uint32_t* wp = reinterpret_cast<uint32_t*>(X) + it;
           const uint32_t in = *wp;
           uint32_t out = 0;
@@ -390,8 +454,8 @@ __global__ void __launch_bounds__(kResThreads, 1) res_level_kernel(const LevelAr
 }  // namespace
 
 cudaError_t launch_res_level(const LevelArgs& args, bool inverse, int grid, uint32_t smem_bytes, cudaStream_t stream) {
-  if (inverse) res_level_kernel<true><<<grid, kResThreads, smem_bytes, stream>>>(args);
-  else res_level_kernel<false><<<grid, kResThreads, smem_bytes, stream>>>(args);
+  if (inverse) res_level_kernel<true><<<grid, kResAllThreads, smem_bytes, stream>>>(args);
+  else res_level_kernel<false><<<grid, kResAllThreads, smem_bytes, stream>>>(args);
   return cudaGetLastError();
 }
 
