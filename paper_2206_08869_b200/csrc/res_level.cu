@@ -142,6 +142,14 @@ __device__ void conv_mma(Run& r, const ResConv& c) {
                       r.blob + c.w_off + (size_t)(sidx % 9) * c.slice_bytes, c.slice_bytes, bar);
         ++r.gload;
       };
+      // operand descriptors: low words (start address, leading-dimension offset) and their K steps
+      const uint32_t lbo_b = (uint32_t)c.n_pad * 16u;
+      const uint32_t da_lo[2] = {ptx::umma_desc_lo(ptx::smem_u32(r.smem + r.H->s_abuf[0]), kTileM * 16),
+                                 ptx::umma_desc_lo(ptx::smem_u32(r.smem + r.H->s_abuf[1]), kTileM * 16)};
+      const uint32_t db_lo0 = ptx::umma_desc_lo(ptx::smem_u32(r.smem + r.H->s_wring), lbo_b);
+      const uint32_t db_slot = r.H->w_slot_bytes >> 4;
+      const uint32_t da_step = (2u * kTileM * 16u) >> 4, db_step = (2u * lbo_b) >> 4;
+      const int ksteps = c.kpad >> 5;
       // every earlier slice has completed (the previous conv ended with a CTA barrier): the ring is free
       for (int sidx = 0; sidx < nslices && sidx < (int)ahead; ++sidx) request(sidx);
       for (int tile = 0; tile < r.ntiles; ++tile)
@@ -159,14 +167,13 @@ __device__ void conv_mma(Run& r, const ResConv& c) {
           const uint32_t wslot = g % nws;
           res_wait_fast(r.ctl, r.status, &r.ctl->w_full[wslot], (g / nws) & 1u);
           ptx::tc_fence_after();
-          const uint32_t sa = ptx::smem_u32(r.smem + r.H->s_abuf[b]);
-          const uint32_t sb = ptx::smem_u32(r.smem + r.H->s_wring + wslot * r.H->w_slot_bytes);
-          const uint32_t lbo_b = (uint32_t)c.n_pad * 16u;
+          uint32_t da = da_lo[b], db = db_lo0 + wslot * db_slot;
           const uint32_t d = r.tmem + (uint32_t)(tile * kResMaxWidth);
-          for (int k = 0; k < (c.kpad >> 5); ++k) {
-            const uint64_t da = ptx::umma_desc(sa + (uint32_t)k * 2u * (kTileM * 16), kTileM * 16, 128);
-            const uint64_t db = ptx::umma_desc(sb + (uint32_t)k * 2u * lbo_b, lbo_b, 128);
-            ptx::umma_i8(d, da, db, idesc, (tap > 0 || k > 0) ? 1u : 0u);
+          ptx::umma_i8_lo(d, da, db, idesc, tap > 0 ? 1u : 0u);
+          for (int k = 1; k < ksteps; ++k) {
+            da += da_step;
+            db += db_step;
+            ptx::umma_i8_lo(d, da, db, idesc, 1u);
           }
           ptx::umma_commit(ptx::smem_u32(&r.ctl->slice_done[b]));
         }
@@ -195,7 +202,10 @@ __device__ void conv_mma(Run& r, const ResConv& c) {
       const int b = (int)(g & 1u);
       const uint32_t use = g >> 1;                      // how often buffer b has been used before
       // the MMAs that last read buffer b must have completed before it is overwritten
-      if (use > 0) res_wait_fast(r.ctl, r.status, &r.ctl->slice_done[b], (use - 1u) & 1u);
+      // (suspended wait: the builders run ahead of the issuing thread, and a spinning warp would take
+      // issue slots from it)
+      if (use > 0 && !ptx::mbar_test_wait(ptx::smem_u32(&r.ctl->slice_done[b]), (use - 1u) & 1u))
+        res_wait(r.ctl, r.status, &r.ctl->slice_done[b], (use - 1u) & 1u);
       uint8_t* abuf = r.smem + r.H->s_abuf[b];
       const int off = ((tap * 11) >> 5) - 1;            // u - 1
       const int shift = off * r.g.w + (tap - (off + 1) * 3 - 1);
