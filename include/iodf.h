@@ -153,7 +153,8 @@ typedef struct iodf_model iodf_model;
  * EOVERFLOW, EVERSION, ENOMEM, ECUDA, EUNSUPPORTED. This build runs couplings of the form
  * conv3x3+ReLU+clip -> conv1x1+ReLU+clip -> conv3x3 with hidden activations inside the signed
  * 8-bit range and hidden widths up to 512 kept channels (above 256 the weights are streamed from
- * L2 for every tile instead of staying in shared memory), and 3x3 prior heads.
+ * L2 for every tile instead of staying in shared memory), couplings with residual blocks (see
+ * iodf_coupling_desc) at levels of at most 256 pixels per image, and 3x3 prior heads.
  */
 int iodf_create(const iodf_model_desc* desc, const int8_t* weights, size_t weights_count,
                 const int32_t* requant, size_t requant_count, int device, iodf_model** out);
