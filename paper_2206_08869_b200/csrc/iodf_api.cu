@@ -507,27 +507,29 @@ int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P,
           sl[wpos(c.n_pad, n, (int)k)] = (uint8_t)w[((size_t)n * 9 + tap) * L.c_in + k];
     }
   }
-  // shared memory: flow variable, the three activation buffers (cleared together at kernel start),
-  // row masks, two A slices, two weight slices
+  // shared memory: flow variable, the three activation buffers in the padded chunk-major layout
+  // (cleared together at kernel start), position table, conv tables, weight ring
   const uint32_t pg = up((uint32_t)px, 32);
-  const int ntiles = (px + kTileM - 1) / kTileM;
+  const int w2 = P.w + 2, guard = w2 + 1;
+  const int ntiles = (int)(up((uint32_t)((P.h + 2) * w2), kTileM) / kTileM);
+  const int rows = guard + ntiles * kTileM + w2 + 1;
+  H.w2 = w2; H.guard = guard; H.rows = rows; H.ntiles = ntiles;
   uint32_t off = 0;
   auto take = [&](uint32_t bytes) { uint32_t o = off; off = up(off + bytes, kAlign); return o; };
   H.s_v = take((uint32_t)P.c * pg * 4);
-  H.s_xa = take((uint32_t)px * H.xa_pitch);
-  H.s_x = take((uint32_t)px * H.x_pitch);
-  H.s_mid = take((uint32_t)px * H.mid_pitch);
+  H.s_xa = take((uint32_t)(H.xa_pitch / 16) * rows * 16);
+  H.s_x = take((uint32_t)(H.x_pitch / 16) * rows * 16);
+  H.s_mid = take((uint32_t)(H.mid_pitch / 16) * rows * 16);
   H.s_rowinfo = take((uint32_t)ntiles * kTileM * 4);
   H.s_tab = take((uint32_t)kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t)));
-  for (int i = 0; i < 2; ++i) H.s_abuf[i] = take((uint32_t)kTileM * kmax);
   // as deep a weight ring as fits (at least two slots)
   H.w_slot_bytes = up((uint32_t)nmax * kmax, kAlign);
   H.n_wslots = kResMaxWSlots;
   while (H.n_wslots > 2 && off + (uint32_t)H.n_wslots * H.w_slot_bytes > smem_limit) --H.n_wslots;
   H.s_wring = take((uint32_t)H.n_wslots * H.w_slot_bytes);
   H.s_total = off;
-  H.tmem_cols = ntiles > 1 ? 2 * kResMaxWidth : kResMaxWidth;
-  if (off > smem_limit || ntiles > 2) return IODF_EUNSUPPORTED;
+  H.tmem_cols = ntiles > 2 ? 4 * kResMaxWidth : (ntiles > 1 ? 2 * kResMaxWidth : kResMaxWidth);
+  if (off > smem_limit || ntiles > 4 || rows * 16 >= (1 << 18)) return IODF_EUNSUPPORTED;
   std::memcpy(blob.data(), &H, sizeof(H));
   std::memcpy(blob.data() + H.coupling_off, cps.data(), sizeof(ResCouplingRec) * cps.size());
   std::memcpy(blob.data() + H.conv_off, convs.data(), sizeof(ResConv) * convs.size());

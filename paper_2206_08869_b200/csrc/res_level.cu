@@ -3,26 +3,28 @@
 // channels), one CTA per image, images of at most 256 pixels at this level.
 //
 // Every conv here is a 3x3 conv over hidden activations, so a pixel needs its neighbours' hidden
-// values: the activations of the whole image stay in shared memory (X: the block tensor, D channels;
-// MID: the first conv's output; both unsigned 8-bit, pixel-major) and a conv is
+// values: the activations of the whole image stay in shared memory (xa: the requantised network
+// input, X: the block tensor of D channels, MID: the first conv's output; 8-bit). They are stored
+// the way tcgen05.mma reads a K-major operand without swizzle, [channel chunk of 16][row][16 bytes],
+// with the image laid out in rows of w + 2 positions (a zero column on either side, a zero row
+// above and below, and w + 3 guard positions before and after). A conv tap (u, v) is then nothing
+// but a row offset (u-1)(w+2) + (v-1) of the operand's start address: no operand is ever built.
 //
-//   for each 128-pixel tile, for each tap (u, v):
-//     A slice  [128 x kpad]   rows = the tile's pixels shifted by the tap (zero outside the image),
-//                             copied from the source buffer into the MMA operand layout
-//     W slice  [n_pad x kpad] the tap's weights, bulk-copied from the packed blob (L2)
-//     D[tile] (+)= A * W^T    tcgen05.mma kind::i8, K = kpad, accumulators of all tiles in TMEM
-//   epilogue: TMEM -> exact 64-bit requantisation -> what the conv's kind says (see ResKind)
+//   for each tap, for each 128-position tile, for each 32 channels:
+//       D[tile] (+)= A(buffer, tile rows shifted by the tap) * W(tap)^T      tcgen05.mma kind::i8
+//   epilogue: TMEM -> exact 64-bit requantisation -> what the conv's kind says (see ResKind);
+//   results are stored at the image's positions only, so the padding stays zero.
 //
-// Slices are double-buffered: while the tensor core works on slice g the builders write slice g+1,
-// and the weights travel through a ring several slices ahead. A block is
+// The (h+2)(w+2) positions are computed in full (outputs at padding positions are discarded): a
+// third more rows than pixels at 16x16, bought with tensor time that is idle anyway. One lane of a
+// 17th warp requests the taps' weight slices from the packed blob (a ring, several slices ahead)
+// and issues the MMAs of a conv back to back; the 16 other warps requantise. A block is
 //   MID = clip(ReLU(rq(conv_a(X))))                        kResHidden
 //   X   = rq(X; M_r, s_r)      for all D channels          the shortcut Q(x), in place
 //   X[idx[j]] = clip(max(X[idx[j]] + rq(conv_b(MID))[j], 0), 0, 255)   kResBranch: scatter add + ReLU
 // which equals Eq. 3 with the scatter add because rq(X) of an 8-bit X with a multiplier below one
 // is again in 0..255, and channels that the second conv does not keep only get the shortcut.
 //
-// Sixteen builder warps write the operand slices and requantise; one more warp's elected lane
-// requests the weight slices and issues the MMAs, so building slice g+1 overlaps issuing slice g.
 // This is a first version of the path: convs run one after another, a conv's epilogue does not
 // overlap the next conv's MMAs.
 #include "res_level.h"
@@ -34,8 +36,8 @@ namespace {
 
 struct __align__(16) ResCtl {
   uint64_t w_full[kResMaxWSlots];   // bulk copy -> issuer: weight ring slot filled
-  uint64_t slice_done[2];   // tensor core -> everyone: the MMAs that read A/W buffer b have completed
-  uint64_t a_full[2];       // builders -> issuer: A slice buffer b written (one arrival per builder warp)
+  uint64_t w_empty[kResMaxWSlots];  // tensor core -> issuer: the MMAs that read ring slot s have completed
+  uint64_t conv_done;       // tensor core -> requantising warps: every MMA of the running conv has completed
   uint32_t tmem_base;
   uint32_t abort;
 };
@@ -82,19 +84,6 @@ struct Geo {
   uint32_t mul_w;
 };
 
-// bit t = u*3+v of the mask: input pixel (i+u-1, j+v-1) is inside the image
-__device__ __forceinline__ uint32_t gather_mask(int p, const Geo& g) {
-  if (p >= g.px) return 0u;
-  const int i = rdiv(p, g.mul_w), j = p - i * g.w;
-  uint32_t m = 0;
-#pragma unroll
-  for (int u = 0; u < 3; ++u)
-#pragma unroll
-    for (int v = 0; v < 3; ++v)
-      if (i + u - 1 >= 0 && i + u - 1 < g.h && j + v - 1 >= 0 && j + v - 1 < g.w) m |= 1u << (u * 3 + v);
-  return m;
-}
-
 struct Run {
   uint8_t* smem;
   ResCtl* ctl;
@@ -105,87 +94,75 @@ struct Run {
   int tid, warp, lane;
   int ntiles;
   uint32_t tmem;
-  uint32_t gslice;          // slices issued so far (buffer = gslice & 1, use count = gslice >> 1)
-  uint32_t gload;           // weight slices requested so far (ring slot = gload % n_wslots), issuing thread only
+  uint32_t gslice;          // weight slices consumed so far (ring slot = gslice % n_wslots), issuing lane only
+  uint32_t gload;           // weight slices requested so far, issuing lane only
+  uint32_t nconv;           // convs run so far (parity of conv_done)
   int32_t* v;
-  const uint32_t* rowinfo;
+  const int32_t* pixel_of;  // pixel index of a padded position, -1 at padding
 };
 
 __device__ __forceinline__ uint8_t* buf_of(const Run& r, int which) {
   return r.smem + (which == 0 ? r.H->s_xa : (which == 1 ? r.H->s_x : r.H->s_mid));
 }
-__device__ __forceinline__ int pitch_of(const Run& r, int which) {
-  return which == 0 ? r.H->xa_pitch : (which == 1 ? r.H->x_pitch : r.H->mid_pitch);
+// byte address of channel c at padded position rr (0 = first computed position) of a buffer
+__device__ __forceinline__ uint8_t* at(const Run& r, uint8_t* buf, int c, int rr) {
+  return buf + ((size_t)(c >> 4) * r.H->rows + r.H->guard + rr) * 16 + (c & 15);
 }
 
-// All nine taps of all tiles: accumulators D[tile][0 .. n_pad) complete in TMEM on return.
+// All nine taps of all tiles: accumulators D[tile][0 .. n_pad) complete in TMEM on return (for the
+// requantising warps; the issuing warp returns as soon as everything is issued).
 __device__ void conv_mma(Run& r, const ResConv& c) {
-  const uint8_t* src = buf_of(r, c.src);
-  const int pitch = pitch_of(r, c.src);
-  const int nchunks = c.kpad >> 4;
-  const uint32_t idesc = ptx::umma_idesc_i8((uint32_t)c.n_pad, c.a_unsigned != 0);
-  // Weight slices travel through a ring of n_wslots slots, requested n_wslots - 2 slices ahead of
-  // their use so that the L2 latency of the copies is off the slice loop. Slice number `g` of the
-  // kernel uses ring slot g % n_wslots; a slot is free once the MMAs of the slice that used it last
-  // have completed, which the wait at the top of a slice guarantees for every slice up to g - 2.
-  const int nslices = r.ntiles * 9;
-  const uint32_t nws = (uint32_t)r.H->n_wslots, ahead = nws - 2u;
-  const uint32_t g0 = r.gslice;
+  const uint32_t parity = r.nconv & 1u;
+  ++r.nconv;
   if (r.warp == kResBuilderWarps) {
-    // ---- issuing warp: weight copies and MMAs; the builders run one slice ahead of it ----
     if (r.lane == 0) {
-      auto request = [&](int sidx) {                // weights of the conv's slice sidx
-        const uint32_t slot = r.gload % nws;
+      const uint32_t nws = (uint32_t)r.H->n_wslots, ahead = nws - 1u;
+      auto request = [&](int tap) {
+        const uint32_t gl = r.gload++;
+        const uint32_t slot = gl % nws, use = gl / nws;
+        // the slice that used this slot last must have been consumed
+        if (use > 0) res_wait_fast(r.ctl, r.status, &r.ctl->w_empty[slot], (use - 1u) & 1u);
         const uint32_t bar = ptx::smem_u32(&r.ctl->w_full[slot]);
         ptx::mbar_expect_tx(bar, c.slice_bytes);
         ptx::bulk_g2s(ptx::smem_u32(r.smem + r.H->s_wring + slot * r.H->w_slot_bytes),
-                      r.blob + c.w_off + (size_t)(sidx % 9) * c.slice_bytes, c.slice_bytes, bar);
-        ++r.gload;
+                      r.blob + c.w_off + (size_t)tap * c.slice_bytes, c.slice_bytes, bar);
       };
-      // operand descriptors: low words (start address, leading-dimension offset) and their K steps
-      const uint32_t lbo_b = (uint32_t)c.n_pad * 16u;
-      const uint32_t da_lo[2] = {ptx::umma_desc_lo(ptx::smem_u32(r.smem + r.H->s_abuf[0]), kTileM * 16),
-                                 ptx::umma_desc_lo(ptx::smem_u32(r.smem + r.H->s_abuf[1]), kTileM * 16)};
-      const uint32_t db_lo0 = ptx::umma_desc_lo(ptx::smem_u32(r.smem + r.H->s_wring), lbo_b);
-      const uint32_t db_slot = r.H->w_slot_bytes >> 4;
-      const uint32_t da_step = (2u * kTileM * 16u) >> 4, db_step = (2u * lbo_b) >> 4;
+      for (int tap = 0; tap < 9 && tap < (int)ahead; ++tap) request(tap);
+      const uint32_t idesc = ptx::umma_idesc_i8((uint32_t)c.n_pad, c.a_unsigned != 0);
+      const uint32_t rows = (uint32_t)r.H->rows;
+      // operand start addresses in 16-byte units
+      const uint32_t a0 = (ptx::smem_u32(buf_of(r, c.src)) >> 4) + (uint32_t)r.H->guard;
+      const uint32_t ring0 = ptx::smem_u32(r.smem + r.H->s_wring) >> 4, slot16 = r.H->w_slot_bytes >> 4;
+      const uint32_t a_hi = (rows & 0x3FFFu) << 16, b_hi = ((uint32_t)c.n_pad & 0x3FFFu) << 16;
       const int ksteps = c.kpad >> 5;
-      // every earlier slice has completed (the previous conv ended with a CTA barrier): the ring is free
-      for (int sidx = 0; sidx < nslices && sidx < (int)ahead; ++sidx) request(sidx);
-      for (int tile = 0; tile < r.ntiles; ++tile)
-        for (int tap = 0; tap < 9; ++tap) {
-          const uint32_t g = r.gslice++;
-          const int b = (int)(g & 1u);
-          const uint32_t use = g >> 1;
-          const int sidx = (int)(g - g0);
-          if (sidx + (int)ahead < nslices) {
-            // its ring slot was last read by slice g - 2
-            if (use > 0) res_wait_fast(r.ctl, r.status, &r.ctl->slice_done[b], (use - 1u) & 1u);
-            request(sidx + (int)ahead);
-          }
-          res_wait_fast(r.ctl, r.status, &r.ctl->a_full[b], use & 1u);
-          const uint32_t wslot = g % nws;
-          res_wait_fast(r.ctl, r.status, &r.ctl->w_full[wslot], (g / nws) & 1u);
-          ptx::tc_fence_after();
-          uint32_t da = da_lo[b], db = db_lo0 + wslot * db_slot;
+      ptx::tc_fence_after();
+      for (int tap = 0; tap < 9; ++tap) {
+        if (tap + (int)ahead < 9) request(tap + (int)ahead);
+        const uint32_t g = r.gslice++;
+        const uint32_t slot = g % nws;
+        res_wait_fast(r.ctl, r.status, &r.ctl->w_full[slot], (g / nws) & 1u);
+        ptx::tc_fence_after();
+        const int u = (tap * 11) >> 5;
+        const int shift = (u - 1) * r.H->w2 + (tap - u * 3 - 1);
+        for (int tile = 0; tile < r.ntiles; ++tile) {
           const uint32_t d = r.tmem + (uint32_t)(tile * kResMaxWidth);
-          ptx::umma_i8_lo(d, da, db, idesc, tap > 0 ? 1u : 0u);
-          for (int k = 1; k < ksteps; ++k) {
-            da += da_step;
-            db += db_step;
-            ptx::umma_i8_lo(d, da, db, idesc, 1u);
+          uint32_t sa = a0 + (uint32_t)(tile * kTileM + shift);
+          uint32_t sb = ring0 + slot * slot16;
+          for (int k = 0; k < ksteps; ++k) {
+            ptx::umma_i8_lo(d, (sa & 0x3FFFu) | a_hi, (sb & 0x3FFFu) | b_hi, idesc, (tap > 0 || k > 0) ? 1u : 0u);
+            sa += 2u * rows;
+            sb += 2u * (uint32_t)c.n_pad;
           }
-          ptx::umma_commit(ptx::smem_u32(&r.ctl->slice_done[b]));
         }
-    } else {
-      r.gslice += (uint32_t)nslices;
+        ptx::umma_commit(ptx::smem_u32(&r.ctl->w_empty[slot]));
+      }
+      ptx::umma_commit(ptx::smem_u32(&r.ctl->conv_done));
     }
     __syncwarp();
     return;
   }
-  // ---- builders ----
-  // the conv's requantisation constants and index list move to shared memory while the slices run
-  // (the previous conv's epilogue, their last reader, ended with a CTA barrier)
+  // requantising warps: the conv's constants and index list move to shared memory meanwhile (the
+  // previous conv's epilogue, their last reader, ended with a CTA barrier)
   {
     uint4* tab = reinterpret_cast<uint4*>(r.smem + r.H->s_tab);
     const uint4* src_rq = reinterpret_cast<const uint4*>(r.blob + c.rq_off);
@@ -196,39 +173,10 @@ __device__ void conv_mma(Run& r, const ResConv& c) {
       for (int i = r.tid; i < c.n; i += kResThreads) ti[i] = si[i];
     }
   }
-  for (int tile = 0; tile < r.ntiles; ++tile) {
-    for (int tap = 0; tap < 9; ++tap) {
-      const uint32_t g = r.gslice++;
-      const int b = (int)(g & 1u);
-      const uint32_t use = g >> 1;                      // how often buffer b has been used before
-      // the MMAs that last read buffer b must have completed before it is overwritten
-      // (suspended wait: the builders run ahead of the issuing thread, and a spinning warp would take
-      // issue slots from it)
-      if (use > 0 && !ptx::mbar_test_wait(ptx::smem_u32(&r.ctl->slice_done[b]), (use - 1u) & 1u))
-        res_wait(r.ctl, r.status, &r.ctl->slice_done[b], (use - 1u) & 1u);
-      uint8_t* abuf = r.smem + r.H->s_abuf[b];
-      const int off = ((tap * 11) >> 5) - 1;            // u - 1
-      const int shift = off * r.g.w + (tap - (off + 1) * 3 - 1);
-      for (int it = r.tid; it < kTileM * nchunks; it += kResThreads) {
-        const int row = it & (kTileM - 1), ch = it >> 7;
-        const int p = tile * kTileM + row;
-        uint4 val = make_uint4(0u, 0u, 0u, 0u);
-        if ((r.rowinfo[p] >> tap) & 1u)
-          val = *reinterpret_cast<const uint4*>(src + (size_t)(p + shift) * pitch + ch * 16);
-        *reinterpret_cast<uint4*>(abuf + (size_t)ch * (kTileM * 16) + row * 16) = val;
-      }
-      ptx::fence_async_smem();
-      __syncwarp();
-      if (r.lane == 0)
-        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ptx::smem_u32(&r.ctl->a_full[b])) : "memory");
-    }
-  }
-  // the last two slices (one per buffer) close the conv
-  const uint32_t g = r.gslice;
-  if (g >= 1) res_wait_fast(r.ctl, r.status, &r.ctl->slice_done[(g - 1) & 1u], (((g - 1) >> 1)) & 1u);
-  if (g >= 2) res_wait_fast(r.ctl, r.status, &r.ctl->slice_done[(g - 2) & 1u], (((g - 2) >> 1)) & 1u);
+  if (!ptx::mbar_test_wait(ptx::smem_u32(&r.ctl->conv_done), parity))
+    res_wait(r.ctl, r.status, &r.ctl->conv_done, parity);
   ptx::tc_fence_after();
-  asm volatile("bar.sync 1, %0;" ::"n"(kResThreads) : "memory");      // builders only: the staged tables are complete
+  asm volatile("bar.sync 1, %0;" ::"n"(kResThreads) : "memory");      // requantising warps: the staged tables are complete
 }
 
 struct StepIo {            // what the epilogue of the last conv / the prior head needs
@@ -245,10 +193,10 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
   const int q = r.warp & 3, split = r.warp >> 2, nsplit = kResThreads / 128;
   const int nch = c.n_pad >> 4;
   uint8_t* dst = buf_of(r, c.dst);
-  const int dpitch = pitch_of(r, c.dst);
   for (int tile = 0; tile < (r.warp < kResBuilderWarps ? r.ntiles : 0); ++tile) {
-    const int p = tile * kTileM + q * 32 + r.lane;
-    const bool valid = p < r.g.px;
+    const int rr = tile * kTileM + q * 32 + r.lane;       // padded position of this thread's row
+    const int p = r.pixel_of[rr];                          // its pixel, or -1 at a padding position
+    const bool valid = p >= 0;
     for (int ch = split; ch < nch; ch += nsplit) {
       uint32_t acc[16];
       __syncwarp();                                   // the tensor-memory load is a whole-warp instruction
@@ -269,7 +217,7 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
           }
           wd[i] = word;
         }
-        *reinterpret_cast<uint4*>(dst + (size_t)p * dpitch + ch * 16) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+        *reinterpret_cast<uint4*>(at(r, dst, ch * 16, rr)) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
       } else {
 #pragma unroll 4
         for (int i = 0; i < 16; ++i) {
@@ -277,7 +225,7 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
           if (col >= c.n) continue;
           const int32_t y = rq_const((int32_t)acc[i], orq[col]);
           if (c.kind == kResBranch) {
-            uint8_t* xp = dst + (size_t)p * dpitch + idx[col];
+            uint8_t* xp = at(r, dst, idx[col], rr);
             *xp = (uint8_t)clampi((int)*xp + y, 0, 255);
           } else if (c.kind == kResOut) {
             uint32_t* vv = reinterpret_cast<uint32_t*>(&r.v[io.colB[col] * r.g.pg + p]);
@@ -291,18 +239,22 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
       }
     }
   }
+  ptx::fence_async_smem();       // the next conv's MMAs read what was stored here
   ptx::tc_fence_before();
   __syncthreads();
 }
 
-// network input: logical channels cols[0 .. n) of the flow variable, requantised to int8, pixel-major
+// network input: logical channels cols[0 .. n) of the flow variable, requantised to int8, at the
+// image's positions of the padded layout
 __device__ void requant_input(Run& r, const int32_t* cols, int n, int32_t m0, int32_t s) {
-  int8_t* xa = reinterpret_cast<int8_t*>(r.smem + r.H->s_xa);
-  const int pitch = r.H->xa_pitch;
+  uint8_t* xa = r.smem + r.H->s_xa;
   for (int it = r.tid; it < (r.warp < kResBuilderWarps ? n * r.g.px : 0); it += kResThreads) {
     const int c = it / r.g.px, p = it - c * r.g.px;
-    xa[(size_t)p * pitch + c] = (int8_t)clampi(rq64(r.v[cols[c] * r.g.pg + p], m0, s), -128, 127);
+    const int i = rdiv(p, r.g.mul_w), j = p - i * r.g.w;
+    const int rr = (i + 1) * r.H->w2 + (j + 1);
+    *at(r, xa, c, rr) = (uint8_t)(int8_t)clampi(rq64(r.v[cols[c] * r.g.pg + p], m0, s), -128, 127);
   }
+  ptx::fence_async_smem();
   __syncthreads();
 }
 
@@ -315,11 +267,11 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
-    for (int s = 0; s < kResMaxWSlots; ++s) ptx::mbar_init(ptx::smem_u32(&ctl.w_full[s]), 1);
-    for (int s = 0; s < 2; ++s) {
-      ptx::mbar_init(ptx::smem_u32(&ctl.slice_done[s]), 1);
-      ptx::mbar_init(ptx::smem_u32(&ctl.a_full[s]), (uint32_t)kResBuilderWarps);
+    for (int s = 0; s < kResMaxWSlots; ++s) {
+      ptx::mbar_init(ptx::smem_u32(&ctl.w_full[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl.w_empty[s]), 1);
     }
+    ptx::mbar_init(ptx::smem_u32(&ctl.conv_done), 1);
     ptx::mbar_init_fence();
     ctl.abort = 0;
   }
@@ -332,20 +284,24 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
   r.smem = smem; r.ctl = &ctl; r.status = a.status; r.blob = a.blob; r.H = H;
   r.g.px = P.px; r.g.h = P.h; r.g.w = P.w; r.g.pg = P.pg; r.g.mul_w = P.mul_w;
   r.tid = tid; r.warp = warp; r.lane = lane;
-  r.ntiles = (P.px + kTileM - 1) / kTileM;
+  r.ntiles = H->ntiles;
   r.tmem = ctl.tmem_base;
   r.gslice = 0;
   r.gload = 0;
+  r.nconv = 0;
   r.v = reinterpret_cast<int32_t*>(smem + H->s_v);
-  uint32_t* rowinfo = reinterpret_cast<uint32_t*>(smem + H->s_rowinfo);
-  r.rowinfo = rowinfo;
+  int32_t* pixel_of = reinterpret_cast<int32_t*>(smem + H->s_rowinfo);
+  r.pixel_of = pixel_of;
 
   const int c = P.c, px = P.px, pg = P.pg, w = P.w;
   const int b = blockIdx.x;                       // one image per CTA
   const bool builder = warp < kResBuilderWarps;
   const int per_img = builder ? c * px : 0;       // the issuing warp takes no part in the element loops
   int32_t* v = r.v;
-  for (int i = tid; i < (builder ? r.ntiles * kTileM : 0); i += kResThreads) rowinfo[i] = gather_mask(i, r.g);
+  for (int rr = tid; rr < (builder ? r.ntiles * kTileM : 0); rr += kResThreads) {
+    const int i = rr / H->w2, j = rr - i * H->w2;          // position (i, j) of the (h+2) x (w+2) frame
+    pixel_of[rr] = (i >= 1 && i <= P.h && j >= 1 && j <= P.w) ? (i - 1) * P.w + (j - 1) : -1;
+  }
   // activation buffers start at zero: padding channels and bytes beyond a conv's outputs stay zero
   // or meet zero weights
   for (uint32_t i = H->s_xa + tid * 16; builder && i < H->s_rowinfo; i += kResThreads * 16)
@@ -404,17 +360,26 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
       const ResConv cv = convs[cp.conv0 + ci];
       conv_mma(r, cv);
       if (cv.kind == kResBranch) {
-        // the shortcut Q(x) of all channels, in place (the first conv of the block has read X already)
+        // the shortcut Q(x) of all channels, in place, at the image's positions (the first conv of
+        // the block has read X already)
         uint8_t* X = smem + H->s_x;
-        const int words = H->x_pitch >> 2;
-        for (int it = tid; it < (builder ? px * words : 0); it += kResThreads) {
-          uint32_t* wp = reinterpret_cast<uint32_t*>(X) + it;
-          const uint32_t in = *wp;
-          uint32_t out = 0;
+        const int chunks = H->x_pitch >> 4, npos = r.ntiles * kTileM;
+        for (int it = tid; it < (builder ? chunks * npos : 0); it += kResThreads) {
+          const int ch = it / npos, rr = it - ch * npos;
+          if (pixel_of[rr] < 0) continue;
+          uint4* wp = reinterpret_cast<uint4*>(at(r, X, ch * 16, rr));
+          uint4 val = *wp;
+          uint32_t* wv = reinterpret_cast<uint32_t*>(&val);
 #pragma unroll
-          for (int jj = 0; jj < 4; ++jj)
-            out |= (uint32_t)clampi(rq64((int32_t)((in >> (8 * jj)) & 0xFFu), cv.short_m0, cv.short_s), 0, 255) << (8 * jj);
-          *wp = out;
+          for (int k = 0; k < 4; ++k) {
+            const uint32_t in = wv[k];
+            uint32_t out = 0;
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj)
+              out |= (uint32_t)clampi(rq64((int32_t)((in >> (8 * jj)) & 0xFFu), cv.short_m0, cv.short_s), 0, 255) << (8 * jj);
+            wv[k] = out;
+          }
+          *wp = val;
         }
         __syncthreads();
       }

@@ -11,8 +11,8 @@
 
 namespace iodf {
 
-constexpr int kResBuilderWarps = 16;                         // build operand slices, requantise
-constexpr int kResThreads = kResBuilderWarps * 32;           // builder threads
+constexpr int kResBuilderWarps = 16;                         // the warps that requantise (and load / store the level)
+constexpr int kResThreads = kResBuilderWarps * 32;           // their threads
 constexpr int kResAllThreads = kResThreads + 32;             // + the warp that issues weight copies and MMAs
 constexpr int kResMaxWidth = 128;      // hidden channels of a residual network (conv outputs), padded to 16
 constexpr int kResMaxPixels = 256;     // pixels per image at a residual level (two 128-row tiles)
@@ -55,11 +55,14 @@ struct ResHead {
   int32_t prior_in_m0, prior_in_s, ls_lo, ls_hi;
   int32_t xa_pitch, x_pitch, mid_pitch;      // bytes per pixel of the three activation buffers (multiples of 32)
   uint32_t coupling_off, conv_off;           // blob offsets of ResCouplingRec[] and ResConv[]
-  uint32_t s_v, s_xa, s_x, s_mid, s_rowinfo, s_abuf[2], s_wring, w_slot_bytes, s_total;   // shared-memory layout
+  uint32_t s_v, s_xa, s_x, s_mid, s_rowinfo, s_unused[2], s_wring, w_slot_bytes, s_total;   // shared-memory layout
   int32_t tmem_cols;
   int32_t n_wslots;              // weight slices in flight: ring of 2 .. kResMaxWSlots slots at s_wring
   uint32_t s_tab;                // the running conv's OutRq[kResMaxWidth] and idx[kResMaxWidth]
-  int32_t pad[7];
+  // padded layout of the activation buffers: rows of w2 = w + 2 positions, (h + 2) * w2 positions
+  // rounded up to ntiles * 128 computed ones, `guard` rows before them, `rows` rows per channel chunk
+  int32_t w2, guard, rows, ntiles;
+  int32_t pad[3];
 };
 static_assert(sizeof(ResHead) == 128, "128-byte header");
 

@@ -77,3 +77,25 @@ def test_residual_and_plain_levels_in_one_model_and_stepped_decode(G):
     G.iodf_check(m)
     np.testing.assert_array_equal(prior.cpu().numpy(), p_ref)
     np.testing.assert_array_equal(xr.cpu().numpy(), x)
+
+
+def test_config_r32_in_the_benchmarks_launch_configuration(G):
+    """The paper's network on the ImageNet32 geometry at the benchmark's batch of 64: the oracle
+    checks sampled images (first, last, two in between), the round trip covers the whole batch."""
+    import torch
+    model = S.config_model("R32")
+    x = S.config_images("R32")
+    B = x.shape[0]
+    idx = np.array([0, 21, 42, B - 1])
+    z_ref, p_ref = O.forward(O.Packed(model), x[idx])
+    m = G.iodf_create(model, B)
+    z, p = G.iodf_forward(m, _t(x))
+    G.iodf_check(m)
+    np.testing.assert_array_equal(z.cpu().numpy()[idx], z_ref)
+    np.testing.assert_array_equal(p.cpu().numpy()[idx], p_ref)
+    xr = G.iodf_inverse(m, z)
+    G.iodf_check(m)
+    np.testing.assert_array_equal(xr.cpu().numpy(), x)
+    # an image's result does not depend on the batch around it
+    z1, _ = G.iodf_forward(m, _t(x[5:6]))
+    assert torch.equal(z1[0], z[5])
