@@ -521,7 +521,7 @@ int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P,
   H.s_x = take((uint32_t)(H.x_pitch / 16) * rows * 16);
   H.s_mid = take((uint32_t)(H.mid_pitch / 16) * rows * 16);
   H.s_rowinfo = take((uint32_t)ntiles * kTileM * 4);
-  H.s_tab = take((uint32_t)kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t)));
+  H.s_tab = take((uint32_t)kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t)) + 256);   // + the shortcut table
   // as deep a weight ring as fits (at least two slots)
   H.w_slot_bytes = up((uint32_t)nmax * kmax, kAlign);
   H.n_wslots = kResMaxWSlots;

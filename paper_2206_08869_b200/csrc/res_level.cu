@@ -97,6 +97,7 @@ struct Run {
   uint32_t gslice;          // weight slices consumed so far (ring slot = gslice % n_wslots), issuing lane only
   uint32_t gload;           // weight slices requested so far, issuing lane only
   uint32_t nconv;           // convs run so far (parity of conv_done)
+  uint32_t prefetched;      // weight slices of the coming conv that were requested already, issuing lane only
   int32_t* v;
   const int32_t* pixel_of;  // pixel index of a padded position, -1 at padding
 };
@@ -111,13 +112,13 @@ __device__ __forceinline__ uint8_t* at(const Run& r, uint8_t* buf, int c, int rr
 
 // All nine taps of all tiles: accumulators D[tile][0 .. n_pad) complete in TMEM on return (for the
 // requantising warps; the issuing warp returns as soon as everything is issued).
-__device__ void conv_mma(Run& r, const ResConv& c) {
+__device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next) {
   const uint32_t parity = r.nconv & 1u;
   ++r.nconv;
   if (r.warp == kResBuilderWarps) {
     if (r.lane == 0) {
       const uint32_t nws = (uint32_t)r.H->n_wslots, ahead = nws - 1u;
-      auto request = [&](int tap) {
+      auto request = [&](const ResConv& c, int tap) {
         const uint32_t gl = r.gload++;
         const uint32_t slot = gl % nws, use = gl / nws;
         // the slice that used this slot last must have been consumed
@@ -127,7 +128,8 @@ __device__ void conv_mma(Run& r, const ResConv& c) {
         ptx::bulk_g2s(ptx::smem_u32(r.smem + r.H->s_wring + slot * r.H->w_slot_bytes),
                       r.blob + c.w_off + (size_t)tap * c.slice_bytes, c.slice_bytes, bar);
       };
-      for (int tap = 0; tap < 9 && tap < (int)ahead; ++tap) request(tap);
+      for (int tap = (int)r.prefetched; tap < 9 && tap < (int)ahead; ++tap) request(c, tap);
+      r.prefetched = 0;
       const uint32_t idesc = ptx::umma_idesc_i8((uint32_t)c.n_pad, c.a_unsigned != 0);
       const uint32_t rows = (uint32_t)r.H->rows;
       // operand start addresses in 16-byte units
@@ -137,7 +139,7 @@ __device__ void conv_mma(Run& r, const ResConv& c) {
       const int ksteps = c.kpad >> 5;
       ptx::tc_fence_after();
       for (int tap = 0; tap < 9; ++tap) {
-        if (tap + (int)ahead < 9) request(tap + (int)ahead);
+        if (tap + (int)ahead < 9) request(c, tap + (int)ahead);
         const uint32_t g = r.gslice++;
         const uint32_t slot = g % nws;
         res_wait_fast(r.ctl, r.status, &r.ctl->w_full[slot], (g / nws) & 1u);
@@ -157,6 +159,11 @@ __device__ void conv_mma(Run& r, const ResConv& c) {
         ptx::umma_commit(ptx::smem_u32(&r.ctl->w_empty[slot]));
       }
       ptx::umma_commit(ptx::smem_u32(&r.ctl->conv_done));
+      // the first weight slices of the conv that follows travel while this conv is requantised
+      if (next) {
+        for (int tap = 0; tap < 9 && tap < (int)ahead; ++tap) request(*next, tap);
+        r.prefetched = ahead < 9u ? ahead : 9u;
+      }
     }
     __syncwarp();
     return;
@@ -171,6 +178,9 @@ __device__ void conv_mma(Run& r, const ResConv& c) {
       int32_t* ti = reinterpret_cast<int32_t*>(tab + kResMaxWidth);
       const int32_t* si = reinterpret_cast<const int32_t*>(r.blob + c.idx_off);
       for (int i = r.tid; i < c.n; i += kResThreads) ti[i] = si[i];
+      // the block's shortcut rq(x; M_r, s_r) as a table over the 256 values of an 8-bit x
+      uint8_t* lut = r.smem + r.H->s_tab + kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t));
+      if (r.tid < 256) lut[r.tid] = (uint8_t)clampi(rq64(r.tid, c.short_m0, c.short_s), 0, 255);
     }
   }
   if (!ptx::mbar_test_wait(ptx::smem_u32(&r.ctl->conv_done), parity))
@@ -289,6 +299,7 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
   r.gslice = 0;
   r.gload = 0;
   r.nconv = 0;
+  r.prefetched = 0;
   r.v = reinterpret_cast<int32_t*>(smem + H->s_v);
   int32_t* pixel_of = reinterpret_cast<int32_t*>(smem + H->s_rowinfo);
   r.pixel_of = pixel_of;
@@ -348,7 +359,7 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
       io.mu = a.prior + (size_t)b * 2u * P.d_fact + P.prior_off;
       io.ls = io.mu + P.d_fact;
       io.ls_lo = H->ls_lo; io.ls_hi = H->ls_hi;
-      conv_mma(r, cv);
+      conv_mma(r, cv, nullptr);
       conv_epilogue(r, cv, io);
       continue;
     }
@@ -358,11 +369,14 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
     requant_input(r, reinterpret_cast<const int32_t*>(a.blob + cp.colA_off), P.ca, cp.in_m0, cp.in_s);
     for (int ci = 0; ci < cp.n_convs; ++ci) {
       const ResConv cv = convs[cp.conv0 + ci];
-      conv_mma(r, cv);
+      const bool has_next = ci + 1 < cp.n_convs;
+      const ResConv nx = convs[cp.conv0 + (has_next ? ci + 1 : ci)];
+      conv_mma(r, cv, has_next ? &nx : nullptr);
       if (cv.kind == kResBranch) {
         // the shortcut Q(x) of all channels, in place, at the image's positions (the first conv of
         // the block has read X already)
         uint8_t* X = smem + H->s_x;
+        const uint8_t* lut = smem + H->s_tab + kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t));   // staged by conv_mma
         const int chunks = H->x_pitch >> 4, npos = r.ntiles * kTileM;
         for (int it = tid; it < (builder ? chunks * npos : 0); it += kResThreads) {
           const int ch = it / npos, rr = it - ch * npos;
@@ -375,8 +389,7 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
             const uint32_t in = wv[k];
             uint32_t out = 0;
 #pragma unroll
-            for (int jj = 0; jj < 4; ++jj)
-              out |= (uint32_t)clampi(rq64((int32_t)((in >> (8 * jj)) & 0xFFu), cv.short_m0, cv.short_s), 0, 255) << (8 * jj);
+            for (int jj = 0; jj < 4; ++jj) out |= (uint32_t)lut[(in >> (8 * jj)) & 0xFFu] << (8 * jj);
             wv[k] = out;
           }
           *wp = val;

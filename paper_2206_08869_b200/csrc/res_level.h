@@ -58,7 +58,7 @@ struct ResHead {
   uint32_t s_v, s_xa, s_x, s_mid, s_rowinfo, s_unused[2], s_wring, w_slot_bytes, s_total;   // shared-memory layout
   int32_t tmem_cols;
   int32_t n_wslots;              // weight slices in flight: ring of 2 .. kResMaxWSlots slots at s_wring
-  uint32_t s_tab;                // the running conv's OutRq[kResMaxWidth] and idx[kResMaxWidth]
+  uint32_t s_tab;                // the running conv's OutRq[kResMaxWidth], idx[kResMaxWidth] and 256-byte shortcut table
   // padded layout of the activation buffers: rows of w2 = w + 2 positions, (h + 2) * w2 positions
   // rounded up to ntiles * 128 computed ones, `guard` rows before them, `rows` rows per channel chunk
   int32_t w2, guard, rows, ntiles;
