@@ -377,10 +377,11 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
         // the block has read X already)
         uint8_t* X = smem + H->s_x;
         const uint8_t* lut = smem + H->s_tab + kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t));   // staged by conv_mma
-        const int chunks = H->x_pitch >> 4, npos = r.ntiles * kTileM;
-        for (int it = tid; it < (builder ? chunks * npos : 0); it += kResThreads) {
-          const int ch = it / npos, rr = it - ch * npos;
-          if (pixel_of[rr] < 0) continue;
+        const int chunks = H->x_pitch >> 4;
+        for (int it = tid; it < (builder ? chunks * px : 0); it += kResThreads) {
+          const int ch = it / px, p = it - ch * px;
+          const int pi = rdiv(p, P.mul_w), pj = p - pi * w;
+          const int rr = (pi + 1) * H->w2 + (pj + 1);
           uint4* wp = reinterpret_cast<uint4*>(at(r, X, ch * 16, rr));
           uint4 val = *wp;
           uint32_t* wv = reinterpret_cast<uint32_t*>(&val);
