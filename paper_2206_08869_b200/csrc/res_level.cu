@@ -17,8 +17,9 @@
 //
 // The (h+2)(w+2) positions are computed in full (outputs at padding positions are discarded): a
 // third more rows than pixels at 16x16, bought with tensor time that is idle anyway. One lane of a
-// 17th warp requests the taps' weight slices from the packed blob (a ring, several slices ahead)
-// and issues the MMAs of a conv back to back; the 16 other warps requantise. A block is
+// 17th warp issues the MMAs of a conv back to back, one lane of an 18th streams the taps' weight
+// slices from the packed blob through a ring, running ahead into the next conv; the 16 other warps
+// requantise. A block is
 //   MID = clip(ReLU(rq(conv_a(X))))                        kResHidden
 //   X   = rq(X; M_r, s_r)      for all D channels          the shortcut Q(x), in place
 //   X[idx[j]] = clip(max(X[idx[j]] + rq(conv_b(MID))[j], 0), 0, 255)   kResBranch: scatter add + ReLU
@@ -95,9 +96,9 @@ struct Run {
   int ntiles;
   uint32_t tmem;
   uint32_t gslice;          // weight slices consumed so far (ring slot = gslice % n_wslots), issuing lane only
-  uint32_t gload;           // weight slices requested so far, issuing lane only
+  uint32_t gload;           // weight slices requested so far, loading lane only
   uint32_t nconv;           // convs run so far (parity of conv_done)
-  uint32_t prefetched;      // weight slices of the coming conv that were requested already, issuing lane only
+  uint32_t prefetched;      // weight slices of the coming conv that were requested already, loading lane only
   int32_t* v;
   const int32_t* pixel_of;  // pixel index of a padded position, -1 at padding
 };
@@ -115,9 +116,12 @@ __device__ __forceinline__ uint8_t* at(const Run& r, uint8_t* buf, int c, int rr
 __device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next) {
   const uint32_t parity = r.nconv & 1u;
   ++r.nconv;
-  if (r.warp == kResBuilderWarps) {
+  if (r.warp == kResBuilderWarps + 1) {
+    // ---- loading warp: the conv's nine weight slices, then the first ones of the conv that follows.
+    // A request blocks while the ring is full (and the copy instruction itself takes hundreds of
+    // clocks to issue), which is why it has a lane of its own.
     if (r.lane == 0) {
-      const uint32_t nws = (uint32_t)r.H->n_wslots, ahead = nws - 1u;
+      const uint32_t nws = (uint32_t)r.H->n_wslots;
       auto request = [&](const ResConv& c, int tap) {
         const uint32_t gl = r.gload++;
         const uint32_t slot = gl % nws, use = gl / nws;
@@ -128,8 +132,24 @@ __device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next) {
         ptx::bulk_g2s(ptx::smem_u32(r.smem + r.H->s_wring + slot * r.H->w_slot_bytes),
                       r.blob + c.w_off + (size_t)tap * c.slice_bytes, c.slice_bytes, bar);
       };
-      for (int tap = (int)r.prefetched; tap < 9 && tap < (int)ahead; ++tap) request(c, tap);
+      for (int tap = (int)r.prefetched; tap < 9; ++tap) request(c, tap);
       r.prefetched = 0;
+      // Slices of the next conv travel while this one is multiplied and requantised. Never more than
+      // the ring holds: their slots are freed by this conv's MMAs, which all complete before the CTA
+      // barrier that this warp, too, has to reach.
+      if (next) {
+        const int npre = (int)(nws < 9u ? nws : 9u);
+        for (int tap = 0; tap < npre; ++tap) request(*next, tap);
+        r.prefetched = (uint32_t)npre;
+      }
+    }
+    __syncwarp();
+    return;
+  }
+  if (r.warp == kResBuilderWarps) {
+    // ---- issuing warp: the conv's MMAs, tap by tap as the weight slices land
+    if (r.lane == 0) {
+      const uint32_t nws = (uint32_t)r.H->n_wslots;
       const uint32_t idesc = ptx::umma_idesc_i8((uint32_t)c.n_pad, c.a_unsigned != 0);
       const uint32_t rows = (uint32_t)r.H->rows;
       // operand start addresses in 16-byte units
@@ -139,7 +159,6 @@ __device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next) {
       const int ksteps = c.kpad >> 5;
       ptx::tc_fence_after();
       for (int tap = 0; tap < 9; ++tap) {
-        if (tap + (int)ahead < 9) request(c, tap + (int)ahead);
         const uint32_t g = r.gslice++;
         const uint32_t slot = g % nws;
         res_wait_fast(r.ctl, r.status, &r.ctl->w_full[slot], (g / nws) & 1u);
@@ -159,11 +178,6 @@ __device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next) {
         ptx::umma_commit(ptx::smem_u32(&r.ctl->w_empty[slot]));
       }
       ptx::umma_commit(ptx::smem_u32(&r.ctl->conv_done));
-      // the first weight slices of the conv that follows travel while this conv is requantised
-      if (next) {
-        for (int tap = 0; tap < 9 && tap < (int)ahead; ++tap) request(*next, tap);
-        r.prefetched = ahead < 9u ? ahead : 9u;
-      }
     }
     __syncwarp();
     return;
