@@ -113,7 +113,7 @@ __device__ __forceinline__ uint8_t* at(const Run& r, uint8_t* buf, int c, int rr
 
 // All nine taps of all tiles: accumulators D[tile][0 .. n_pad) complete in TMEM on return (for the
 // requantising warps; the issuing warp returns as soon as everything is issued).
-__device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next) {
+__device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next, const int32_t* colB) {
   const uint32_t parity = r.nconv & 1u;
   ++r.nconv;
   if (r.warp == kResBuilderWarps + 1) {
@@ -195,6 +195,10 @@ __device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next) {
       // the block's shortcut rq(x; M_r, s_r) as a table over the 256 values of an 8-bit x
       uint8_t* lut = r.smem + r.H->s_tab + kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t));
       if (r.tid < 256) lut[r.tid] = (uint8_t)clampi(rq64(r.tid, c.short_m0, c.short_s), 0, 255);
+    } else if (c.kind == kResOut) {
+      // the physical columns of x_b's channels, in place of the index list
+      int32_t* ti = reinterpret_cast<int32_t*>(tab + kResMaxWidth);
+      for (int i = r.tid; i < c.n; i += kResThreads) ti[i] = colB[i];
     }
   }
   if (!ptx::mbar_test_wait(ptx::smem_u32(&r.ctl->conv_done), parity))
@@ -242,17 +246,30 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
           wd[i] = word;
         }
         *reinterpret_cast<uint4*>(at(r, dst, ch * 16, rr)) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+      } else if (c.kind == kResBranch) {
+        // all sixteen shortcut bytes are read before any is written back (a byte store could alias
+        // anything for the compiler and would otherwise serialise the sixteen updates)
+        uint8_t* xp[16];
+        int xv[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int col = ch * 16 + i;
+          xp[i] = at(r, dst, col < c.n ? idx[col] : 0, rr);
+          xv[i] = *xp[i];
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int col = ch * 16 + i;
+          if (col < c.n) *xp[i] = (uint8_t)clampi(xv[i] + rq_const((int32_t)acc[i], orq[col]), 0, 255);
+        }
       } else {
 #pragma unroll 4
         for (int i = 0; i < 16; ++i) {
           const int col = ch * 16 + i;
           if (col >= c.n) continue;
           const int32_t y = rq_const((int32_t)acc[i], orq[col]);
-          if (c.kind == kResBranch) {
-            uint8_t* xp = at(r, dst, idx[col], rr);
-            *xp = (uint8_t)clampi((int)*xp + y, 0, 255);
-          } else if (c.kind == kResOut) {
-            uint32_t* vv = reinterpret_cast<uint32_t*>(&r.v[io.colB[col] * r.g.pg + p]);
+          if (c.kind == kResOut) {
+            uint32_t* vv = reinterpret_cast<uint32_t*>(&r.v[idx[col] * r.g.pg + p]);       // idx: staged columns of x_b
             *vv = io.subtract ? (*vv - (uint32_t)y) : (*vv + (uint32_t)y);
           } else {   // kResPrior: first half mu, second half the clipped log-scale index
             const int half = c.n >> 1;
@@ -373,7 +390,7 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
       io.mu = a.prior + (size_t)b * 2u * P.d_fact + P.prior_off;
       io.ls = io.mu + P.d_fact;
       io.ls_lo = H->ls_lo; io.ls_hi = H->ls_hi;
-      conv_mma(r, cv, nullptr);
+      conv_mma(r, cv, nullptr, nullptr);
       conv_epilogue(r, cv, io);
       continue;
     }
@@ -385,7 +402,7 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
       const ResConv cv = convs[cp.conv0 + ci];
       const bool has_next = ci + 1 < cp.n_convs;
       const ResConv nx = convs[cp.conv0 + (has_next ? ci + 1 : ci)];
-      conv_mma(r, cv, has_next ? &nx : nullptr);
+      conv_mma(r, cv, has_next ? &nx : nullptr, io.colB);
       if (cv.kind == kResBranch) {
         // the shortcut Q(x) of all channels, in place, at the image's positions (the first conv of
         // the block has read X already)
