@@ -16,8 +16,9 @@
 //   results are stored at the image's positions only, so the padding stays zero.
 //
 // The (h+2)(w+2) positions are computed in full (outputs at padding positions are discarded): a
-// third more rows than pixels at 16x16, bought with tensor time that is idle anyway. One lane of a
-// 17th warp issues the MMAs of a conv back to back, one lane of an 18th streams the taps' weight
+// third more rows than pixels at 16x16, bought with tensor time that is idle anyway. One lane each
+// of two more warps issues the MMAs of a conv back to back (tiles dealt between them), one lane of a
+// last warp streams the taps' weight
 // slices from the packed blob through a ring, running ahead into the next conv; the 16 other warps
 // requantise. A block is
 //   MID = clip(ReLU(rq(conv_a(X))))                        kResHidden
@@ -116,7 +117,7 @@ __device__ __forceinline__ uint8_t* at(const Run& r, uint8_t* buf, int c, int rr
 __device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next, const int32_t* colB) {
   const uint32_t parity = r.nconv & 1u;
   ++r.nconv;
-  if (r.warp == kResBuilderWarps + 1) {
+  if (r.warp == kResBuilderWarps + kResIssuers) {
     // ---- loading warp: the conv's nine weight slices, then the first ones of the conv that follows.
     // A request blocks while the ring is full (and the copy instruction itself takes hundreds of
     // clocks to issue), which is why it has a lane of its own.
@@ -146,8 +147,11 @@ __device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next, const in
     __syncwarp();
     return;
   }
-  if (r.warp == kResBuilderWarps) {
-    // ---- issuing warp: the conv's MMAs, tap by tap as the weight slices land
+  if (r.warp >= kResBuilderWarps) {
+    // ---- issuing warps: the conv's MMAs, tap by tap as the weight slices land; issuer i takes the
+    // tiles i, i + kResIssuers, ... (accumulators are per tile, so the issuers are independent; an MMA
+    // costs its issuing lane ~100 clocks, the tensor core much less)
+    const int me = r.warp - kResBuilderWarps;
     if (r.lane == 0) {
       const uint32_t nws = (uint32_t)r.H->n_wslots;
       const uint32_t idesc = ptx::umma_idesc_i8((uint32_t)c.n_pad, c.a_unsigned != 0);
@@ -165,7 +169,7 @@ __device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next, const in
         ptx::tc_fence_after();
         const int u = (tap * 11) >> 5;
         const int shift = (u - 1) * r.H->w2 + (tap - u * 3 - 1);
-        for (int tile = 0; tile < r.ntiles; ++tile) {
+        for (int tile = me; tile < r.ntiles; tile += kResIssuers) {
           const uint32_t d = r.tmem + (uint32_t)(tile * kResMaxWidth);
           uint32_t sa = a0 + (uint32_t)(tile * kTileM + shift);
           uint32_t sb = ring0 + slot * slot16;
@@ -310,9 +314,9 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
   if (tid == 0) {
     for (int s = 0; s < kResMaxWSlots; ++s) {
       ptx::mbar_init(ptx::smem_u32(&ctl.w_full[s]), 1);
-      ptx::mbar_init(ptx::smem_u32(&ctl.w_empty[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctl.w_empty[s]), (uint32_t)kResIssuers);      // every issuer commits to it
     }
-    ptx::mbar_init(ptx::smem_u32(&ctl.conv_done), 1);
+    ptx::mbar_init(ptx::smem_u32(&ctl.conv_done), (uint32_t)kResIssuers);
     ptx::mbar_init_fence();
     ctl.abort = 0;
   }
