@@ -410,6 +410,11 @@ def main():
             "latency_batch1": lat,
         }
         out.update(extra)
+        if cfg == "R32":
+            # the paper's own latency for this architecture, for context only: another GPU, a trained
+            # model, floating-point requantisation, the first conv of every coupling in FP32
+            out["paper_context"] = {"ms_per_sample": 0.27, "batch": 64, "hardware": "Tesla T4, TensorRT 8.2",
+                                    "source": "Table 4, IODF on ImageNet32"}
         if world == 1:
             r, n, dt = oracle_rate(model, cfg, B, cores)
             out["cpu_baseline"] = {"value": r, "unit": UNIT, "cores": cores, "kind": "oracle",
