@@ -13,7 +13,7 @@ namespace iodf {
 
 constexpr int kResBuilderWarps = 16;                         // the warps that requantise (and load / store the level)
 constexpr int kResThreads = kResBuilderWarps * 32;           // their threads
-constexpr int kResIssuers = 2;                               // warps whose elected lane issues MMAs (tiles dealt between them)
+constexpr int kResIssuers = 3;                               // warps whose elected lane issues MMAs (tiles dealt between them)
 constexpr int kResAllThreads = kResThreads + 32 * (kResIssuers + 1);   // + the issuing warps and the warp that streams weights
 constexpr int kResMaxWidth = 128;      // hidden channels of a residual network (conv outputs), padded to 16
 constexpr int kResMaxPixels = 256;     // pixels per image at a residual level (two 128-row tiles)
