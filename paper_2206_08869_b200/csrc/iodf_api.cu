@@ -528,7 +528,8 @@ int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P,
   while (H.n_wslots > 2 && off + (uint32_t)H.n_wslots * H.w_slot_bytes > smem_limit) --H.n_wslots;
   H.s_wring = take((uint32_t)H.n_wslots * H.w_slot_bytes);
   H.s_total = off;
-  H.tmem_cols = ntiles > 2 ? 4 * kResMaxWidth : (ntiles > 1 ? 2 * kResMaxWidth : kResMaxWidth);
+  // one tile: every issuing warp keeps a partial accumulator of its own
+  H.tmem_cols = (ntiles > 2 || ntiles == 1) ? 4 * kResMaxWidth : 2 * kResMaxWidth;
   if (off > smem_limit || ntiles > 4 || rows * 16 >= (1 << 18)) return IODF_EUNSUPPORTED;
   std::memcpy(blob.data(), &H, sizeof(H));
   std::memcpy(blob.data() + H.coupling_off, cps.data(), sizeof(ResCouplingRec) * cps.size());

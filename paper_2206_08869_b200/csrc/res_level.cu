@@ -17,8 +17,8 @@
 //
 // The (h+2)(w+2) positions are computed in full (outputs at padding positions are discarded): a
 // third more rows than pixels at 16x16, bought with tensor time that is idle anyway. One lane each
-// of two more warps issues the MMAs of a conv back to back (tiles dealt between them), one lane of a
-// last warp streams the taps' weight
+// of three more warps issues the MMAs of a conv back to back (tiles dealt between them, or the taps
+// when there is one tile), one lane of a last warp streams the taps' weight
 // slices from the packed blob through a ring, running ahead into the next conv; the 16 other warps
 // requantise. A block is
 //   MID = clip(ReLU(rq(conv_a(X))))                        kResHidden
@@ -169,14 +169,29 @@ __device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next, const in
         ptx::tc_fence_after();
         const int u = (tap * 11) >> 5;
         const int shift = (u - 1) * r.H->w2 + (tap - u * 3 - 1);
-        for (int tile = me; tile < r.ntiles; tile += kResIssuers) {
-          const uint32_t d = r.tmem + (uint32_t)(tile * kResMaxWidth);
-          uint32_t sa = a0 + (uint32_t)(tile * kTileM + shift);
-          uint32_t sb = ring0 + slot * slot16;
-          for (int k = 0; k < ksteps; ++k) {
-            ptx::umma_i8_lo(d, (sa & 0x3FFFu) | a_hi, (sb & 0x3FFFu) | b_hi, idesc, (tap > 0 || k > 0) ? 1u : 0u);
-            sa += 2u * rows;
-            sb += 2u * (uint32_t)c.n_pad;
+        if (r.ntiles == 1) {
+          // one tile: the taps are dealt between the issuers instead, each accumulating its own
+          // partial sum in its own TMEM columns (integer partial sums add up exactly in the epilogue)
+          if (tap % kResIssuers == me) {
+            const uint32_t d = r.tmem + (uint32_t)(me * kResMaxWidth);
+            uint32_t sa = a0 + (uint32_t)shift;
+            uint32_t sb = ring0 + slot * slot16;
+            for (int k = 0; k < ksteps; ++k) {
+              ptx::umma_i8_lo(d, (sa & 0x3FFFu) | a_hi, (sb & 0x3FFFu) | b_hi, idesc, (tap >= kResIssuers || k > 0) ? 1u : 0u);
+              sa += 2u * rows;
+              sb += 2u * (uint32_t)c.n_pad;
+            }
+          }
+        } else {
+          for (int tile = me; tile < r.ntiles; tile += kResIssuers) {
+            const uint32_t d = r.tmem + (uint32_t)(tile * kResMaxWidth);
+            uint32_t sa = a0 + (uint32_t)(tile * kTileM + shift);
+            uint32_t sb = ring0 + slot * slot16;
+            for (int k = 0; k < ksteps; ++k) {
+              ptx::umma_i8_lo(d, (sa & 0x3FFFu) | a_hi, (sb & 0x3FFFu) | b_hi, idesc, (tap > 0 || k > 0) ? 1u : 0u);
+              sa += 2u * rows;
+              sb += 2u * (uint32_t)c.n_pad;
+            }
           }
         }
         ptx::umma_commit(ptx::smem_u32(&r.ctl->w_empty[slot]));
@@ -234,6 +249,16 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
       __syncwarp();                                   // the tensor-memory load is a whole-warp instruction
       ptx::tmem_ld16(r.tmem + (uint32_t)(tile * kResMaxWidth + ch * 16) + ((uint32_t)(q * 32) << 16), acc);
       ptx::tmem_ld_wait16(acc);
+      if (r.ntiles == 1) {                            // the issuers' partial sums over their taps
+#pragma unroll
+        for (int part = 1; part < kResIssuers; ++part) {
+          uint32_t more[16];
+          ptx::tmem_ld16(r.tmem + (uint32_t)(part * kResMaxWidth + ch * 16) + ((uint32_t)(q * 32) << 16), more);
+          ptx::tmem_ld_wait16(more);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) acc[i] += more[i];
+        }
+      }
       if (!valid) {
         // rows beyond the image: nothing to store
       } else if (c.kind == kResHidden) {
