@@ -220,10 +220,35 @@ __device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next, const in
       for (int i = r.tid; i < c.n; i += kResThreads) ti[i] = colB[i];
     }
   }
+  asm volatile("bar.sync 1, %0;" ::"n"(kResThreads) : "memory");      // requantising warps: the staged tables are complete
+  if (c.kind == kResBranch) {
+    // The shortcut Q(x) of all channels, in place, at the image's positions, while the second conv is
+    // being multiplied: its MMAs read MID, and the block's first conv has read X already.
+    uint8_t* X = r.smem + r.H->s_x;
+    const uint8_t* lut = r.smem + r.H->s_tab + kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t));
+    const int chunks = r.H->x_pitch >> 4, px = r.g.px;
+    for (int it = r.tid; it < chunks * px; it += kResThreads) {
+      const int ch = it / px, p = it - ch * px;
+      const int pi = rdiv(p, r.g.mul_w), pj = p - pi * r.g.w;
+      const int rr = (pi + 1) * r.H->w2 + (pj + 1);
+      uint4* wp = reinterpret_cast<uint4*>(at(r, X, ch * 16, rr));
+      uint4 val = *wp;
+      uint32_t* wv = reinterpret_cast<uint32_t*>(&val);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const uint32_t in = wv[k];
+        uint32_t out = 0;
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) out |= (uint32_t)lut[(in >> (8 * jj)) & 0xFFu] << (8 * jj);
+        wv[k] = out;
+      }
+      *wp = val;
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kResThreads) : "memory");    // before the epilogue adds to X
+  }
   if (!ptx::mbar_test_wait(ptx::smem_u32(&r.ctl->conv_done), parity))
     res_wait(r.ctl, r.status, &r.ctl->conv_done, parity);
   ptx::tc_fence_after();
-  asm volatile("bar.sync 1, %0;" ::"n"(kResThreads) : "memory");      // requantising warps: the staged tables are complete
 }
 
 struct StepIo {            // what the epilogue of the last conv / the prior head needs
@@ -432,31 +457,6 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
       const bool has_next = ci + 1 < cp.n_convs;
       const ResConv nx = convs[cp.conv0 + (has_next ? ci + 1 : ci)];
       conv_mma(r, cv, has_next ? &nx : nullptr, io.colB);
-      if (cv.kind == kResBranch) {
-        // the shortcut Q(x) of all channels, in place, at the image's positions (the first conv of
-        // the block has read X already)
-        uint8_t* X = smem + H->s_x;
-        const uint8_t* lut = smem + H->s_tab + kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t));   // staged by conv_mma
-        const int chunks = H->x_pitch >> 4;
-        for (int it = tid; it < (builder ? chunks * px : 0); it += kResThreads) {
-          const int ch = it / px, p = it - ch * px;
-          const int pi = rdiv(p, P.mul_w), pj = p - pi * w;
-          const int rr = (pi + 1) * H->w2 + (pj + 1);
-          uint4* wp = reinterpret_cast<uint4*>(at(r, X, ch * 16, rr));
-          uint4 val = *wp;
-          uint32_t* wv = reinterpret_cast<uint32_t*>(&val);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const uint32_t in = wv[k];
-            uint32_t out = 0;
-#pragma unroll
-            for (int jj = 0; jj < 4; ++jj) out |= (uint32_t)lut[(in >> (8 * jj)) & 0xFFu] << (8 * jj);
-            wv[k] = out;
-          }
-          *wp = val;
-        }
-        __syncthreads();
-      }
       conv_epilogue(r, cv, io);
     }
   }
