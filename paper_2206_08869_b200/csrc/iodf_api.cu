@@ -439,9 +439,11 @@ int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P,
   int maxD = 32, maxK = 32, kmax = 32, nmax = 16;
   struct Src { const iodf_layer_desc* L; };
   std::vector<const iodf_layer_desc*> conv_layer;
-  auto add_conv = [&](const iodf_layer_desc& L, int kind, int src, int dst, bool a_unsigned) {
+  // `n`: outputs the kernel computes (a block's second conv is widened to the D channels it is added to)
+  auto add_conv = [&](const iodf_layer_desc& L, int kind, int src, int dst, bool a_unsigned, uint32_t n = 0) {
     ResConv c{};
-    c.n = (int)L.c_out; c.n_pad = (int)up(L.c_out, 16); c.kpad = (int)up(L.c_in, 32);
+    if (n == 0) n = L.c_out;
+    c.n = (int)n; c.n_pad = (int)up(n, 16); c.kpad = (int)up(L.c_in, 32);
     c.a_unsigned = a_unsigned; c.kind = kind; c.src = src; c.dst = dst;
     c.slice_bytes = (uint32_t)c.n_pad * (uint32_t)c.kpad;
     kmax = std::max(kmax, c.kpad); nmax = std::max(nmax, c.n_pad);
@@ -458,7 +460,7 @@ int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P,
     for (uint32_t b = 0; b < cp.n_blocks; ++b) {
       maxK = std::max(maxK, (int)up(cp.layers[1 + 2 * b].c_out, 32));
       add_conv(cp.layers[1 + 2 * b], kResHidden, 1, 2, true);
-      const int j = add_conv(cp.layers[2 + 2 * b], kResBranch, 2, 1, true);
+      const int j = add_conv(cp.layers[2 + 2 * b], kResBranch, 2, 1, true, cp.layers[0].c_out);
       convs[j].short_m0 = cp.blocks[b].short_m0; convs[j].short_s = cp.blocks[b].short_s;
     }
     add_conv(cp.layers[cp.n_layers - 1], kResOut, 1, 1, true);
@@ -491,20 +493,26 @@ int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P,
     const iodf_layer_desc& L = *conv_layer[ci];
     c.rq_off = place(sizeof(OutRq) * (size_t)c.n_pad);
     std::vector<OutRq> rq(c.n_pad, OutRq{1 << 30, 0, 1u << 30, 0u});          // padding: 0 -> 0
-    put_out_rq(rq.data(), L, B);
-    std::memcpy(blob.data() + c.rq_off, rq.data(), sizeof(OutRq) * rq.size());
-    if (c.kind == kResBranch) {
-      const iodf_resblock_desc& rb = *branch_block[block_of_branch++];
-      c.idx_off = place(4 * (size_t)c.n);
-      std::memcpy(blob.data() + c.idx_off, rb.idx, 4 * (size_t)c.n);
+    // Scatter add (Sec. 4.5) at pack time: filter j of a block's second conv becomes row idx[j] of a
+    // conv as wide as the shortcut. Rows without a filter have zero weights, no bias and requantise 0
+    // to 0, so the sum is the same and the kernel adds sixteen adjacent channels at a time.
+    const int32_t* row_of = nullptr;
+    if (c.kind == kResBranch) row_of = branch_block[block_of_branch++]->idx;
+    if (row_of) {
+      std::vector<OutRq> compact(L.c_out);
+      put_out_rq(compact.data(), L, B);
+      for (uint32_t j = 0; j < L.c_out; ++j) rq[row_of[j]] = compact[j];
+    } else {
+      put_out_rq(rq.data(), L, B);
     }
+    std::memcpy(blob.data() + c.rq_off, rq.data(), sizeof(OutRq) * rq.size());
     c.w_off = place(9 * (size_t)c.slice_bytes);
     const int8_t* w = B.w + L.weight_off;
     for (int tap = 0; tap < 9; ++tap) {
       uint8_t* sl = blob.data() + c.w_off + (size_t)tap * c.slice_bytes;
-      for (int n = 0; n < c.n; ++n)
+      for (uint32_t n = 0; n < L.c_out; ++n)
         for (uint32_t k = 0; k < L.c_in; ++k)
-          sl[wpos(c.n_pad, n, (int)k)] = (uint8_t)w[((size_t)n * 9 + tap) * L.c_in + k];
+          sl[wpos(c.n_pad, row_of ? row_of[n] : (int)n, (int)k)] = (uint8_t)w[((size_t)n * 9 + tap) * L.c_in + k];
     }
   }
   // shared memory: flow variable, the three activation buffers in the padded chunk-major layout

@@ -25,7 +25,11 @@
 //   X   = rq(X; M_r, s_r)      for all D channels          the shortcut Q(x), in place
 //   X[idx[j]] = clip(max(X[idx[j]] + rq(conv_b(MID))[j], 0), 0, 255)   kResBranch: scatter add + ReLU
 // which equals Eq. 3 with the scatter add because rq(X) of an 8-bit X with a multiplier below one
-// is again in 0..255, and channels that the second conv does not keep only get the shortcut.
+// is again in 0..255, and channels that the second conv does not keep only get the shortcut. The
+// scatter itself happens when the level is packed: conv_b's filter j is stored as row idx[j] of a
+// D-row weight matrix (zero rows, which requantise to 0, elsewhere), so the kernel's update is a
+// plain 16-channel-wide add. The extra rows cost tensor time that is idle; byte-wise scattered
+// updates cost shared-memory bank conflicts that were not.
 //
 // This is a first version of the path: convs run one after another, a conv's epilogue does not
 // overlap the next conv's MMAs.
@@ -165,22 +169,23 @@ __device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next, const in
       for (int tap = 0; tap < 9; ++tap) {
         const uint32_t g = r.gslice++;
         const uint32_t slot = g % nws;
+        // one tile: the taps are dealt between the issuers, and a tap's slice is waited for and
+        // released by its issuer alone (w_empty then counts one arrival)
+        if (r.ntiles == 1 && tap % kResIssuers != me) continue;
         res_wait_fast(r.ctl, r.status, &r.ctl->w_full[slot], (g / nws) & 1u);
         ptx::tc_fence_after();
         const int u = (tap * 11) >> 5;
         const int shift = (u - 1) * r.H->w2 + (tap - u * 3 - 1);
         if (r.ntiles == 1) {
-          // one tile: the taps are dealt between the issuers instead, each accumulating its own
-          // partial sum in its own TMEM columns (integer partial sums add up exactly in the epilogue)
-          if (tap % kResIssuers == me) {
-            const uint32_t d = r.tmem + (uint32_t)(me * kResMaxWidth);
-            uint32_t sa = a0 + (uint32_t)shift;
-            uint32_t sb = ring0 + slot * slot16;
-            for (int k = 0; k < ksteps; ++k) {
-              ptx::umma_i8_lo(d, (sa & 0x3FFFu) | a_hi, (sb & 0x3FFFu) | b_hi, idesc, (tap >= kResIssuers || k > 0) ? 1u : 0u);
-              sa += 2u * rows;
-              sb += 2u * (uint32_t)c.n_pad;
-            }
+          // each issuer accumulates a partial sum over its taps in its own TMEM columns (integer
+          // partial sums add up exactly in the epilogue)
+          const uint32_t d = r.tmem + (uint32_t)(me * kResMaxWidth);
+          uint32_t sa = a0 + (uint32_t)shift;
+          uint32_t sb = ring0 + slot * slot16;
+          for (int k = 0; k < ksteps; ++k) {
+            ptx::umma_i8_lo(d, (sa & 0x3FFFu) | a_hi, (sb & 0x3FFFu) | b_hi, idesc, (tap >= kResIssuers || k > 0) ? 1u : 0u);
+            sa += 2u * rows;
+            sb += 2u * (uint32_t)c.n_pad;
           }
         } else {
           for (int tile = me; tile < r.ntiles; tile += kResIssuers) {
@@ -208,9 +213,6 @@ __device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next, const in
     const uint4* src_rq = reinterpret_cast<const uint4*>(r.blob + c.rq_off);
     for (int i = r.tid; i < c.n_pad; i += kResThreads) tab[i] = src_rq[i];
     if (c.kind == kResBranch) {
-      int32_t* ti = reinterpret_cast<int32_t*>(tab + kResMaxWidth);
-      const int32_t* si = reinterpret_cast<const int32_t*>(r.blob + c.idx_off);
-      for (int i = r.tid; i < c.n; i += kResThreads) ti[i] = si[i];
       // the block's shortcut rq(x; M_r, s_r) as a table over the 256 values of an 8-bit x
       uint8_t* lut = r.smem + r.H->s_tab + kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t));
       if (r.tid < 256) lut[r.tid] = (uint8_t)clampi(rq64(r.tid, c.short_m0, c.short_s), 0, 255);
@@ -301,21 +303,25 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
         }
         *reinterpret_cast<uint4*>(at(r, dst, ch * 16, rr)) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
       } else if (c.kind == kResBranch) {
-        // all sixteen shortcut bytes are read before any is written back (a byte store could alias
-        // anything for the compiler and would otherwise serialise the sixteen updates)
-        uint8_t* xp[16];
-        int xv[16];
+        // The conv's outputs sit at their channels of X already (the scatter add was done on the
+        // weights, when the level was packed; a channel without a filter requantises 0 to 0), so the
+        // update is sixteen adjacent bytes: one 16-byte read of the shortcut, one 16-byte write.
+        uint4* xp = reinterpret_cast<uint4*>(at(r, dst, ch * 16, rr));
+        const uint4 xv = *xp;
+        const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+        uint32_t wd[4];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int col = ch * 16 + i;
-          xp[i] = at(r, dst, col < c.n ? idx[col] : 0, rr);
-          xv[i] = *xp[i];
-        }
+        for (int i = 0; i < 4; ++i) {
+          uint32_t word = 0;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int col = ch * 16 + i;
-          if (col < c.n) *xp[i] = (uint8_t)clampi(xv[i] + rq_const((int32_t)acc[i], orq[col]), 0, 255);
+          for (int jj = 0; jj < 4; ++jj) {
+            const int col = ch * 16 + i * 4 + jj;
+            const int y = clampi((int)((xw[i] >> (8 * jj)) & 0xFFu) + rq_const((int32_t)acc[i * 4 + jj], orq[col]), 0, 255);
+            word |= (uint32_t)y << (8 * jj);
+          }
+          wd[i] = word;
         }
+        *xp = make_uint4(wd[0], wd[1], wd[2], wd[3]);
       } else {
 #pragma unroll 4
         for (int i = 0; i < 16; ++i) {
@@ -364,7 +370,8 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
   if (tid == 0) {
     for (int s = 0; s < kResMaxWSlots; ++s) {
       ptx::mbar_init(ptx::smem_u32(&ctl.w_full[s]), 1);
-      ptx::mbar_init(ptx::smem_u32(&ctl.w_empty[s]), (uint32_t)kResIssuers);      // every issuer commits to it
+      // a slot is released by every issuer that read it: all of them, or the tap's one at single-tile levels
+      ptx::mbar_init(ptx::smem_u32(&ctl.w_empty[s]), H->ntiles == 1 ? 1u : (uint32_t)kResIssuers);
     }
     ptx::mbar_init(ptx::smem_u32(&ctl.conv_done), (uint32_t)kResIssuers);
     ptx::mbar_init_fence();

@@ -22,7 +22,8 @@ constexpr int kResMaxWSlots = 8;       // depth of the weight-slice ring
 // what a conv's epilogue does with its requantised outputs
 enum ResKind : int32_t {
   kResHidden = 0,     // ReLU + clip to 0..255, written as bytes to the conv's destination buffer
-  kResBranch = 1,     // second conv of a block: added through idx[] to the (already requantised) shortcut in X
+  kResBranch = 1,     // second conv of a block, as wide as X (its filters sit at the rows idx[] names, zero
+                      // rows elsewhere): added channel by channel to the (already requantised) shortcut in X
   kResOut = 2,        // last conv: the translation, added to / subtracted from the flow variable
   kResPrior = 3       // prior head: mu and clipped log-scale index to global memory
 };
@@ -32,7 +33,7 @@ struct ResConv {
   uint32_t w_off;          // blob offset of slice 0
   uint32_t slice_bytes;    // n_pad * kpad
   uint32_t rq_off;         // blob offset of OutRq[n_pad] (padding channels requantise 0 to 0)
-  uint32_t idx_off;        // kResBranch: blob offset of int32 idx[n]
+  uint32_t idx_off;        // unused (the index list of a block is applied when the level is packed)
   int32_t n, n_pad;        // outputs, and padded to 16
   int32_t kpad;            // input bytes per pixel and tap, a multiple of 32 (<= the source's pitch)
   int32_t a_unsigned;      // input is unsigned 8-bit (hidden activations) or signed (network / head input)
