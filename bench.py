@@ -281,7 +281,7 @@ def main():
                     G.iodf_inverse_level(m, lv, G.IODF_LEVEL_PRIOR, zs[k], prior=ps[k])
                 G.iodf_inverse_level(m, lv, G.IODF_LEVEL_COUPLINGS, zs[k], x_u8=xo[k])
         ms = timed(stepped, dec_steps)
-        ok = bool(all(torch.equal(xo[i], xs[i]) for i in range(min(N_SETS, dec_steps))))
+        ok = bool(all(torch.equal(xo[i], xs[i]) for i in range(min(N_SETS, args.steps + args.warmup))))   # the sets that were encoded
         extra["decode_level_stepped"] = {"value": B / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
                                          "launches_per_step": L + sum(has_prior), "round_trip_exact": ok}
         # the batch as the patch grid of one image: patches_y x patches_x patches of the model's input size
