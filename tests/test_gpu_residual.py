@@ -54,6 +54,32 @@ def test_residual_models_bit_exact(G, hw, splits, couplings, hidden, blocks, pru
     _both_ways(G, model, x)
 
 
+def test_index_lists_in_any_order_and_chunks_without_a_filter(G):
+    """Sec. 4.5: the kept outputs go back to the channels the index list names, whatever its order.
+    Here every block's list is shuffled (its filters stay paired with their channels' positions in
+    the list), and the first block of each coupling keeps nothing among channels 16..31, so a whole
+    16-channel group of the block tensor only gets the shortcut."""
+    model = S.make_residual_model(0xE800, 3, 16, 16, [True, True], 2, 48, 3, prune=(0.3, 0.6))
+    rng = np.random.default_rng(0xE801)
+    for lv in model["levels"]:
+        for cp in lv["couplings"]:
+            for b, rb in enumerate(cp["blocks"]):
+                ly = cp["layers"][2 + 2 * b]
+                keep = np.arange(len(rb["idx"]))
+                if b == 0:
+                    keep = keep[(rb["idx"] < 16) | (rb["idx"] >= 32)]
+                keep = rng.permutation(keep)
+                rb["idx"] = np.ascontiguousarray(rb["idx"][keep])
+                for k in ("w", "bias", "m0", "s"):
+                    ly[k] = np.ascontiguousarray(ly[k][keep])
+                if ly.get("gate") is not None:
+                    ly["gate"] = np.ascontiguousarray(ly["gate"][keep])
+                ly["c_out"] = len(keep)
+                assert len(keep) > 0 and not np.all(np.diff(rb["idx"]) > 0)
+    x = S.smooth_field_images(0xE802, 3, 16, 16, 2.0)
+    _both_ways(G, model, x)
+
+
 def test_residual_and_plain_levels_in_one_model_and_stepped_decode(G):
     """A model whose first level uses residual couplings and whose second the three-conv couplings;
     decoded level by level with the blocks that are not decoded yet poisoned."""
