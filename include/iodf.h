@@ -45,7 +45,7 @@ typedef enum {
   IODF_ETIMEOUT = -5,     /* a bounded device-side wait gave up (reported by iodf_check)             */
   IODF_EUNSUPPORTED = -6, /* a valid model whose shape this build cannot run (see iodf_create)       */
   IODF_EOVERFLOW = -7,    /* a worst-case accumulator |sum| + |bias| would leave the int32 range     */
-  IODF_ELIMIT = -8,       /* the request needs more than the fixed scratch of iodf_forward_static   */
+  IODF_ELIMIT = -8,       /* the request exceeds a fixed capacity (static scratch, output buffer)    */
   IODF_EDATA = -9         /* entropy coder: a scale index outside the table or a malformed stream   */
 } iodf_status;
 
@@ -67,10 +67,9 @@ typedef struct {
 } iodf_layer_desc;
 
 /*
- * One additive coupling (Eq. 2, Sec. 3). Before the coupling the C channels are permuted,
- * y[k] = x[perm[k]]; x_a = y[0 : C/2] feeds the network, x_b = y[C/2 : C] is updated:
- *   a0 = clip(rq(x_a; in_m0, in_s), -128, 127);  t = layers(a0);  z_b = x_b + t  (mod 2^32).
- * The last layer must have relu = 0 and has_clamp = 0 (its rq output is the integer translation).
+ * One residual block of a coupling network (Eq. 3, Sec. 4.1; scatter add of Sec. 4.5): how the
+ * block's shortcut is requantised, how the sum is clipped, and which of the D channels of the
+ * block tensor each kept output of the block's second conv is added to (see iodf_coupling_desc).
  */
 typedef struct {
   int32_t short_m0, short_s;      /* shortcut requantisation Q(x) of the block, per tensor           */
@@ -80,6 +79,11 @@ typedef struct {
 } iodf_resblock_desc;
 
 /*
+ * One additive coupling (Eq. 2, Sec. 3). Before the coupling the C channels are permuted,
+ * y[k] = x[perm[k]]; x_a = y[0 : C/2] feeds the network, x_b = y[C/2 : C] is updated:
+ *   a0 = clip(rq(x_a; in_m0, in_s), -128, 127);  t = layers(a0);  z_b = x_b + t  (mod 2^32).
+ * The last layer must have relu = 0 and has_clamp = 0 (its rq output is the integer translation).
+ *
  * With n_blocks > 0 the network is the residual form of Eq. 3 (Sec. 4.1) with the scatter add of
  * Sec. 4.5 (App. B.1: eight blocks, 3x3 convs, 128 hidden channels): layers = [conv_in,
  * (conv_a, conv_b) per block, conv_out], n_layers = 2 + 2 n_blocks. conv_in maps the requantised
@@ -87,8 +91,8 @@ typedef struct {
  *   m = clip(ReLU(rq(conv_a(x))));  b = rq(conv_b(m))   (conv_b: relu = 0, has_clamp = 0, K' kept outputs)
  *   x = clip(max(rq(x; short_m0, short_s) [all D channels]  +  scatter of b through idx, 0), clamp_lo, clamp_hi)
  * and conv_out maps x to the integer translation. This build runs it for 3x3 convs with D and every
- * kept width <= 128, hidden activations in 0..255, and levels of at most 256 pixels per image;
- * all couplings of a level must then be of this form.
+ * kept width <= 128, hidden activations in 0..255, and levels of at most 256 pixels per
+ * image; all couplings of a level must then be of this form.
  */
 typedef struct {
   const int32_t* perm;            /* HOST, C entries, a permutation of 0..C-1                        */
@@ -164,13 +168,19 @@ void iodf_destroy(iodf_model* m);
 int iodf_get_layout(const iodf_model* m, iodf_layout* out);
 
 /*
- * Encode: x_u8 DEV uint8 [B][in_c][in_h][in_w]  ->  z DEV int32 [B][d] and, if `prior` is not
- * NULL, prior DEV int32 [B][2][d_fact]. 1 <= B <= max_batch. Pointers must be 16-byte aligned.
+ * Encode, z = f(x) (Sec. 3: the flow is the composition of the levels' additive couplings, Eq. 2,
+ * with the coupling networks evaluated in integers, Sec. 4.1; App. B.1 for the level structure):
+ * x_u8 DEV uint8 [B][in_c][in_h][in_w]  ->  z DEV int32 [B][d] and, if `prior` is not NULL, prior
+ * DEV int32 [B][2][d_fact] (the (mu, s) of Sec. 3's discretised logistic prior for every
+ * factored-out element). 1 <= B <= max_batch. Pointers must be 16-byte aligned. Enqueues one
+ * kernel per level on `cuda_stream`; allocates nothing; the caller owns all three buffers.
+ * Errors: IODF_EINVAL (null or misaligned pointer, B out of range), IODF_ECUDA (launch failure).
  */
 int iodf_forward(iodf_model* m, const uint8_t* x_u8, int B, int32_t* z, int32_t* prior, void* cuda_stream);
 
 /*
- * Decode: z DEV int32 [B][d] -> x_u8 DEV uint8 [B][in_c][in_h][in_w] (the low 8 bits of each
+ * Decode, x = f^-1(z) (Eq. 2 inverted: x_b = z_b - round(t(z_a)), levels and couplings in reverse
+ * order, Sec. 3): z DEV int32 [B][d] -> x_u8 DEV uint8 [B][in_c][in_h][in_w] (the low 8 bits of each
  * recovered value). If `prior` is not NULL the same prior parameters as iodf_forward are written.
  * If `out_of_range_count` (DEV uint32) is not NULL, the number of recovered values outside 0..255
  * is ADDED to it (the caller zeroes it); this can only be non-zero for a z that no image encodes to.
@@ -206,7 +216,7 @@ int iodf_inverse_level(iodf_model* m, int level, int phase, const int32_t* z, in
 
 /*
  * Patch-based coding of one high-resolution image (Sec. 5.3: a large image is cut into patches
- * of the training resolution, which "naturally gives rise to a large batch size"). image_u8 is DEV
+ * of the training resolution, so one image already is a large batch). image_u8 is DEV
  * uint8 [in_c][H][W] with H, W multiples of in_h, in_w; patch b = (b / (W/in_w), b % (W/in_w)) in
  * row-major order is image b of a batch of B = (H/in_h)*(W/in_w) <= max_batch images. The cut is an
  * index map of the first level's load (encode) and last store (decode): no patch batch is
@@ -220,7 +230,7 @@ int iodf_inverse_patches(iodf_model* m, const int32_t* z, int H, int W, uint8_t*
 
 /*
  * Entropy coding of the latents on the GPU (Sec. 3: factorised discrete logistic prior; App. A:
- * range-ANS; Sec. 5.3 leaves "an optimized GPU implementation of rANS" as future work).
+ * range-ANS; Sec. 5.3 codes on the CPU and names a GPU coder as future work).
  *
  * The prior's integer form is given by the caller (HOST arrays, copied):
  *   sigmoid_table[u + umax], u in [-umax, umax], umax <= 8192: a non-decreasing table of
@@ -373,6 +383,27 @@ int iodf_inverse_timed(iodf_model* m, const int32_t* z, int B, uint8_t* x_u8, in
 int iodf_forward_static(iodf_model* m, const uint8_t* x_u8, int B, int32_t* z, int32_t* prior, void* cuda_stream);
 /* Bytes of the fixed array one image needs for this model (0 for a single-level model). */
 size_t iodf_static_scratch_bytes_per_image(const iodf_model* m);
+
+/*
+ * Self-test of the failure path (the paper has no counterpart). Every device-side wait of the
+ * library is bounded: when its tries run out it sets the model's status word and the kernel drains
+ * and returns, which iodf_check reports as IODF_ETIMEOUT. This call enqueues a one-warp kernel that
+ * runs that same wait, with `tries` (1..100) suspended tries of up to 100 us each, on a barrier that
+ * nothing arrives on, so that the path can be exercised without a fault: afterwards iodf_check
+ * returns IODF_ETIMEOUT once, then IODF_OK, and the model works as before.
+ */
+int iodf_selftest_timeout(iodf_model* m, uint32_t tries, void* cuda_stream);
+
+/*
+ * The tensor roofline's denominator, measured (the paper has no counterpart; Sec. 4.1's point is
+ * that the 8-bit multiply-accumulates dominate). Enqueues one kernel in which one CTA per SM issues
+ * mma_groups * 8 tcgen05.mma kind::i8 instructions of shape 128 x 256 x 32 (int8 x int8 -> int32 in
+ * tensor memory) from operands resident in shared memory, and nothing else. *ops_out (HOST, may be
+ * NULL) receives the int8 OPs (2 per multiply-accumulate) of the launch; the caller times the
+ * launch with events on `cuda_stream`. mma_groups in [1, 2^22]; m only supplies the device and
+ * the status word of the kernel's bounded wait (check with iodf_check).
+ */
+int iodf_int8_mma_peak(iodf_model* m, uint32_t mma_groups, void* cuda_stream, unsigned long long* ops_out);
 
 /* Number of kernel launches one iodf_forward / iodf_inverse call enqueues. */
 int iodf_launches_per_call(const iodf_model* m, int inverse);

@@ -9,7 +9,8 @@ from .binding import (IodfError, Model, iodf_create, iodf_destroy, iodf_forward,
                       iodf_forward_host, iodf_inverse_host, iodf_forward_timed, iodf_inverse_timed,
                       iodf_get_layout, iodf_forward_static, iodf_static_scratch_bytes_per_image,
                       IODF_STATIC_SCRATCH_BYTES, iodf_check, iodf_strerror,
-                      iodf_launches_per_call, load_library, DECLARED_SYMBOLS)
+                      iodf_launches_per_call, iodf_selftest_timeout, iodf_int8_mma_peak, load_library,
+                      DECLARED_SYMBOLS)
 
 __all__ = ["IodfError", "Model", "iodf_create", "iodf_destroy", "iodf_forward", "iodf_inverse",
            "iodf_inverse_level", "IODF_LEVEL_PRIOR", "IODF_LEVEL_COUPLINGS", "iodf_forward_patches",
@@ -18,4 +19,5 @@ __all__ = ["IodfError", "Model", "iodf_create", "iodf_destroy", "iodf_forward", 
            "iodf_compress_host", "iodf_decompress_host",
            "iodf_forward_host", "iodf_inverse_host", "iodf_forward_timed", "iodf_inverse_timed", "iodf_get_layout", "iodf_forward_static", "iodf_static_scratch_bytes_per_image",
            "IODF_STATIC_SCRATCH_BYTES", "iodf_check", "iodf_strerror",
-           "iodf_launches_per_call", "load_library", "DECLARED_SYMBOLS"]
+           "iodf_launches_per_call", "iodf_selftest_timeout", "iodf_int8_mma_peak", "load_library",
+           "DECLARED_SYMBOLS"]

@@ -18,6 +18,7 @@ DECLARED_SYMBOLS = ["iodf_create", "iodf_destroy", "iodf_get_layout", "iodf_forw
                     "iodf_rans_unpack", "iodf_compress_host", "iodf_decompress_host",
                     "iodf_forward_host", "iodf_inverse_host", "iodf_forward_timed", "iodf_inverse_timed", "iodf_forward_static",
                     "iodf_static_scratch_bytes_per_image", "iodf_check", "iodf_launches_per_call",
+                    "iodf_selftest_timeout", "iodf_int8_mma_peak",
                     "iodf_strerror", "iodf_last_cuda_error"]
 
 
@@ -143,6 +144,10 @@ def load_library(path=None):
     L.iodf_static_scratch_bytes_per_image.argtypes = [vp]
     L.iodf_check.restype = C.c_int
     L.iodf_check.argtypes = [vp, vp]
+    L.iodf_selftest_timeout.restype = C.c_int
+    L.iodf_selftest_timeout.argtypes = [vp, C.c_uint32, vp]
+    L.iodf_int8_mma_peak.restype = C.c_int
+    L.iodf_int8_mma_peak.argtypes = [vp, C.c_uint32, vp, C.POINTER(C.c_ulonglong)]
     L.iodf_launches_per_call.restype = C.c_int
     L.iodf_launches_per_call.argtypes = [vp, C.c_int]
     L.iodf_strerror.restype = C.c_char_p
@@ -500,6 +505,21 @@ def iodf_check(model, stream=None):
     rc = load_library().iodf_check(model.handle, _stream(stream))
     if rc != 0:
         raise IodfError(rc, "iodf_check")
+
+
+def iodf_selftest_timeout(model, tries=3, stream=None):
+    rc = load_library().iodf_selftest_timeout(model.handle, int(tries), _stream(stream))
+    if rc != 0:
+        raise IodfError(rc, "iodf_selftest_timeout")
+
+
+def iodf_int8_mma_peak(model, mma_groups, stream=None):
+    """Enqueue the MMA-only kernel; returns the int8 OPs of the launch."""
+    ops = C.c_ulonglong(0)
+    rc = load_library().iodf_int8_mma_peak(model.handle, int(mma_groups), _stream(stream), C.byref(ops))
+    if rc != 0:
+        raise IodfError(rc, "iodf_int8_mma_peak")
+    return int(ops.value)
 
 
 def iodf_launches_per_call(model, inverse=False):

@@ -15,6 +15,7 @@
 #include "rans_kernel.h"
 #include "res_level.h"
 #include "level_kernel.h"
+#include "selftest.h"
 
 using namespace iodf;
 
@@ -28,6 +29,7 @@ struct HostLevel {
   LevelPlan plan;
   std::vector<uint8_t> blob;
   int grid_group = 1;
+  int32_t ls_lo = 0, ls_hi = 0;      // clip of the prior head's log-scale index (levels with a head)
 };
 
 }  // namespace
@@ -664,6 +666,7 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
     P.c = (int)c; P.h = (int)h; P.w = (int)w; P.px = (int)(h * w); P.ca = ca; P.cb = cb;
     P.n_couplings = (int)lv.n_couplings;
     P.split = lv.split ? 1 : 0; P.has_prior = lv.has_prior ? 1 : 0;
+    hl.ls_lo = lv.ls_lo; hl.ls_hi = lv.ls_hi;
     P.is_first = li == 0; P.is_last = li + 1 == desc->n_levels;
     P.keep_c = lv.split ? ca : (int)c;
     P.z_off = lay.z_off[li]; P.prior_off = lay.prior_off[li]; P.z_final_off = lay.z_final_off;
@@ -1112,7 +1115,11 @@ int iodf_codec_create(const iodf_model* m, const iodf_codec_desc* desc, iodf_cod
   for (size_t li = 0; li < m->levels.size(); ++li) {
     const LevelPlan& P = m->levels[li].plan;
     if (!P.split) continue;
-    // the scale indices a prior head can emit must be table entries
+    // every scale index a prior head of this level can emit must be an entry of the scale table
+    if (P.has_prior && (m->levels[li].ls_lo < 0 || m->levels[li].ls_hi >= (int32_t)desc->n_scales)) {
+      delete c;
+      return IODF_EINVAL;
+    }
     add_block(P.z_off, (uint64_t)P.cb * P.px, P.has_prior ? (long long)P.prior_off : -1);
     c->layout.block_level[nb - 1] = (int32_t)li;
   }
@@ -1120,10 +1127,14 @@ int iodf_codec_create(const iodf_model* m, const iodf_codec_desc* desc, iodf_cod
   a.n_blocks = nb; a.n_streams = first;
   c->layout.n_blocks = (uint32_t)nb; c->layout.n_streams = (uint32_t)first; c->layout.words_per_stream = (uint32_t)a.cap;
   int prev = -1;
-  CUC(c, cudaGetDevice(&prev));
-  CUC(c, cudaSetDevice(c->device));
   const size_t rbytes = 4 * (size_t)desc->n_scales, gbytes = 2 * (size_t)(2 * desc->umax + 1);
-  cudaError_t e = cudaMalloc(&c->d_tables, rbytes + gbytes);
+  cudaError_t e = cudaGetDevice(&prev);
+  if (e == cudaSuccess) e = cudaSetDevice(c->device);
+  if (e != cudaSuccess) {
+    delete c;
+    return IODF_ECUDA;
+  }
+  e = cudaMalloc(&c->d_tables, rbytes + gbytes);
   if (e == cudaSuccess) e = cudaMemcpy(c->d_tables, desc->inv_scale, rbytes, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemcpy(c->d_tables + rbytes, desc->sigmoid_table, gbytes, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMalloc(&c->d_errors, sizeof(uint32_t));
@@ -1365,6 +1376,20 @@ int iodf_check(iodf_model* m, void* cuda_stream) {
   return IODF_OK;
 }
 
+int iodf_selftest_timeout(iodf_model* m, uint32_t tries, void* cuda_stream) {
+  if (!m || tries < 1 || tries > 100u) return IODF_EINVAL;
+  CU(m, launch_timeout_probe(m->d_status, tries, (cudaStream_t)cuda_stream));
+  return IODF_OK;
+}
+
+int iodf_int8_mma_peak(iodf_model* m, uint32_t mma_groups, void* cuda_stream, unsigned long long* ops_out) {
+  if (!m || mma_groups < 1 || mma_groups > (1u << 22)) return IODF_EINVAL;
+  int sms = 0;
+  CU(m, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, m->device));
+  CU(m, launch_int8_mma_peak(m->d_status, mma_groups, sms, (cudaStream_t)cuda_stream, ops_out));
+  return IODF_OK;
+}
+
 int iodf_launches_per_call(const iodf_model* m, int inverse) {
   (void)inverse;
   return m ? (int)m->levels.size() : 0;
@@ -1380,7 +1405,7 @@ const char* iodf_strerror(int status) {
     case IODF_ETIMEOUT: return "a bounded device-side wait gave up";
     case IODF_EUNSUPPORTED: return "model shape not supported by this build";
     case IODF_EOVERFLOW: return "worst-case accumulator leaves the int32 range";
-    case IODF_ELIMIT: return "request exceeds the fixed scratch of iodf_forward_static";
+    case IODF_ELIMIT: return "request exceeds a fixed capacity (static scratch or caller's output buffer)";
     case IODF_EDATA: return "entropy coder: scale index outside the table or malformed stream";
     default: return "unknown status";
   }

@@ -65,19 +65,9 @@ struct Ctx {
   uint32_t tmem_slot;     // current tile slot's first column, this warp's lane quarter
 };
 
-// Bounded wait on an mbarrier phase. After one wait in the CTA has given up, every later wait
-// returns at once, so a stuck CTA drains in bounded time, frees its TMEM and exits.
-__device__ __noinline__ bool wait_bar(Ctl* ctl, uint32_t* status, uint64_t* bar, uint32_t parity) {
-  volatile uint32_t* ab = &ctl->abort;
-  if (*ab) return false;
-  const uint32_t b = ptx::smem_u32(bar);
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (ptx::mbar_try_wait(b, parity)) return true;
-    if (*ab) return false;
-  }
-  *ab = 1;
-  atomicExch(status, 1u);
-  return false;
+// Bounded wait of this kernel: see ptx::bounded_wait.
+__device__ __forceinline__ bool wait_bar(Ctl* ctl, uint32_t* status, uint64_t* bar, uint32_t parity) {
+  return ptx::bounded_wait(&ctl->abort, status, bar, parity, kSpinLimit);
 }
 
 // The control thread's waits are short and on the critical path of every tile phase: it polls

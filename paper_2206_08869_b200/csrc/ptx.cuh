@@ -47,6 +47,23 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+// Bounded wait on an mbarrier phase: at most `limit` suspended tries (each up to 100 us). When the
+// limit runs out the CTA's abort flag and the device status word are set and the wait returns
+// false; once the abort flag is set every later wait of the CTA returns false at once, so a stuck
+// CTA drains in bounded time, frees its tensor memory and exits.
+static __device__ __noinline__ bool bounded_wait(volatile uint32_t* abort_flag, uint32_t* status, uint64_t* bar,
+                                                 uint32_t parity, uint32_t limit) {
+  if (*abort_flag) return false;
+  const uint32_t b = smem_u32(bar);
+  for (uint32_t it = 0; it < limit; ++it) {
+    if (mbar_try_wait(b, parity)) return true;
+    if (*abort_flag) return false;
+  }
+  *abort_flag = 1;
+  atomicExch(status, 1u);
+  return false;
+}
+
 // Predicated fire-and-forget add to a 32-bit word in shared memory.
 __device__ __forceinline__ void red_add_s32(uint32_t saddr, int val, bool pred) {
   asm volatile(

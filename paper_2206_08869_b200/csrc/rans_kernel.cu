@@ -2,7 +2,7 @@
 // table form and range-ANS (App. A) with a 32-bit state renormalised in 16-bit words, one thread
 // per stream. The streams are independent (an image's coded blocks are cut into streams of about
 // `elems_per_stream` interleaved elements), so a batch of 128 ImageNet64-sized latents is 6 144
-// streams: the paper's "optimized GPU implementation of rANS" left as future work (Sec. 5.3).
+// streams: the GPU coder that Sec. 5.3 names as future work (the paper codes on the CPU).
 //
 //   symbol of an element   k = clamp(z - mu, -2048, 2048) + 2048          (0 and 4096: escapes, then
 //                                                                          z follows as 2 x 16 raw bits)

@@ -48,18 +48,9 @@ struct __align__(16) ResCtl {
   uint32_t abort;
 };
 
-// bounded wait on an mbarrier phase; after one wait has given up every later one returns at once
-__device__ __noinline__ bool res_wait(ResCtl* ctl, uint32_t* status, uint64_t* bar, uint32_t parity) {
-  volatile uint32_t* ab = &ctl->abort;
-  if (*ab) return false;
-  const uint32_t b = ptx::smem_u32(bar);
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (ptx::mbar_try_wait(b, parity)) return true;
-    if (*ab) return false;
-  }
-  *ab = 1;
-  atomicExch(status, 1u);
-  return false;
+// bounded wait of this kernel: see ptx::bounded_wait
+__device__ __forceinline__ bool res_wait(ResCtl* ctl, uint32_t* status, uint64_t* bar, uint32_t parity) {
+  return ptx::bounded_wait(&ctl->abort, status, bar, parity, kSpinLimit);
 }
 
 // usually the phase has completed already: probe inline before the bounded blocking wait
@@ -316,7 +307,10 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
 #pragma unroll
           for (int jj = 0; jj < 4; ++jj) {
             const int col = ch * 16 + i * 4 + jj;
-            const int y = clampi((int)((xw[i] >> (8 * jj)) & 0xFFu) + rq_const((int32_t)acc[i * 4 + jj], orq[col]), 0, 255);
+            // the branch value is clipped to +-255 first: the sum then stays far inside 32 bits for
+            // any requantisation constants, and the clip to 0..255 below gives the same result
+            const int br = clampi(rq_const((int32_t)acc[i * 4 + jj], orq[col]), -255, 255);
+            const int y = clampi((int)((xw[i] >> (8 * jj)) & 0xFFu) + br, 0, 255);
             word |= (uint32_t)y << (8 * jj);
           }
           wd[i] = word;

@@ -125,3 +125,19 @@ def test_config_r32_in_the_benchmarks_launch_configuration(G):
     # an image's result does not depend on the batch around it
     z1, _ = G.iodf_forward(m, _t(x[5:6]))
     assert torch.equal(z1[0], z[5])
+
+
+def test_branch_output_near_the_int32_limit(G):
+    """A block's second conv with shift 0, a multiplier just under one and biases as large as the
+    accumulator bound allows: its requantised outputs reach +-(2^31 - 2), and adding the shortcut
+    byte must still clip to 0..255 as the oracle's 64-bit sum does."""
+    model = S.make_residual_model(0xE900, 3, 8, 8, [True], 1, 16, 2, prune=None)
+    for cp in model["levels"][0]["couplings"]:
+        ly = cp["layers"][2]                       # conv_b of the first block
+        worst = np.abs(ly["w"].astype(np.int64)).reshape(ly["c_out"], -1).sum(axis=1) * 255
+        big = (2 ** 31 - 1) - worst
+        ly["bias"][:] = np.where(np.arange(ly["c_out"]) % 2 == 0, big, -big).astype(np.int32)
+        ly["m0"][:] = 2 ** 31 - 1
+        ly["s"][:] = 0
+    x = S.smooth_field_images(0xE901, 2, 8, 8, 2.0)
+    _both_ways(G, model, x)

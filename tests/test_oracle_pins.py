@@ -307,3 +307,70 @@ def test_bad_descriptors_are_rejected():
     model["levels"][0]["couplings"][0]["layers"][0]["m0"][0] = 5
     with pytest.raises(ValueError):
         O.Packed(model)
+
+
+# ---- prior head: (mu, s) of the factored-out half from the kept half (Sec. 3, App. B.1) ---------
+def _clip(v, lo, hi):
+    return min(max(v, lo), hi)
+
+
+def test_prior_head_one_pixel_against_rational_arithmetic():
+    """A 1x1-pixel level: the head's 3x3 conv is its centre tap, so mu and the log-scale index can be
+    written out with exact fractions: input requant with its clip to -128..127 (one kept value is
+    large enough to hit 127), dot product, bias, per-channel rq, clip of the log-scale half only."""
+    model = _zero_model(S.make_model(81, 1, 2, 2, [True], 1, 3, prune=None, prior=True, perm="reverse"))
+    hd = model["levels"][0]["prior"]
+    hd["in_m0"], hd["in_s"] = (1 << 31) - 1, 0                 # multiplier just under 1: 255 -> clip at 127
+    hd["ls_lo"], hd["ls_hi"] = 2, 9
+    ly = hd["layer"]
+    st = S.Stream(82, "head")
+    ly["w"][:] = st.integers(-127, 128, ly["w"].size).astype(np.int8).reshape(ly["w"].shape)
+    ly["bias"][:] = [37, -1200, 2500, -90000]                  # ls biases on both sides of the clip
+    ly["m0"][:] = st.integers(1 << 30, 1 << 31, 4).astype(np.int32)
+    ly["s"][:] = [3, 5, 4, 2]
+    x = np.array([[[[255, 60], [7, 200]]]], dtype=np.uint8)    # squeeze order: 255, 60, 7, 200
+    z, p = O.forward(O.Packed(model), x)
+    keep = [255, 60]                                           # identity permutation, zero translation
+    a = [_clip(_rq_exact(v, hd["in_m0"], hd["in_s"]), -128, 127) for v in keep]
+    assert a == [127, 60]
+    out = []
+    for co in range(4):
+        acc = sum(int(ly["w"][co, 1, 1, ci]) * a[ci] for ci in range(2)) + int(ly["bias"][co])
+        out.append(_rq_exact(acc, int(ly["m0"][co]), int(ly["s"][co])))
+    want_mu = out[:2]
+    want_ls = [_clip(v, 2, 9) for v in out[2:]]
+    assert out[2] > 9 and out[3] < 2                           # both sides of the clip are exercised
+    assert p.shape == (1, 2, 2)
+    assert p[0, 0].tolist() == want_mu
+    assert p[0, 1].tolist() == want_ls
+    assert z[0].tolist() == [7, 200, 255, 60]                  # factored-out half first, kept half last
+    _, _, p2, _ = O.inverse(O.Packed(model), z)
+    np.testing.assert_array_equal(p2, p)
+
+
+def test_prior_layout_across_levels_with_constant_heads():
+    """Zero weights everywhere and constant head biases: every mu / log-scale index is rq(bias) of
+    its channel, so the prior array must be [mu of level 0 | mu of level 1] then [ls of level 0 | ls
+    of level 1], each block channel-major over the level's pixels."""
+    model = _zero_model(S.make_model(83, 1, 4, 4, [True, True], 1, 3, prune=None, prior=True))
+    want = [[], []]
+    for li, lv in enumerate(model["levels"]):
+        hd = lv["prior"]
+        ly = hd["layer"]
+        ly["w"][:] = 0
+        cb, px = ly["c_out"] // 2, lv["h"] * lv["w"]
+        ly["bias"][:] = [1000 * (li + 1) + 97 * c for c in range(cb)] + [40 * (li + 1) + 55 * c for c in range(cb)]
+        ly["s"][:] = 3
+        hd["ls_lo"], hd["ls_hi"] = 0, 63
+        vals = [_rq_exact(int(b), int(m), 3) for b, m in zip(ly["bias"], ly["m0"])]
+        for c in range(cb):
+            want[0] += [vals[c]] * px
+            want[1] += [_clip(vals[cb + c], 0, 63)] * px
+    x = S.smooth_field_images(84, 3, 4, 4, 1.0)[:, :1]
+    _, p = O.forward(O.Packed(model), x)
+    d, d_fact, _ = S.latent_sizes(model)
+    assert p.shape == (3, 2, d_fact) and d_fact == len(want[0]) == 12
+    for b in range(3):
+        assert p[b, 0].tolist() == want[0]
+        assert p[b, 1].tolist() == want[1]
+    assert len(set(want[0])) == 6 and len(set(want[1])) > 2    # the blocks are distinguishable

@@ -4,12 +4,14 @@ A plug-in living inside a host process that owns the device memory pool, or a se
 batch larger than the max_batch its model was created for at a moment when allocating is off
 limits, cannot use the workspace that iodf_create obtained with cudaMalloc. This entry point keeps
 the data passed between the level kernels in a fixed array inside the library image instead. The
-test calls it through the C ABI twice in a row and requires the same bits as iodf_forward; it runs
-last so that a run that stops at the first failure has already covered everything else."""
+test calls it through the C ABI twice in a row and requires the same bits as iodf_forward and as
+the CPU oracle; it runs last so that a run that stops at the first failure has already covered
+everything else."""
 import numpy as np
 import pytest
 
 import iodf_synth as S
+import oracle as O
 
 pytestmark = pytest.mark.gpu
 
@@ -25,7 +27,8 @@ def test_static_scratch_encode_matches_iodf_forward_twice():
     assert 0 < per_image * 24 <= G.IODF_STATIC_SCRATCH_BYTES
 
     for call, seed in enumerate((1, 2)):    # two calls in a row; the array keeps the first call's data
-        x = torch.from_numpy(S.smooth_field_images(seed, 24 - 5 * call, 32, 32, 2.0)).cuda()
+        x_host = S.smooth_field_images(seed, 24 - 5 * call, 32, 32, 2.0)
+        x = torch.from_numpy(x_host).cuda()
         B = x.shape[0]
         z_ref, p_ref = G.iodf_forward(big, x)
         G.iodf_check(big)
@@ -35,6 +38,9 @@ def test_static_scratch_encode_matches_iodf_forward_twice():
         G.iodf_check(small)
         assert torch.equal(z, z_ref), "call %d: latents differ" % call
         assert torch.equal(p, p_ref), "call %d: prior parameters differ" % call
+        z_cpu, p_cpu = O.forward(O.Packed(model), x_host)      # and the expected bits themselves
+        np.testing.assert_array_equal(z.cpu().numpy(), z_cpu)
+        np.testing.assert_array_equal(p.cpu().numpy(), p_cpu)
 
     # beyond the fixed array: a clear error, nothing launched
     too_many = G.IODF_STATIC_SCRATCH_BYTES // per_image + 1
@@ -43,4 +49,4 @@ def test_static_scratch_encode_matches_iodf_forward_twice():
     with pytest.raises(G.IodfError) as e:
         G.iodf_forward_static(small, x, z, None)
     assert e.value.status == -8
-    assert "fixed scratch" in str(e.value)
+    assert "fixed capacity" in str(e.value)
