@@ -259,7 +259,7 @@ def _stream(stream):
     if stream is None:
         import torch
         return C.c_void_p(torch.cuda.current_stream().cuda_stream)
-    return C.c_void_p(int(stream))
+    return C.c_void_p(int(getattr(stream, "cuda_stream", stream)))    # a torch stream or a raw handle
 
 
 def _ptr(t):
