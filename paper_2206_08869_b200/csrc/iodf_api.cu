@@ -15,6 +15,7 @@
 #include "rans_kernel.h"
 #include "res_level.h"
 #include "level_kernel.h"
+#include "level_pipe.h"
 #include "selftest.h"
 
 using namespace iodf;
@@ -322,14 +323,33 @@ uint32_t pow2_cols(uint32_t need) {
   return c;
 }
 
+// Levels of at least this many tiles per CTA run in the kernel that splits a tile's work by role
+// (level_pipe.cu) when they are eligible for it. Measured on the ImageNet64-shaped flow: 5 % faster
+// than the general kernel at eight tiles per image, 5 % slower at two (nothing follows the one
+// pair of tiles that the role split could overlap with).
+#ifndef IODF_PIPE_MIN_TILES
+#define IODF_PIPE_MIN_TILES 4
+#endif
+constexpr int kPipeMinTiles = IODF_PIPE_MIN_TILES;
+
+// What that kernel needs to know about a level.
+struct PipeDims {
+  bool eligible = false;           // every coupling in the folded flavour with the 0..127 clip
+  uint32_t a1_bytes = 16;          // im2col operand of a tile (couplings and prior head)
+  uint32_t n_hidden = 0;           // widest accumulator of the first two GEMMs (and of the prior head)
+  uint32_t n_taps = 0;             // accumulator of the third GEMM: nine taps x padded C/2
+};
+
 // Choose images per CTA, tiles in flight and the shared-memory layout. Returns false if nothing fits.
+//   pipe:   two tile slots, every weight matrix resident, the work of a tile split by role
+//           (level_pipe.cu; needs an eligible level of several tiles per CTA)
 //   mode 0: two tile slots, every weight matrix resident      (needs all N <= 256 and >= 2 tiles)
 //   mode 1: one tile slot, every weight matrix resident
 //   mode 2: one tile slot, W1 and W3 share a slot and are re-fetched per tile
 //   mode 3: one tile slot, weights streamed per tile in 32-byte K-slices through a small ring
 //           (the only mode for hidden widths above 256: a 512 x 512 matrix alone is 256 KB)
 bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32_t wmax[3], uint32_t n_max,
-               uint32_t limit, uint32_t max_batch, int num_sms) {
+               uint32_t limit, uint32_t max_batch, int num_sms, const PipeDims& pd) {
   int group = P.px >= kTileM ? 1 : kTileM / P.px;
   group = std::max(1, std::min<int>(group, (int)max_batch));
   // A level's time is set by the serial chain of its couplings inside one CTA, not by how many
@@ -338,9 +358,14 @@ bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32
   while (group > 1 && ((int)max_batch + group - 1) / group < num_sms) group /= 2;
   for (; group >= 1; group = (group > 1 ? group / 2 : 0)) {
     const int tiles = (group * P.px + kTileM - 1) / kTileM;
-    for (int mode = 0; mode < 4; ++mode) {
+    // the role-split kernel first with im2col buffers of its own (mode -2), then sharing the slot's buffer (-1)
+    for (int mode = -2; mode < 4; ++mode) {
+      const bool pipe = mode < 0;
+      // per-tap partials in columns of their own when two slots of both kinds fit the 512 columns
+      const bool r3_separate = 2u * pd.n_hidden + 2u * pd.n_taps <= 512u;
+      if (pipe && (!pd.eligible || tiles < kPipeMinTiles || std::max(pd.n_hidden, pd.n_taps) > (uint32_t)kSlotCols)) continue;
       if (mode == 0 && (tiles < 2 || n_max > (uint32_t)kSlotCols)) continue;
-      if (mode < 3 && n_max > 2u * kSlotCols) continue;
+      if (mode >= 0 && mode < 3 && n_max > 2u * kSlotCols) continue;
       if (mode == 3 && n_max <= (uint32_t)kSlotCols) continue;   // resident weights are faster when they fit
       const uint32_t pg = up((uint32_t)group * P.px, 32);
       uint32_t off = 0;
@@ -351,7 +376,9 @@ bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32
       P.s_rowinfo = take((uint32_t)tiles * kTileM * 4);
       P.s_gran = take((uint32_t)P.n_gran * 8);
       P.s_a[0] = take(a_bytes);
-      P.s_a[1] = mode == 0 ? take(a_bytes) : P.s_a[0];
+      P.s_a[1] = (pipe || mode == 0) ? take(a_bytes) : P.s_a[0];
+      P.s_a1[0] = mode == -2 ? take(pd.a1_bytes) : P.s_a[0];
+      P.s_a1[1] = mode == -2 ? take(pd.a1_bytes) : P.s_a[1];
       P.s_meta[0] = take(meta_bytes);
       P.s_meta[1] = take(meta_bytes);
       P.ring_slot_bytes = up(32u * n_max, kAlign);
@@ -364,10 +391,14 @@ bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32
         P.s_w[2] = mode == 2 ? P.s_w[0] : take(wmax[2]);
       }
       P.s_total = off;
+      P.pipe = pipe ? 1 : 0;
+      P.r_col[0] = r3_separate ? (int)pd.n_hidden : kSlotCols;
+      P.r_col[1] = r3_separate ? 2 * (int)pd.n_hidden : 0;
+      P.r_col[2] = r3_separate ? (int)pd.n_taps : kSlotCols;
       P.w13_alias = mode == 2;
       P.streamed = mode == 3;
       P.nslots = mode == 0 ? 2 : 1;
-      P.tmem_cols = (int)(mode == 0 ? 2 * kSlotCols : pow2_cols(n_max));
+      P.tmem_cols = (int)(pipe ? 512 : (mode == 0 ? 2 * kSlotCols : pow2_cols(n_max)));
       P.group = group;
       P.pg = (int)pg;
       P.tiles = tiles;
@@ -698,6 +729,8 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
     }
     uint32_t a_bytes = 16, meta = 16, wmax[3] = {16, 16, 16};
     uint32_t n_max = 32;
+    PipeDims pd;
+    pd.eligible = lv.n_couplings > 0;
     std::vector<PackedBlock> blocks;
     for (uint32_t ki = 0; ki < lv.n_couplings; ++ki) {
       const iodf_coupling_desc& cp = lv.couplings[ki];
@@ -711,6 +744,11 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
       blocks.push_back(pack_coupling(cp, B, ca, cb, pi.data(), pi.data() + ca, a1, a2r, &d));
       a_bytes = std::max<uint32_t>(a_bytes, kTileM * std::max(d.kd1, std::max(d.kd2, d.kd3)));
       n_max = std::max<uint32_t>(n_max, std::max(d.n1, std::max(d.n2, d.n3)));
+      const CouplingMeta* cm = reinterpret_cast<const CouplingMeta*>(blocks.back().meta.data());
+      if (cm->mode1 != 3 || cm->mode2 != 3 || a1.lo != 0 || a1.hi != 127 || a2r.lo != 0 || a2r.hi != 127) pd.eligible = false;
+      pd.n_hidden = std::max<uint32_t>(pd.n_hidden, (uint32_t)std::max(d.n1, d.n2));
+      pd.a1_bytes = std::max<uint32_t>(pd.a1_bytes, (uint32_t)kTileM * d.kd1);
+      pd.n_taps = std::max<uint32_t>(pd.n_taps, (uint32_t)d.n3);
     }
     for (int k = 0; k < (int)c; ++k) P.col_out[k] = pi[k];
     PackedBlock prior_block;
@@ -719,6 +757,8 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
       prior_block = pack_prior(lv, B, ca, cb, &n, &kd);
       a_bytes = std::max<uint32_t>(a_bytes, kTileM * kd);
       n_max = std::max<uint32_t>(n_max, n);
+      pd.n_hidden = std::max<uint32_t>(pd.n_hidden, (uint32_t)n);
+      pd.a1_bytes = std::max<uint32_t>(pd.a1_bytes, (uint32_t)kTileM * kd);
     }
     if (n_max > 512) return IODF_EUNSUPPORTED;
     {   // im2col granule table of the level's first convs (couplings and prior head share it)
@@ -747,7 +787,7 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
       wmax[0] = std::max(wmax[0], P.prior.w_bytes[0]);
     }
     if (hl.blob.empty()) hl.blob.resize(kAlign, 0);
-    if (!plan_smem(P, a_bytes, meta, wmax, n_max, (uint32_t)smem_limit, desc->max_batch, num_sms))
+    if (!plan_smem(P, a_bytes, meta, wmax, n_max, (uint32_t)smem_limit, desc->max_batch, num_sms, pd))
       return IODF_EUNSUPPORTED;
     // the index maps divide numbers below group * c * px by at most c * px with a 32-bit magic multiplier
     if ((uint64_t)P.group * c * h * w * ((uint64_t)c * h * w) >= (1ull << 32)) return IODF_EUNSUPPORTED;
@@ -761,6 +801,7 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
   (void)max_smem;
   CU(m, configure_level_kernels((uint32_t)smem_limit));
   CU(m, configure_res_kernels((uint32_t)smem_limit));
+  CU(m, configure_pipe_kernels((uint32_t)smem_limit));
   const size_t L = desc->n_levels;
   m->d_plan.assign(L, nullptr); m->d_blob.assign(L, nullptr); m->d_keep.assign(L, nullptr);
   for (size_t li = 0; li < L; ++li) {
@@ -795,6 +836,14 @@ void set_patch_grid(LevelArgs& a, const PatchGrid& g) {
   a.mul_patches_x = g.patches_x > 1 ? (uint32_t)(((1ull << 32) + g.patches_x - 1) / g.patches_x) : 0u;
 }
 
+// The kernel that runs a level: residual couplings, the stage pipeline, or the general kernel.
+cudaError_t launch_any_level(const LevelPlan& P, const LevelArgs& a, bool inverse, int B, cudaStream_t st) {
+  const int grid = (B + P.group - 1) / P.group;
+  if (P.residual) return launch_res_level(a, inverse, grid, P.s_total, st);
+  if (P.pipe) return launch_level_pipe(a, inverse, grid, P.s_total, st);
+  return launch_level(a, inverse, grid, P.s_total, st);
+}
+
 int run_forward(iodf_model* m, const uint8_t* x, int B, int32_t* z, int32_t* prior, cudaStream_t st,
                 bool timed = false, PatchGrid grid = PatchGrid()) {
   const size_t L = m->levels.size();
@@ -813,8 +862,7 @@ int run_forward(iodf_model* m, const uint8_t* x, int B, int32_t* z, int32_t* pri
     a.status = m->d_status;
     a.batch = B;
     if (li == 0) set_patch_grid(a, grid);
-    CU(m, P.residual ? launch_res_level(a, false, (B + P.group - 1) / P.group, P.s_total, st)
-                      : launch_level(a, false, (B + P.group - 1) / P.group, P.s_total, st));
+    CU(m, launch_any_level(P, a, false, B, st));
     if (timed) CU(m, cudaEventRecord(m->ev[li + 1], st));
   }
   return IODF_OK;
@@ -838,8 +886,7 @@ int launch_inverse_level(iodf_model* m, int li, int phase, const int32_t* z, int
   a.batch = B;
   a.phase = phase;
   if (li == 0) set_patch_grid(a, grid);
-  CU(m, P.residual ? launch_res_level(a, true, (B + P.group - 1) / P.group, P.s_total, st)
-                    : launch_level(a, true, (B + P.group - 1) / P.group, P.s_total, st));
+  CU(m, launch_any_level(P, a, true, B, st));
   return IODF_OK;
 }
 
@@ -961,8 +1008,7 @@ int iodf_forward_static(iodf_model* m, const uint8_t* x_u8, int B, int32_t* z, i
     a.oor = nullptr;
     a.status = m->d_status;
     a.batch = B;
-    CU(m, P.residual ? launch_res_level(a, false, (B + P.group - 1) / P.group, P.s_total, st)
-                      : launch_level(a, false, (B + P.group - 1) / P.group, P.s_total, st));
+    CU(m, launch_any_level(P, a, false, B, st));
   }
   return IODF_OK;
 }

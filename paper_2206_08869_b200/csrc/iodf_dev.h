@@ -116,8 +116,15 @@ struct LevelPlan {
   int32_t streamed;              // 1: weights are streamed per tile in 32-byte K-slices through a ring of
                                  //    kRingDepth slots at s_w[0] (hidden widths above 256, one tile in flight)
   uint32_t ring_slot_bytes;
+  int32_t pipe;                  // 1: the level runs in the kernel that splits a tile's work by role (several
+                                 //    tiles per CTA, two tile slots, resident weights, folded requantisation with
+                                 //    the 0..127 clip)
+  int32_t r_col[3];              // that kernel's tensor-memory columns: slot s has its hidden-layer accumulators
+                                 //    at s * r_col[0] and its per-tap partials at r_col[1] + s * r_col[2]
+                                 //    (r_col[1] = 0: the partials share the slot's main columns)
   // shared-memory byte offsets
   uint32_t s_v, s_xa, s_acc, s_rowinfo, s_gran, s_a[2], s_meta[2], s_w[3], s_total;
+  uint32_t s_a1[2];              // role-split kernel: the slots' im2col operands (= s_a[] when they share the buffer)
   // magic multipliers for the index maps: n / d = umulhi(n, ceil(2^32 / d)) for n * d < 2^32 (0: d = 1)
   uint32_t mul_per_img, mul_4px, mul_w2, mul_px, mul_w;
   uint32_t recip_gpa, recip_gpb; // floor(g / (cpad/8)) = (g * recip_gpa) >> 16 for g < 4096; same for cbp/8

@@ -277,3 +277,18 @@ def test_config4_batch_sweep_stress_width_512(G, batch):
             z64, _ = G.iodf_forward(m, _t(x[b0:b0 + 64]))
             np.testing.assert_array_equal(z64.cpu().numpy(), z[b0:b0 + 64])
         G.iodf_check(m)
+
+
+@pytest.mark.parametrize("hw,hidden,prune,batch", [
+    (64, 40, (0.4, 0.7), 3),     # 1024-pixel first level: eight tiles, per-tap partials in columns of their own
+    (48, 24, None, 2),           # 576 pixels: five tiles, a ragged last one, image rows that straddle warps
+    (64, 200, None, 2),          # wide hidden layers: the per-tap partials share the slot's columns
+])
+def test_levels_of_many_tiles_in_the_role_split_kernel(G, hw, hidden, prune, batch):
+    """First levels of four tiles and more run in the kernel that gives the im2col / shifted sum,
+    the requantisation and the MMA issue to different warps; the deeper levels of the same models
+    run in the general kernel. Encode, prior parameters, decode and the out-of-range count against
+    the oracle, for every image."""
+    model = S.make_model(0xB100 + hw + hidden, 3, hw, hw, [True, True], 3, hidden, prune=prune)
+    x = S.smooth_field_images(0xB200 + hw, batch, hw, hw, 3.0)
+    _check_both_ways(G, model, x)
