@@ -260,6 +260,9 @@ CONFIGS = {
     # each conv3x3 -> 8 gated residual blocks -> conv3x3 on 128 hidden channels, about half pruned
     "R32": dict(seed=0x10DF0032, batch=64, hw=32, sigma=2.0, splits=[True] * 3, n_couplings=8,
                 hidden=128, prune=(0.40, 0.70), prior=True, perm="random", n_blocks=8),
+    # the same network on the ImageNet64 geometry (Sec. 5, App. B.1): 4 levels, the first of 32 x 32 pixels
+    "R64": dict(seed=0x10DF0064, batch=32, hw=64, sigma=4.0, splits=[True] * 4, n_couplings=8,
+                hidden=128, prune=(0.40, 0.70), prior=True, perm="random", n_blocks=8),
 }
 
 

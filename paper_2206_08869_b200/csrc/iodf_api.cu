@@ -421,9 +421,18 @@ int cuda_fail(iodf_model* m, cudaError_t e) {
     if (e__ != cudaSuccess) return cuda_fail(m, e__); \
   } while (0)
 
+// Row bands of an image at a residual level: 1 while the whole image fits one CTA, otherwise the
+// smallest power of two that brings a band down to kResMaxPixels pixels (bands of at least two rows;
+// 0 if there is none up to kResMaxBands).
+int residual_bands(uint32_t h, uint32_t w) {
+  for (uint32_t nb = 1; nb <= (uint32_t)kResMaxBands; nb *= 2)
+    if (h % nb == 0 && (nb == 1 || h / nb >= 2) && (h / nb) * w <= (uint32_t)kResMaxPixels) return (int)nb;
+  return 0;
+}
+
 // A coupling with residual blocks (layers already checked one by one): shapes, ranges and what this
 // build runs.
-int check_residual(const iodf_coupling_desc& cp, const Blobs& B, uint32_t ca, uint32_t cb, uint32_t px) {
+int check_residual(const iodf_coupling_desc& cp, const Blobs& B, uint32_t ca, uint32_t cb, uint32_t h, uint32_t w) {
   if (!cp.blocks || cp.n_layers != 2 + 2 * cp.n_blocks) return IODF_EINVAL;
   const iodf_layer_desc& cin = cp.layers[0];
   const iodf_layer_desc& cout = cp.layers[cp.n_layers - 1];
@@ -444,7 +453,7 @@ int check_residual(const iodf_coupling_desc& cp, const Blobs& B, uint32_t ca, ui
     }
   }
   // what the residual kernel runs
-  if (px > (uint32_t)kResMaxPixels) return IODF_EUNSUPPORTED;
+  if (residual_bands(h, w) == 0) return IODF_EUNSUPPORTED;
   for (uint32_t q = 0; q < cp.n_layers; ++q) {
     const iodf_layer_desc& L = cp.layers[q];
     if (L.k != 3 || L.c_out > (uint32_t)kResMaxWidth || L.c_in > (uint32_t)kResMaxWidth) return IODF_EUNSUPPORTED;
@@ -550,18 +559,24 @@ int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P,
   }
   // shared memory: flow variable, the three activation buffers in the padded chunk-major layout
   // (cleared together at kernel start), position table, conv tables, weight ring
-  const uint32_t pg = up((uint32_t)px, 32);
+  // one CTA per image, or per band of hb rows (a cluster of `bands` CTAs per image)
+  const int bands = residual_bands((uint32_t)P.h, (uint32_t)P.w);
+  if (bands == 0) return IODF_EUNSUPPORTED;
+  const int hb = P.h / bands;
+  (void)px;
+  const uint32_t pg = up((uint32_t)(hb * P.w), 32);
   const int w2 = P.w + 2, guard = w2 + 1;
-  const int ntiles = (int)(up((uint32_t)((P.h + 2) * w2), kTileM) / kTileM);
+  const int ntiles = (int)(up((uint32_t)((hb + 2) * w2), kTileM) / kTileM);
   const int rows = guard + ntiles * kTileM + w2 + 1;
   H.w2 = w2; H.guard = guard; H.rows = rows; H.ntiles = ntiles;
+  H.bands = bands; H.hb = hb;
   uint32_t off = 0;
   auto take = [&](uint32_t bytes) { uint32_t o = off; off = up(off + bytes, kAlign); return o; };
   H.s_v = take((uint32_t)P.c * pg * 4);
   H.s_xa = take((uint32_t)(H.xa_pitch / 16) * rows * 16);
   H.s_x = take((uint32_t)(H.x_pitch / 16) * rows * 16);
   H.s_mid = take((uint32_t)(H.mid_pitch / 16) * rows * 16);
-  H.s_rowinfo = take((uint32_t)ntiles * kTileM * 4);
+  H.s_rowinfo = take((uint32_t)ntiles * kTileM * 8);     // pixel and edge-row tables
   H.s_tab = take((uint32_t)kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t)) + 256);   // + the shortcut table
   // as deep a weight ring as fits (at least two slots)
   H.w_slot_bytes = up((uint32_t)nmax * kmax, kAlign);
@@ -576,6 +591,7 @@ int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P,
   std::memcpy(blob.data() + H.coupling_off, cps.data(), sizeof(ResCouplingRec) * cps.size());
   std::memcpy(blob.data() + H.conv_off, convs.data(), sizeof(ResConv) * convs.size());
   P.residual = 1;
+  P.res_bands = bands;
   P.group = 1; P.pg = (int)pg; P.tiles = ntiles; P.rep = 1; P.nslots = 1;
   P.s_total = H.s_total;
   return IODF_OK;
@@ -627,7 +643,7 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
         cin = cp.layers[q].c_out;
       }
       if (cp.n_blocks > 0) {
-        int rc = check_residual(cp, B, ca, cb, px);
+        int rc = check_residual(cp, B, ca, cb, h, w);
         if (rc) return rc;
         if (ki > 0 && lv.couplings[0].n_blocks == 0) return IODF_EUNSUPPORTED;    // one kind per level
         for (uint32_t q = 0; q < cp.n_layers; ++q)
@@ -839,7 +855,7 @@ void set_patch_grid(LevelArgs& a, const PatchGrid& g) {
 // The kernel that runs a level: residual couplings, the stage pipeline, or the general kernel.
 cudaError_t launch_any_level(const LevelPlan& P, const LevelArgs& a, bool inverse, int B, cudaStream_t st) {
   const int grid = (B + P.group - 1) / P.group;
-  if (P.residual) return launch_res_level(a, inverse, grid, P.s_total, st);
+  if (P.residual) return launch_res_level(a, inverse, B, P.res_bands, P.s_total, st);
   if (P.pipe) return launch_level_pipe(a, inverse, grid, P.s_total, st);
   return launch_level(a, inverse, grid, P.s_total, st);
 }

@@ -110,6 +110,7 @@ struct LevelPlan {
   int32_t residual;              // 1: the level's couplings are residual-block networks (its own kernel; the
                                  //    level blob then starts with a ResHead and the fields on tiles, slots and
                                  //    the shared-memory layout below are unused)
+  int32_t res_bands;             // residual levels: row bands per image (CTAs of a cluster), 1 = one CTA per image
   int32_t nslots;                // tiles in flight per CTA: 1 or 2
   int32_t tmem_cols;
   int32_t w13_alias;             // 1: W1 and W3 share a slot and are re-fetched per tile

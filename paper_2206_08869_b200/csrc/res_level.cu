@@ -1,6 +1,7 @@
 // One flow level whose couplings use the paper's residual-block network (Eq. 3, Sec. 4.1; scatter
 // add, Sec. 4.5; App. B.1: conv 3x3 -> L blocks of two 3x3 convs -> conv 3x3, all on `hidden`
-// channels), one CTA per image, images of at most 256 pixels at this level.
+// channels), one CTA per image of at most 256 pixels at this level; larger images (up to 2048 pixels)
+// are cut into row bands, one CTA of a thread-block cluster each (see "Row bands" below).
 //
 // Every conv here is a 3x3 conv over hidden activations, so a pixel needs its neighbours' hidden
 // values: the activations of the whole image stay in shared memory (xa: the requantised network
@@ -31,8 +32,15 @@
 // plain 16-channel-wide add. The extra rows cost tensor time that is idle; byte-wise scattered
 // updates cost shared-memory bank conflicts that were not.
 //
-// This is a first version of the path: convs run one after another, a conv's epilogue does not
-// overlap the next conv's MMAs.
+// Row bands. A 3x3 conv needs the rows above and below a band. Each CTA of the cluster keeps its band
+// in the same padded layout with two more rows: the band's own rows in the middle, the neighbouring
+// bands' edge rows (or the zero padding at the image's border) above and below. Whatever writes
+// activations (network input, every conv's epilogue) also writes a band's first and last row into
+// the neighbours' edge rows through distributed shared memory, and the barrier that separates a
+// conv from the next one is then a cluster barrier. The index lists of the level's load and store
+// take the band's offset; nothing else changes.
+//
+// Convs run one after another: a conv's epilogue does not overlap the next conv's MMAs.
 #include "res_level.h"
 #include "ptx.cuh"
 
@@ -76,8 +84,33 @@ __device__ __forceinline__ int32_t rq_const(int32_t acc, const OutRq o) {     //
 
 __device__ __forceinline__ int clampi(int v, int lo, int hi) { return min(max(v, lo), hi); }
 
+// ---- thread-block cluster: rank, barrier, stores into a peer CTA's shared memory -------------------
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// every thread of every CTA of the cluster; orders shared-memory writes (local and remote) before it
+// with reads after it
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t peer_addr(const void* p, uint32_t rank) {
+  uint32_t a;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(ptx::smem_u32(p)), "r"(rank));
+  return a;
+}
+__device__ __forceinline__ void peer_store16(uint32_t addr, const uint4 v) {
+  asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void peer_store1(uint32_t addr, uint32_t byte) {
+  asm volatile("st.shared::cluster.u8 [%0], %1;" ::"r"(addr), "r"(byte) : "memory");
+}
+
 struct Geo {
-  int px, h, w, pg;
+  int px, h, w, pg;        // the CTA's band: pixels, rows, width, pixel slots
   uint32_t mul_w;
 };
 
@@ -96,8 +129,37 @@ struct Run {
   uint32_t nconv;           // convs run so far (parity of conv_done)
   uint32_t prefetched;      // weight slices of the coming conv that were requested already, loading lane only
   int32_t* v;
-  const int32_t* pixel_of;  // pixel index of a padded position, -1 at padding
+  const int32_t* pixel_of;  // pixel index (within the band) of a padded position, -1 at padding
+  const int32_t* halo_of;   // 0, or where a position is mirrored in a neighbouring band: (its padded position there << 1) | (1: the band below)
+  int bands, band;          // row bands of the image (CTAs of the cluster) and this CTA's
+  int px_full;              // pixels of the whole image at this level (strides of the global layouts)
+  int q0;                   // the band's first pixel
 };
+
+// End of a step that wrote activations: they must be visible to the tensor core's reads (this CTA's
+// and, for edge rows, the neighbours') before the next conv is issued.
+__device__ __forceinline__ void step_barrier(const Run& r) {
+  ptx::fence_async_smem();
+  ptx::tc_fence_before();
+  if (r.bands > 1) {
+    cluster_barrier();
+    ptx::fence_async_smem();     // what the neighbours wrote here, towards the async proxy
+  } else {
+    __syncthreads();
+  }
+}
+// the same 16 bytes / byte in the neighbouring band's edge row, if the position is one of this band's edge rows
+__device__ __forceinline__ void mirror16(const Run& r, uint8_t* buf, int c, int rr, const uint4 v) {
+  const int hrec = r.halo_of[rr];
+  if (hrec) peer_store16(peer_addr(buf + ((size_t)(c >> 4) * r.H->rows + r.H->guard + (hrec >> 1)) * 16 + (c & 15),
+                                   (uint32_t)(r.band + ((hrec & 1) ? 1 : -1))), v);
+}
+__device__ __forceinline__ void mirror1(const Run& r, uint8_t* buf, int c, int rr, uint32_t byte) {
+  const int hrec = r.halo_of[rr];
+  if (hrec) peer_store1(peer_addr(buf + ((size_t)(c >> 4) * r.H->rows + r.H->guard + (hrec >> 1)) * 16 + (c & 15),
+                                  (uint32_t)(r.band + ((hrec & 1) ? 1 : -1))), byte);
+}
+
 
 __device__ __forceinline__ uint8_t* buf_of(const Run& r, int which) {
   return r.smem + (which == 0 ? r.H->s_xa : (which == 1 ? r.H->s_x : r.H->s_mid));
@@ -292,7 +354,9 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
           }
           wd[i] = word;
         }
-        *reinterpret_cast<uint4*>(at(r, dst, ch * 16, rr)) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+        const uint4 val = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+        *reinterpret_cast<uint4*>(at(r, dst, ch * 16, rr)) = val;
+        if (r.bands > 1) mirror16(r, dst, ch * 16, rr, val);
       } else if (c.kind == kResBranch) {
         // The conv's outputs sit at their channels of X already (the scatter add was done on the
         // weights, when the level was packed; a channel without a filter requantises 0 to 0), so the
@@ -315,7 +379,9 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
           }
           wd[i] = word;
         }
-        *xp = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+        const uint4 val = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+        *xp = val;
+        if (r.bands > 1) mirror16(r, dst, ch * 16, rr, val);
       } else {
 #pragma unroll 4
         for (int i = 0; i < 16; ++i) {
@@ -327,16 +393,14 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
             *vv = io.subtract ? (*vv - (uint32_t)y) : (*vv + (uint32_t)y);
           } else {   // kResPrior: first half mu, second half the clipped log-scale index
             const int half = c.n >> 1;
-            if (col < half) io.mu[(size_t)col * r.g.px + p] = y;
-            else io.ls[(size_t)(col - half) * r.g.px + p] = clampi(y, io.ls_lo, io.ls_hi);
+            if (col < half) io.mu[(size_t)col * r.px_full + p] = y;
+            else io.ls[(size_t)(col - half) * r.px_full + p] = clampi(y, io.ls_lo, io.ls_hi);
           }
         }
       }
     }
   }
-  ptx::fence_async_smem();       // the next conv's MMAs read what was stored here
-  ptx::tc_fence_before();
-  __syncthreads();
+  step_barrier(r);               // the next conv's MMAs read what was stored here
 }
 
 // network input: logical channels cols[0 .. n) of the flow variable, requantised to int8, at the
@@ -347,10 +411,11 @@ __device__ void requant_input(Run& r, const int32_t* cols, int n, int32_t m0, in
     const int c = it / r.g.px, p = it - c * r.g.px;
     const int i = rdiv(p, r.g.mul_w), j = p - i * r.g.w;
     const int rr = (i + 1) * r.H->w2 + (j + 1);
-    *at(r, xa, c, rr) = (uint8_t)(int8_t)clampi(rq64(r.v[cols[c] * r.g.pg + p], m0, s), -128, 127);
+    const uint32_t byte = (uint32_t)(uint8_t)(int8_t)clampi(rq64(r.v[cols[c] * r.g.pg + p], m0, s), -128, 127);
+    *at(r, xa, c, rr) = (uint8_t)byte;
+    if (r.bands > 1) mirror1(r, xa, c, rr, byte);
   }
-  ptx::fence_async_smem();
-  __syncthreads();
+  step_barrier(r);
 }
 
 template <bool kInv>
@@ -376,9 +441,17 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
   __syncthreads();
   ptx::tc_fence_after();
 
+  // one CTA per image, or per band of rows of an image (the CTAs of a cluster)
+  const int bands = H->bands, hb = H->hb;
+  const int band = bands > 1 ? (int)cluster_rank() : 0;
+  const int b = blockIdx.x / bands;               // image
+  const int w = P.w, pg = P.pg, c = P.c;
+  const int pxb = hb * w;                         // pixels of the band
+  const int q0 = band * pxb;                      // the band's first pixel in the image
+
   Run r;
   r.smem = smem; r.ctl = &ctl; r.status = a.status; r.blob = a.blob; r.H = H;
-  r.g.px = P.px; r.g.h = P.h; r.g.w = P.w; r.g.pg = P.pg; r.g.mul_w = P.mul_w;
+  r.g.px = pxb; r.g.h = hb; r.g.w = w; r.g.pg = pg; r.g.mul_w = P.mul_w;
   r.tid = tid; r.warp = warp; r.lane = lane;
   r.ntiles = H->ntiles;
   r.tmem = ctl.tmem_base;
@@ -388,47 +461,59 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
   r.prefetched = 0;
   r.v = reinterpret_cast<int32_t*>(smem + H->s_v);
   int32_t* pixel_of = reinterpret_cast<int32_t*>(smem + H->s_rowinfo);
+  int32_t* halo_of = pixel_of + r.ntiles * kTileM;
   r.pixel_of = pixel_of;
+  r.halo_of = halo_of;
+  r.bands = bands; r.band = band; r.px_full = P.px; r.q0 = q0;
 
-  const int c = P.c, px = P.px, pg = P.pg, w = P.w;
-  const int b = blockIdx.x;                       // one image per CTA
   const bool builder = warp < kResBuilderWarps;
-  const int per_img = builder ? c * px : 0;       // the issuing warp takes no part in the element loops
+  const int per_band = builder ? c * pxb : 0;     // the issuing warps take no part in the element loops
   int32_t* v = r.v;
   for (int rr = tid; rr < (builder ? r.ntiles * kTileM : 0); rr += kResThreads) {
-    const int i = rr / H->w2, j = rr - i * H->w2;          // position (i, j) of the (h+2) x (w+2) frame
-    pixel_of[rr] = (i >= 1 && i <= P.h && j >= 1 && j <= P.w) ? (i - 1) * P.w + (j - 1) : -1;
+    const int i = rr / H->w2, j = rr - i * H->w2;          // position (i, j) of the (hb+2) x (w+2) frame
+    const bool own = i >= 1 && i <= hb && j >= 1 && j <= w;
+    pixel_of[rr] = own ? (i - 1) * w + (j - 1) : -1;
+    // the band's first row is the row below the band above's last one, and the other way round
+    int hrec = 0;
+    if (own && i == 1 && band > 0) hrec = ((rr + hb * H->w2) << 1) | 0;
+    if (own && i == hb && band + 1 < bands) hrec = ((rr - hb * H->w2) << 1) | 1;
+    halo_of[rr] = hrec;
   }
   // activation buffers start at zero: padding channels and bytes beyond a conv's outputs stay zero
   // or meet zero weights
   for (uint32_t i = H->s_xa + tid * 16; builder && i < H->s_rowinfo; i += kResThreads * 16)
     *reinterpret_cast<uint4*>(smem + i) = make_uint4(0u, 0u, 0u, 0u);
 
+  // the level's input: pre-squeeze rows 2 * band * hb .. of [c/4][2h][2w] (encode), or the band's pixels
+  // of the kept channels and of z's block (decode)
+  const int px = P.px;
   if (!kInv) {
-    const int w2 = 2 * w;
-    for (int e = tid; e < per_img; e += kResThreads) {
-      const int ci = rdiv(e, P.mul_4px), r2 = e - ci * 4 * px;
-      const int y = rdiv(r2, P.mul_w2), x = r2 - y * w2;
-      size_t src = (size_t)b * per_img + e;
+    const int w2 = 2 * w, rows2 = 2 * hb;
+    for (int e = tid; e < per_band; e += kResThreads) {
+      const int ci = e / (rows2 * w2), r2 = e - ci * rows2 * w2;
+      const int y = r2 / w2, x = r2 - y * w2;
+      const int gy = 2 * band * hb + y;                    // row of the whole pre-squeeze image
+      size_t src = ((size_t)b * (c / 4) + ci) * (size_t)(4 * px) + (size_t)gy * w2 + x;
       if (P.is_first && a.img_w > 0) {
         const int by = rdiv(b, a.mul_patches_x), bx = b - by * a.patches_x;
-        src = ((size_t)ci * a.img_h + (size_t)(by * 2 * P.h + y)) * a.img_w + (size_t)(bx * w2 + x);
+        src = ((size_t)ci * a.img_h + (size_t)(by * 2 * P.h + gy)) * a.img_w + (size_t)(bx * w2 + x);
       }
       const int32_t val = P.is_first ? (int32_t) reinterpret_cast<const uint8_t*>(a.in)[src]
                                      : reinterpret_cast<const int32_t*>(a.in)[src];
       v[(ci * 4 + (y & 1) * 2 + (x & 1)) * pg + (y >> 1) * w + (x >> 1)] = val;
     }
   } else {
-    for (int e = tid; e < per_img; e += kResThreads) {
-      const int k = rdiv(e, P.mul_px), q = e - k * px;
+    for (int e = tid; e < per_band; e += kResThreads) {
+      const int k = e / pxb, q = e - k * pxb;
       if (a.phase == 1 && k >= P.keep_c) continue;
       const int32_t val =
-          (k < P.keep_c) ? reinterpret_cast<const int32_t*>(a.in)[(size_t)b * (size_t)a.in_stride + (size_t)k * px + q]
-                         : a.z[(size_t)b * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q];
+          (k < P.keep_c) ? reinterpret_cast<const int32_t*>(a.in)[(size_t)b * (size_t)a.in_stride + (size_t)k * px + q0 + q]
+                         : a.z[(size_t)b * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q0 + q];
       v[P.col_out[k] * pg + q] = val;
     }
   }
-  __syncthreads();
+  // nobody writes into a neighbour's edge rows before that neighbour has cleared its buffers
+  if (bands > 1) cluster_barrier(); else __syncthreads();
 
   const ResCouplingRec* cps = reinterpret_cast<const ResCouplingRec*>(a.blob + H->coupling_off);
   const ResConv* convs = reinterpret_cast<const ResConv*>(a.blob + H->conv_off);
@@ -442,7 +527,7 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
     if (prior) {
       const ResConv cv = convs[H->prior_conv];
       requant_input(r, P.col_out, P.ca, H->prior_in_m0, H->prior_in_s);
-      io.mu = a.prior + (size_t)b * 2u * P.d_fact + P.prior_off;
+      io.mu = a.prior + (size_t)b * 2u * P.d_fact + P.prior_off + q0;
       io.ls = io.mu + P.d_fact;
       io.ls_lo = H->ls_lo; io.ls_hi = H->ls_hi;
       conv_mma(r, cv, nullptr, nullptr);
@@ -464,24 +549,25 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
 
   if (!kInv) {
     int32_t* keep_out = reinterpret_cast<int32_t*>(a.out);
-    for (int e = tid; e < per_img; e += kResThreads) {
-      const int k = rdiv(e, P.mul_px), q = e - k * px;
+    for (int e = tid; e < per_band; e += kResThreads) {
+      const int k = e / pxb, q = e - k * pxb;
       const int32_t val = v[P.col_out[k] * pg + q];
-      if (k >= P.keep_c) a.z[(size_t)b * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q] = val;
-      else if (P.is_last) a.z[(size_t)b * P.d + P.z_final_off + (size_t)k * px + q] = val;
-      else keep_out[((size_t)b * P.keep_c + k) * (size_t)px + q] = val;
+      if (k >= P.keep_c) a.z[(size_t)b * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q0 + q] = val;
+      else if (P.is_last) a.z[(size_t)b * P.d + P.z_final_off + (size_t)k * px + q0 + q] = val;
+      else keep_out[((size_t)b * P.keep_c + k) * (size_t)px + q0 + q] = val;
     }
   } else if (a.phase != 1) {
-    const int w2 = 2 * w;
+    const int w2 = 2 * w, rows2 = 2 * hb;
     uint32_t bad = 0;
-    for (int e = tid; e < per_img; e += kResThreads) {
-      const int ci = rdiv(e, P.mul_4px), r2 = e - ci * 4 * px;
-      const int y = rdiv(r2, P.mul_w2), x = r2 - y * w2;
+    for (int e = tid; e < per_band; e += kResThreads) {
+      const int ci = e / (rows2 * w2), r2 = e - ci * rows2 * w2;
+      const int y = r2 / w2, x = r2 - y * w2;
+      const int gy = 2 * band * hb + y;
       const int32_t val = v[(ci * 4 + (y & 1) * 2 + (x & 1)) * pg + (y >> 1) * w + (x >> 1)];
-      size_t dst = (size_t)b * per_img + e;
+      size_t dst = ((size_t)b * (c / 4) + ci) * (size_t)(4 * px) + (size_t)gy * w2 + x;
       if (P.is_first && a.img_w > 0) {
         const int by = rdiv(b, a.mul_patches_x), bx = b - by * a.patches_x;
-        dst = ((size_t)ci * a.img_h + (size_t)(by * 2 * P.h + y)) * a.img_w + (size_t)(bx * w2 + x);
+        dst = ((size_t)ci * a.img_h + (size_t)(by * 2 * P.h + gy)) * a.img_w + (size_t)(bx * w2 + x);
       }
       if (P.is_first) {
         reinterpret_cast<uint8_t*>(a.out)[dst] = (uint8_t)((uint32_t)val & 0xFFu);
@@ -503,10 +589,23 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
 
 }  // namespace
 
-cudaError_t launch_res_level(const LevelArgs& args, bool inverse, int grid, uint32_t smem_bytes, cudaStream_t stream) {
-  if (inverse) res_level_kernel<true><<<grid, kResAllThreads, smem_bytes, stream>>>(args);
-  else res_level_kernel<false><<<grid, kResAllThreads, smem_bytes, stream>>>(args);
-  return cudaGetLastError();
+cudaError_t launch_res_level(const LevelArgs& args, bool inverse, int images, int bands, uint32_t smem_bytes,
+                             cudaStream_t stream) {
+  // one CTA per image, or a cluster of `bands` CTAs per image
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)(images * bands));
+  cfg.blockDim = dim3((unsigned)kResAllThreads);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)bands;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = bands > 1 ? 1 : 0;
+  if (inverse) return cudaLaunchKernelEx(&cfg, res_level_kernel<true>, args);
+  return cudaLaunchKernelEx(&cfg, res_level_kernel<false>, args);
 }
 
 cudaError_t configure_res_kernels(uint32_t max_smem_bytes) {

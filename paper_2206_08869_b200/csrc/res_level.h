@@ -16,7 +16,8 @@ constexpr int kResThreads = kResBuilderWarps * 32;           // their threads
 constexpr int kResIssuers = 3;                               // warps whose elected lane issues MMAs (tiles dealt between them)
 constexpr int kResAllThreads = kResThreads + 32 * (kResIssuers + 1);   // + the issuing warps and the warp that streams weights
 constexpr int kResMaxWidth = 128;      // hidden channels of a residual network (conv outputs), padded to 16
-constexpr int kResMaxPixels = 256;     // pixels per image at a residual level (two 128-row tiles)
+constexpr int kResMaxPixels = 256;     // pixels of an image that one CTA holds at a residual level
+constexpr int kResMaxBands = 8;        // row bands of an image (= CTAs of a thread-block cluster) at larger levels
 constexpr int kResMaxWSlots = 8;       // depth of the weight-slice ring
 
 // what a conv's epilogue does with its requantised outputs
@@ -64,11 +65,18 @@ struct ResHead {
   // padded layout of the activation buffers: rows of w2 = w + 2 positions, (h + 2) * w2 positions
   // rounded up to ntiles * 128 computed ones, `guard` rows before them, `rows` rows per channel chunk
   int32_t w2, guard, rows, ntiles;
-  int32_t pad[3];
+  // Levels of more than kResMaxPixels pixels per image: the image is cut into `bands` bands of hb rows,
+  // one CTA of a thread-block cluster each (bands = 1, hb = h otherwise). Every CTA keeps its band in
+  // the padded layout above with (hb + 2) rows; the row above and below hold the neighbouring bands'
+  // edge rows, which the neighbours write through distributed shared memory after every conv.
+  int32_t bands, hb;
+  int32_t pad[1];
 };
 static_assert(sizeof(ResHead) == 128, "128-byte header");
 
 cudaError_t configure_res_kernels(uint32_t max_smem_bytes);
-cudaError_t launch_res_level(const LevelArgs& args, bool inverse, int grid, uint32_t smem_bytes, cudaStream_t stream);
+// `images` images of `bands` row bands each (bands > 1: one thread-block cluster per image)
+cudaError_t launch_res_level(const LevelArgs& args, bool inverse, int images, int bands, uint32_t smem_bytes,
+                             cudaStream_t stream);
 
 }  // namespace iodf

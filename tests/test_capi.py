@@ -103,9 +103,12 @@ def test_gated_models_must_be_compacted():
 
 
 def test_residual_couplings_beyond_the_kernels_limits_are_refused():
-    """Residual-block couplings run for levels of at most 256 pixels per image and widths up to 128;
-    anything else must be refused on the host (IODF_EUNSUPPORTED), a malformed index list is EINVAL."""
-    m = S.make_residual_model(3, 3, 64, 64, [True], 1, 8, 1)          # 1024 pixels at the level
+    """Residual-block couplings run for levels of at most 2048 pixels per image (eight row bands of
+    256 pixels) and widths up to 128; anything else must be refused on the host (IODF_EUNSUPPORTED),
+    a malformed index list is EINVAL."""
+    m = S.make_residual_model(3, 3, 128, 128, [True], 1, 8, 1)        # 4096 pixels at the level
+    assert _status(m) == -6
+    m = S.make_residual_model(3, 3, 2, 1024, [True], 1, 8, 1)         # one row of 512 pixels: no bands of two rows
     assert _status(m) == -6
     m = S.make_residual_model(3, 3, 8, 8, [True], 1, 136, 1)          # hidden width above 128
     assert _status(m) == -6

@@ -47,11 +47,25 @@ def _both_ways(G, model, x):
     (16, [True, True], 2, 24, 2, (0.4, 0.8), 5),          # 64- and 16-pixel levels, odd kept widths
     (32, [True, True, True], 2, 40, 2, (0.4, 0.7), 3),    # 256 pixels: two tiles per image
     (16, [True, False], 1, 128, 8, (0.4, 0.7), 2),        # the paper's width and depth: 128 channels, 8 blocks
+    (64, [True, True], 1, 24, 2, (0.4, 0.7), 3),          # 1024 pixels: four row bands per image (a cluster), then 256
+    (48, [True], 2, 16, 1, None, 2),                      # 576 pixels: four bands of six rows, image rows of 24 pixels
 ])
 def test_residual_models_bit_exact(G, hw, splits, couplings, hidden, blocks, prune, batch):
     model = S.make_residual_model(0xE500 + hw + hidden, 3, hw, hw, splits, couplings, hidden, blocks, prune=prune)
     x = S.smooth_field_images(0xE600 + hw, batch, hw, hw, 2.0)
     _both_ways(G, model, x)
+
+
+def test_first_level_of_the_imagenet64_geometry_at_the_papers_width(G):
+    """App. B.1 on 64 x 64 images: the first level has 32 x 32 pixels, which one CTA cannot hold; it
+    runs as four row bands per image whose edge rows are exchanged after every conv. Width 128, eight
+    blocks, one coupling per level to keep the oracle's time down; batch position must not matter."""
+    import torch
+    model = S.make_residual_model(0xEA00, 3, 64, 64, [True, True], 1, 128, 8, prune=(0.4, 0.7))
+    x = S.smooth_field_images(0xEA01, 3, 64, 64, 4.0)
+    m, z_ref, p_ref = _both_ways(G, model, x)
+    z1, _ = G.iodf_forward(m, _t(x[2:3]))
+    np.testing.assert_array_equal(z1.cpu().numpy()[0], z_ref[2])
 
 
 def test_index_lists_in_any_order_and_chunks_without_a_filter(G):
@@ -141,3 +155,21 @@ def test_branch_output_near_the_int32_limit(G):
         ly["s"][:] = 0
     x = S.smooth_field_images(0xE901, 2, 8, 8, 2.0)
     _both_ways(G, model, x)
+
+
+def test_config_r64_in_the_benchmarks_launch_configuration(G):
+    """The paper's network on the ImageNet64 geometry (Sec. 5, App. B.1) at the benchmark's batch: the
+    oracle checks two sampled images, the round trip covers the whole batch."""
+    model = S.config_model("R64")
+    x = S.config_images("R64")
+    B = x.shape[0]
+    idx = np.array([0, B - 1])
+    z_ref, p_ref = O.forward(O.Packed(model), x[idx])
+    m = G.iodf_create(model, B)
+    z, p = G.iodf_forward(m, _t(x))
+    G.iodf_check(m)
+    np.testing.assert_array_equal(z.cpu().numpy()[idx], z_ref)
+    np.testing.assert_array_equal(p.cpu().numpy()[idx], p_ref)
+    xr = G.iodf_inverse(m, z)
+    G.iodf_check(m)
+    np.testing.assert_array_equal(xr.cpu().numpy(), x)
