@@ -13,7 +13,7 @@ M_BITS = 16
 WINDOW = 2048
 
 
-def logistic_codec(n_scales=64, umax=1024, final_ls=40, elems_per_stream=256):
+def logistic_codec(n_scales=64, umax=1024, final_ls=40, elems_per_stream=128):
     M = 1 << M_BITS
     u = np.arange(-umax, umax + 1, dtype=np.float64)
     top = M - (2 * WINDOW + 1)

@@ -110,11 +110,16 @@ __global__ void __launch_bounds__(kThreadsPerBlock) rans_encode_kernel(const Ran
 }
 
 // Decode: one WARP per stream. The state, the word pointer and every step are the same in all 32
-// lanes; only the symbol search is shared out: instead of 13 dependent bisection steps, three rounds
-// in which lane L tests one candidate k each (steps of 129, 5 and 1) and a ballot picks the largest
-// k with Cum(k) <= slot. A stream's latency, which bounds the decompressor (a block's streams are
-// few and long), drops about threefold; the redundant lanes are free because the kernel is
-// latency-bound.
+// lanes; what the lanes share out is everything that would otherwise be a dependent trip to memory
+// or a dependent search step on the stream's serial chain (state -> symbol -> state):
+//   * the symbol search: instead of 13 bisection steps, three rounds in which lane L tests one
+//     candidate k each (steps of 129, 5 and 1) and a ballot picks the largest k with Cum(k) <= slot;
+//     the last round's values also give C = Cum(k) and Cum(k + 1) by shuffle;
+//   * the prior parameters: the (mu, scale index) of the next 32 elements are loaded by the 32 lanes
+//     in one go and handed out by shuffle, so no global-memory latency sits between two symbols;
+//   * the coded words: the lanes hold a window of the stream's next 32 words (the decoder reads the
+//     stream backwards), refilled when used up; a renormalisation is a shuffle.
+// A stream's latency bounds the decompressor (a block's streams are few and long).
 __global__ void __launch_bounds__(kThreadsPerBlock) rans_decode_kernel(const RansArgs a, int q,
                                                                        const uint16_t* __restrict__ words,
                                                                        const uint32_t* __restrict__ counts,
@@ -133,48 +138,70 @@ __global__ void __launch_bounds__(kThreadsPerBlock) rans_decode_kernel(const Ran
   const long sid = (long)b * a.n_streams + blk.first_stream + j;
   const long n_el = (blk.n - j + ns - 1) / ns;
   const uint16_t* in = words + sid * a.cap;
-  long pos = min((long)counts[sid], (long)a.cap);
+  long pos = min((long)counts[sid], (long)a.cap);      // words not yet consumed: in[0 .. pos)
   uint32_t bad = 0;
+  // window of the next 32 words: lane L holds in[top - 1 - L] (0 before the stream's first word)
+  long top = pos;
+  uint32_t win = (top - 1 - lane >= 0) ? in[top - 1 - lane] : 0u;
   auto next = [&]() -> uint32_t {               // never reads before the stream's first word
     if (pos <= 0) { bad = 1u; return 0u; }
-    return in[--pos];
+    int used = (int)(top - pos);
+    if (used == 32) {
+      top = pos;
+      win = (top - 1 - lane >= 0) ? in[top - 1 - lane] : 0u;
+      used = 0;
+    }
+    --pos;
+    return __shfl_sync(0xFFFFFFFFu, win, used);
   };
   uint32_t x = next() << 16;
   x |= next();
   int32_t* zb = z + (long)b * a.d + blk.z_off;
   const int32_t* pb = prior + (long)b * 2 * a.d_fact;
-  for (long i = 0; i < n_el; ++i) {
-    const long e = j + i * ns;
-    int32_t mu; int ls;
-    prior_of(a, blk, pb, e, &mu, &ls, &bad);
-    const uint32_t slot = x & 0xFFFFu;
-    // largest k in [0, 4096] with Cum(k) <= slot (Cum(0) = 0 <= slot always; Cum(k > 4096) = M > slot)
-    int k = 0;
+  for (long i0 = 0; i0 < n_el; i0 += 32) {
+    // this lane's element of the next 32: its prior parameters now, its decoded value at the end
+    int32_t mu_l = 0, zv_l = 0;
+    int ls_l = a.final_ls;
+    if (i0 + lane < n_el) prior_of(a, blk, pb, j + (i0 + lane) * ns, &mu_l, &ls_l, &bad);
+    const int n_here = (int)min(32l, n_el - i0);
+    for (int ii = 0; ii < n_here; ++ii) {
+      const int32_t mu = __shfl_sync(0xFFFFFFFFu, mu_l, ii);
+      const int ls = __shfl_sync(0xFFFFFFFFu, ls_l, ii);
+      const uint32_t slot = x & 0xFFFFu;
+      // largest k in [0, 4096] with Cum(k) <= slot (Cum(0) = 0 <= slot always; Cum(k > 4096) = M > slot)
+      int k = 0;
 #pragma unroll
-    for (int round = 0; round < 3; ++round) {
-      const int step = round == 0 ? 129 : (round == 1 ? 5 : 1);
-      const int cand = k + lane * step;
-      const unsigned ok = __ballot_sync(0xFFFFFFFFu, cum(t, ls, cand) <= slot);   // a prefix of the lanes (Cum is monotone)
-      k += (31 - __clz((int)ok)) * step;
-    }
-    const uint32_t C = cum(t, ls, k), F = cum(t, ls, k + 1) - C;
-    x = F * (x >> 16) + slot - C;
-    if (x < (1u << 16)) x = (x << 16) | next();
-    int32_t zv;
-    if (k == 0 || k == 2 * kWin) {
-      const uint32_t h = x & 0xFFFFu;
-      x >>= 16;                                  // F = 1, C = slot: x = x / M
+      for (int round = 0; round < 2; ++round) {
+        const int step = round == 0 ? 129 : 5;
+        const unsigned ok = __ballot_sync(0xFFFFFFFFu, cum(t, ls, k + lane * step) <= slot);   // a prefix of the lanes (Cum is monotone)
+        k += (31 - __clz((int)ok)) * step;
+      }
+      const uint32_t cl = cum(t, ls, k + lane);
+      const int sel = 31 - __clz((int)__ballot_sync(0xFFFFFFFFu, cl <= slot));
+      k += sel;
+      const uint32_t C = __shfl_sync(0xFFFFFFFFu, cl, sel);
+      const uint32_t Cn = sel < 31 ? __shfl_sync(0xFFFFFFFFu, cl, sel + 1) : cum(t, ls, k + 1);
+      const uint32_t F = Cn - C;
+      x = F * (x >> 16) + slot - C;
       if (x < (1u << 16)) x = (x << 16) | next();
-      const uint32_t l = x & 0xFFFFu;
-      x >>= 16;
-      if (x < (1u << 16)) x = (x << 16) | next();
-      zv = (int32_t)((h << 16) | l);
-    } else {
-      zv = (int32_t)((long long)mu + (k - kWin));
+      int32_t zv;
+      if (k == 0 || k == 2 * kWin) {
+        const uint32_t h = x & 0xFFFFu;
+        x >>= 16;                                  // F = 1, C = slot: x = x / M
+        if (x < (1u << 16)) x = (x << 16) | next();
+        const uint32_t l = x & 0xFFFFu;
+        x >>= 16;
+        if (x < (1u << 16)) x = (x << 16) | next();
+        zv = (int32_t)((h << 16) | l);
+      } else {
+        zv = (int32_t)((long long)mu + (k - kWin));
+      }
+      if (lane == ii) zv_l = zv;
     }
-    if (lane == 0) zb[e] = zv;
+    if (i0 + lane < n_el) zb[j + (i0 + lane) * ns] = zv_l;
   }
   if (pos != 0 || x != (1u << 16)) bad = 1u;     // every word used and the state back at its start
+  bad = __any_sync(0xFFFFFFFFu, bad != 0) ? 1u : 0u;
   if (bad && lane == 0 && a.errors) atomicAdd(a.errors, 1u);
 }
 
