@@ -513,6 +513,10 @@ __device__ __forceinline__ void requant_input(const PixelPass& pp, const int32_t
 }
 
 // ---- a level's input and output index maps ---------------------------------------------------------
+// Planes of at least this many bytes leave through bulk copies; smaller ones (the deep levels: 16 or 64
+// pixels per image) are cheaper to store with the threads than to issue one copy each for.
+constexpr int kBulkStoreMinBytes = 1024;
+
 // Encode: space-to-depth on load (first level: uint8 images, or the patch grid of one image).
 // Decode: merge of the channels that come back from the deeper level with this level's block of z.
 template <bool kInv>
@@ -563,6 +567,25 @@ __device__ __forceinline__ void level_store(const LevelPlan& P, const LevelArgs&
     // split on store: factored-out half -> z block of this level; kept half -> next level (or
     // the final z block)
     int32_t* keep_out = reinterpret_cast<int32_t*>(a.out);
+    if (px * 4 >= kBulkStoreMinBytes && (px & 3) == 0) {    // (16-byte granularity of the copies)
+      // A channel plane of an image is px contiguous words both in shared memory and in every
+      // destination layout: one bulk copy shared -> global per plane, issued by as many threads as
+      // there are planes, instead of a pass of the threads over the elements. The planes were
+      // written through the generic proxy: every thread fences its writes towards the async proxy
+      // first, and the issuing threads wait until their copies have read shared memory.
+      ptx::fence_async_smem();
+      asm volatile("bar.sync 2, %0;" ::"r"(nthreads) : "memory");
+      for (int pl = tid; pl < nimg * c; pl += nthreads) {
+        const int g = pl / c, k = pl - g * c;
+        const size_t b = (size_t)(img0 + g);
+        int32_t* dst = k >= P.keep_c ? a.z + b * P.d + P.z_off + (size_t)(k - P.keep_c) * px
+                       : (P.is_last ? a.z + b * P.d + P.z_final_off + (size_t)k * px
+                                    : keep_out + (b * P.keep_c + k) * (size_t)px);
+        ptx::bulk_s2g(dst, ptx::smem_u32(v + P.col_out[k] * pg + g * px), (uint32_t)px * 4u);
+      }
+      ptx::bulk_s2g_commit_and_wait_read();
+      return;
+    }
 #pragma unroll 4
     for (int e = tid; e < nimg * per_img; e += nthreads) {
       const int g = fdiv(e, P.mul_per_img), r = e - g * per_img;
