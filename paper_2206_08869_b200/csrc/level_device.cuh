@@ -527,6 +527,32 @@ __device__ __forceinline__ void level_load(const LevelPlan& P, const LevelArgs& 
   if (!kInv) {
     // space-to-depth on load: plane c*4 + dy*2 + dx, pixel (i, j) <- in[c][2i+dy][2j+dx]
     const int w2 = 2 * w;
+    if ((w & 1) == 0 && (a.img_w & 3) == 0) {
+      // Four neighbours of an input row per thread and step: one 4-byte (uint8 images) or 16-byte
+      // (int32 channels) load, and two 8-byte stores, one into the dx = 0 plane and one into the
+      // dx = 1 plane. Every index below is a multiple of four, so the accesses are aligned.
+#pragma unroll 2
+      for (int e = 4 * tid; e < nimg * per_img; e += 4 * nthreads) {
+        const int g = fdiv(e, P.mul_per_img), r = e - g * per_img;
+        const int ci = fdiv(r, P.mul_4px), r2 = r - ci * 4 * px;
+        const int y = fdiv(r2, P.mul_w2), x = r2 - y * w2;
+        size_t src = (size_t)(img0 + g) * per_img + r;
+        if (P.is_first && a.img_w > 0) {                 // patch (by, bx) of one large image
+          const int by = fdiv(img0 + g, a.mul_patches_x), bx = img0 + g - by * a.patches_x;
+          src = ((size_t)ci * a.img_h + (size_t)(by * 2 * P.h + y)) * a.img_w + (size_t)(bx * w2 + x);
+        }
+        int4 q;
+        if (P.is_first) {
+          const uint32_t b4 = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const uint8_t*>(a.in) + src);
+          q = make_int4((int)(b4 & 0xFFu), (int)((b4 >> 8) & 0xFFu), (int)((b4 >> 16) & 0xFFu), (int)(b4 >> 24));
+        } else {
+          q = *reinterpret_cast<const int4*>(reinterpret_cast<const int32_t*>(a.in) + src);
+        }
+        int32_t* d0 = v + (ci * 4 + (y & 1) * 2) * pg + g * px + (y >> 1) * w + (x >> 1);
+        *reinterpret_cast<int2*>(d0) = make_int2(q.x, q.z);
+        *reinterpret_cast<int2*>(d0 + pg) = make_int2(q.y, q.w);
+      }
+    } else
 #pragma unroll 4
     for (int e = tid; e < nimg * per_img; e += nthreads) {
       const int g = fdiv(e, P.mul_per_img), r = e - g * per_img;
