@@ -284,9 +284,8 @@ def main():
     peak_burst, peak_sustained = measure_int8_peak(G, m, stream, torch)
     peak_int8 = peak_burst                      # a step is far below a second: the burst figure applies
     achieved = 2.0 * top_macs * B / (lvl[top] * 1e-3) / 1e12
-    res = bool(model["levels"][top]["couplings"][0].get("blocks"))
     traffic, traffic_note = stored_traffic("config%s_b%d_level%d" % (cfg, B, top))
-    roofline = {"bound": "tensor", "kernel": "%s<encode> level %d" % ("res_level_kernel" if res else "level_kernel", top),
+    roofline = {"bound": "tensor", "kernel": "%s<encode> level %d" % (G.iodf_level_kernel_name(m, top), top),
                 "achieved": achieved, "peak": peak_int8, "unit": "TOP/s (int8)", "frac": achieved / peak_int8,
                 "traffic": traffic, "traffic_note": traffic_note,
                 "peak_source": "tcgen05.mma kind::i8 128x256x32 MMA-only kernel, all SMs, measured in this run (burst: best ~10 ms launch)",

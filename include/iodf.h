@@ -405,6 +405,10 @@ int iodf_selftest_timeout(iodf_model* m, uint32_t tries, void* cuda_stream);
  */
 int iodf_int8_mma_peak(iodf_model* m, uint32_t mma_groups, void* cuda_stream, unsigned long long* ops_out);
 
+/* Name of the kernel template that runs level `level` of this model (for profiles and reports): the
+ * library picks one per level when the model is created. "" for a bad argument. */
+const char* iodf_level_kernel_name(const iodf_model* m, int level);
+
 /* Number of kernel launches one iodf_forward / iodf_inverse call enqueues. */
 int iodf_launches_per_call(const iodf_model* m, int inverse);
 

@@ -9,7 +9,8 @@ from .binding import (IodfError, Model, iodf_create, iodf_destroy, iodf_forward,
                       iodf_forward_host, iodf_inverse_host, iodf_forward_timed, iodf_inverse_timed,
                       iodf_get_layout, iodf_forward_static, iodf_static_scratch_bytes_per_image,
                       IODF_STATIC_SCRATCH_BYTES, iodf_check, iodf_strerror,
-                      iodf_launches_per_call, iodf_selftest_timeout, iodf_int8_mma_peak, load_library,
+                      iodf_launches_per_call, iodf_selftest_timeout, iodf_int8_mma_peak, iodf_level_kernel_name,
+                      load_library,
                       DECLARED_SYMBOLS)
 
 __all__ = ["IodfError", "Model", "iodf_create", "iodf_destroy", "iodf_forward", "iodf_inverse",
@@ -19,5 +20,6 @@ __all__ = ["IodfError", "Model", "iodf_create", "iodf_destroy", "iodf_forward", 
            "iodf_compress_host", "iodf_decompress_host",
            "iodf_forward_host", "iodf_inverse_host", "iodf_forward_timed", "iodf_inverse_timed", "iodf_get_layout", "iodf_forward_static", "iodf_static_scratch_bytes_per_image",
            "IODF_STATIC_SCRATCH_BYTES", "iodf_check", "iodf_strerror",
-           "iodf_launches_per_call", "iodf_selftest_timeout", "iodf_int8_mma_peak", "load_library",
+           "iodf_launches_per_call", "iodf_selftest_timeout", "iodf_int8_mma_peak", "iodf_level_kernel_name",
+           "load_library",
            "DECLARED_SYMBOLS"]

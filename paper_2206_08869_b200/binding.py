@@ -18,7 +18,7 @@ DECLARED_SYMBOLS = ["iodf_create", "iodf_destroy", "iodf_get_layout", "iodf_forw
                     "iodf_rans_unpack", "iodf_compress_host", "iodf_decompress_host",
                     "iodf_forward_host", "iodf_inverse_host", "iodf_forward_timed", "iodf_inverse_timed", "iodf_forward_static",
                     "iodf_static_scratch_bytes_per_image", "iodf_check", "iodf_launches_per_call",
-                    "iodf_selftest_timeout", "iodf_int8_mma_peak",
+                    "iodf_selftest_timeout", "iodf_int8_mma_peak", "iodf_level_kernel_name",
                     "iodf_strerror", "iodf_last_cuda_error"]
 
 
@@ -148,6 +148,8 @@ def load_library(path=None):
     L.iodf_selftest_timeout.argtypes = [vp, C.c_uint32, vp]
     L.iodf_int8_mma_peak.restype = C.c_int
     L.iodf_int8_mma_peak.argtypes = [vp, C.c_uint32, vp, C.POINTER(C.c_ulonglong)]
+    L.iodf_level_kernel_name.restype = C.c_char_p
+    L.iodf_level_kernel_name.argtypes = [vp, C.c_int]
     L.iodf_launches_per_call.restype = C.c_int
     L.iodf_launches_per_call.argtypes = [vp, C.c_int]
     L.iodf_strerror.restype = C.c_char_p
@@ -520,6 +522,10 @@ def iodf_int8_mma_peak(model, mma_groups, stream=None):
     if rc != 0:
         raise IodfError(rc, "iodf_int8_mma_peak")
     return int(ops.value)
+
+
+def iodf_level_kernel_name(model, level):
+    return load_library().iodf_level_kernel_name(model.handle, int(level)).decode()
 
 
 def iodf_launches_per_call(model, inverse=False):

@@ -1452,6 +1452,12 @@ int iodf_int8_mma_peak(iodf_model* m, uint32_t mma_groups, void* cuda_stream, un
   return IODF_OK;
 }
 
+const char* iodf_level_kernel_name(const iodf_model* m, int level) {
+  if (!m || level < 0 || level >= (int)m->levels.size()) return "";
+  const LevelPlan& P = m->levels[level].plan;
+  return P.residual ? "res_level_kernel" : (P.pipe ? "level_pipe_kernel" : "level_kernel");
+}
+
 int iodf_launches_per_call(const iodf_model* m, int inverse) {
   (void)inverse;
   return m ? (int)m->levels.size() : 0;
