@@ -21,6 +21,8 @@ def source_hash():
     h = hashlib.sha256(" ".join(NVCC_FLAGS).encode())
     deps = sorted(glob.glob(os.path.join(CSRC, "*"))) + [os.path.join(HERE, "..", "include", "iodf.h")]
     for p in deps:
+        if os.path.isdir(p):         # csrc/microbench: stand-alone programs, not part of the library
+            continue
         h.update(os.path.basename(p).encode())
         with open(p, "rb") as f:
             h.update(f.read())

@@ -392,6 +392,7 @@ bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32
       }
       P.s_total = off;
       P.pipe = pipe ? 1 : 0;
+      P.lean = (pd.eligible && mode != 3) ? 1 : 0;
       P.r_col[0] = r3_separate ? (int)pd.n_hidden : kSlotCols;
       P.r_col[1] = r3_separate ? 2 * (int)pd.n_hidden : 0;
       P.r_col[2] = r3_separate ? (int)pd.n_taps : kSlotCols;
@@ -857,7 +858,7 @@ cudaError_t launch_any_level(const LevelPlan& P, const LevelArgs& a, bool invers
   const int grid = (B + P.group - 1) / P.group;
   if (P.residual) return launch_res_level(a, inverse, B, P.res_bands, P.s_total, st);
   if (P.pipe) return launch_level_pipe(a, inverse, grid, P.s_total, st);
-  return launch_level(a, inverse, grid, P.s_total, st);
+  return launch_level(a, inverse, P.lean != 0, grid, P.s_total, st);
 }
 
 int run_forward(iodf_model* m, const uint8_t* x, int B, int32_t* z, int32_t* prior, cudaStream_t st,

@@ -117,6 +117,8 @@ struct LevelPlan {
   int32_t streamed;              // 1: weights are streamed per tile in 32-byte K-slices through a ring of
                                  //    kRingDepth slots at s_w[0] (hidden widths above 256, one tile in flight)
   uint32_t ring_slot_bytes;
+  int32_t lean;                  // 1: every hidden layer in the folded requantisation flavour with the 0..127 clip,
+                                 //    weights not streamed: the general kernel's small variant runs the level
   int32_t pipe;                  // 1: the level runs in the kernel that splits a tile's work by role (several
                                  //    tiles per CTA, two tile slots, resident weights, folded requantisation with
                                  //    the 0..127 clip)

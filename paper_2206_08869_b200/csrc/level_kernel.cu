@@ -312,7 +312,11 @@ __device__ void run_control_streamed(const Ctx& cx, const LevelPlan& P, const Le
 }
 
 // ---- workers ----------------------------------------------------------------------------------
-template <bool kInv>
+// kLean: every hidden layer of the level is in the folded requantisation flavour with the 0..127
+// clip (what the model packer produces for the usual layers), so that the epilogues need one code
+// path instead of seven. The deep levels run every phase's code once per coupling, and what they
+// wait for most, beside memory, is instruction fetch: the smaller the loop body, the better.
+template <bool kInv, bool kLean>
 __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const LevelArgs& a, const Steps& st, int img0, int pvalid,
                             int ntv) {
   uint8_t* smem = cx.smem;
@@ -413,13 +417,16 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
         for (int sl = 0; sl < nt; ++sl) {                     // requant, conv 1x1
           wait_d(sl);
           use_slot(sl);
-          epilogue_hidden(cx, M.mode1, M.us1, M.n1, M.kd2, h1, u1, M.lo1, M.hi1, kBiasColumnsLo, kBiasColumnsHi, sA);
+          if (kLean) epilogue_hidden_t(cx, M.n1, M.kd2, Requant<kModeFolded, kClipS8Relu>{h1, u1, 0, 127, M.us1 - 1, 1ll << (30 + M.us1)},
+                                       kBiasColumnsLo, kBiasColumnsHi, sA);
+          else epilogue_hidden(cx, M.mode1, M.us1, M.n1, M.kd2, h1, u1, M.lo1, M.hi1, kBiasColumnsLo, kBiasColumnsHi, sA);
           arrive_a(sl);
         }
         for (int sl = 0; sl < nt; ++sl) {                     // requant, conv 3x3 as per-tap partials
           wait_d(sl);
           use_slot(sl);
-          epilogue_hidden(cx, M.mode2, M.us2, M.n2, M.kd3, h2, u2, M.lo2, M.hi2, 0u, 0u, sA);
+          if (kLean) epilogue_hidden_t(cx, M.n2, M.kd3, Requant<kModeFolded, kClipS8Relu>{h2, u2, 0, 127, M.us2 - 1, 1ll << (30 + M.us2)}, 0u, 0u, sA);
+          else epilogue_hidden(cx, M.mode2, M.us2, M.n2, M.kd3, h2, u2, M.lo2, M.hi2, 0u, 0u, sA);
           arrive_a(sl);
         }
         for (int sl = 0; sl < nt; ++sl) {                     // shifted sum into the accumulator
@@ -438,7 +445,7 @@ __device__ __forceinline__ void run_workers(Ctx& cx, const LevelPlan& P, const L
   }
 }
 
-template <bool kInv>
+template <bool kInv, bool kLean>
 __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
   extern __shared__ __align__(1024) uint8_t smem[];
   __shared__ Ctl ctl;
@@ -501,7 +508,7 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
   if (warp >= kWorkerWarps) {
     // The packed blocks are written once at model creation, so the first copies need not wait for
     // the previous kernel; run_control starts them before it joins the workers' first barrier.
-    if (P.streamed) {
+    if (!kLean && P.streamed) {
       cta_barrier();                     // the workers have loaded the flow variable
       run_control_streamed(cx, P, a, st, ntv);
     } else {
@@ -520,7 +527,7 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
     level_load<kInv>(P, a, v, img0, nimg, tid, kWorkers);
     cta_barrier();
 
-    run_workers<kInv>(cx, P, a, st, img0, pvalid, ntv);
+    run_workers<kInv, kLean>(cx, P, a, st, img0, pvalid, ntv);
 
     level_store<kInv>(P, a, v, img0, nimg, tid, lane, kWorkers);
   }
@@ -532,7 +539,8 @@ __global__ void __launch_bounds__(kThreads, 1) level_kernel(const LevelArgs a) {
 
 }  // namespace
 
-cudaError_t launch_level(const LevelArgs& args, bool inverse, int grid, uint32_t smem_bytes, cudaStream_t stream) {
+cudaError_t launch_level(const LevelArgs& args, bool inverse, bool lean, int grid, uint32_t smem_bytes,
+                         cudaStream_t stream) {
   // Programmatic dependent launch: the CTAs of this level may start (barrier set-up, TMEM
   // allocation, index records) while the previous kernel in the stream drains; the kernel itself
   // waits for that kernel's completion before it touches anything a kernel writes.
@@ -546,15 +554,18 @@ cudaError_t launch_level(const LevelArgs& args, bool inverse, int grid, uint32_t
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (inverse) return cudaLaunchKernelEx(&cfg, level_kernel<true>, args);
-  return cudaLaunchKernelEx(&cfg, level_kernel<false>, args);
+  if (lean) return inverse ? cudaLaunchKernelEx(&cfg, level_kernel<true, true>, args)
+                           : cudaLaunchKernelEx(&cfg, level_kernel<false, true>, args);
+  return inverse ? cudaLaunchKernelEx(&cfg, level_kernel<true, false>, args)
+                 : cudaLaunchKernelEx(&cfg, level_kernel<false, false>, args);
 }
 
 cudaError_t configure_level_kernels(uint32_t max_smem_bytes) {
-  cudaError_t e = cudaFuncSetAttribute(level_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)max_smem_bytes);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(level_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem_bytes);
+  cudaError_t e = cudaFuncSetAttribute(level_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem_bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(level_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem_bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(level_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem_bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(level_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem_bytes);
+  return e;
 }
 
 }  // namespace iodf

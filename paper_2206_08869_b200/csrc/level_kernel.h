@@ -36,6 +36,9 @@ struct LevelArgs {
 };
 
 cudaError_t configure_level_kernels(uint32_t max_smem_bytes);
-cudaError_t launch_level(const LevelArgs& args, bool inverse, int grid, uint32_t smem_bytes, cudaStream_t stream);
+// lean: the kernel variant for levels whose hidden layers all use the folded requantisation flavour with the
+// 0..127 clip and whose weights are not streamed (LevelPlan::lean)
+cudaError_t launch_level(const LevelArgs& args, bool inverse, bool lean, int grid, uint32_t smem_bytes,
+                         cudaStream_t stream);
 
 }  // namespace iodf
