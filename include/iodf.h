@@ -91,8 +91,10 @@ typedef struct {
  *   m = clip(ReLU(rq(conv_a(x))));  b = rq(conv_b(m))   (conv_b: relu = 0, has_clamp = 0, K' kept outputs)
  *   x = clip(max(rq(x; short_m0, short_s) [all D channels]  +  scatter of b through idx, 0), clamp_lo, clamp_hi)
  * and conv_out maps x to the integer translation. This build runs it for 3x3 convs with D and every
- * kept width <= 128, hidden activations in 0..255, and levels of at most 256 pixels per
- * image; all couplings of a level must then be of this form.
+ * kept width <= 128, hidden activations in 0..255, and levels of at most 2048 pixels per
+ * image (above 256 pixels the rows of an image are shared out over up to eight CTAs of one
+ * thread-block cluster, which needs bands of at least two rows); all couplings of a level must
+ * then be of this form.
  */
 typedef struct {
   const int32_t* perm;            /* HOST, C entries, a permutation of 0..C-1                        */
@@ -158,7 +160,7 @@ typedef struct iodf_model iodf_model;
  * conv3x3+ReLU+clip -> conv1x1+ReLU+clip -> conv3x3 with hidden activations inside the signed
  * 8-bit range and hidden widths up to 512 kept channels (above 256 the weights are streamed from
  * L2 for every tile instead of staying in shared memory), couplings with residual blocks (see
- * iodf_coupling_desc) at levels of at most 256 pixels per image, and 3x3 prior heads.
+ * iodf_coupling_desc) at levels of at most 2048 pixels per image, and 3x3 prior heads.
  */
 int iodf_create(const iodf_model_desc* desc, const int8_t* weights, size_t weights_count,
                 const int32_t* requant, size_t requant_count, int device, iodf_model** out);
