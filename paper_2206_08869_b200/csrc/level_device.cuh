@@ -467,6 +467,11 @@ struct PixelPass {
   int pg, ca, cb, cpad, pvalid;
   uint32_t mul_pv;       // magic multiplier of pvalid (0: pvalid = 1)
   int tid, nthreads;     // this thread among the threads that share the pass
+  // pvalid and pg multiples of four: four pixels of a plane per 16-byte access
+  __device__ __forceinline__ bool by_four() const { return ((pvalid | pg) & 3) == 0; }
+  __device__ __forceinline__ uint32_t mul_pv4() const {
+    return pvalid > 4 ? (uint32_t)((0xFFFFFFFFull / (uint32_t)(pvalid >> 2)) + 1ull) : 0u;
+  }
 };
 
 // x_b +/-= rq(acc + bias) of the coupling whose meta block is M. Work item = (channel, pixel),
@@ -477,6 +482,28 @@ __device__ __forceinline__ void apply_translation(const PixelPass& pp, const Cou
   const uint8_t* pm = reinterpret_cast<const uint8_t*>(M);
   const int32_t* colB = reinterpret_cast<const int32_t*>(pm + M->off_colB);
   const OutRq* orq = reinterpret_cast<const OutRq*>(pm + M->off_out);
+  if (pp.by_four()) {
+    // work item = (channel, four neighbouring pixels): one 16-byte load and store per plane
+    const int q = pp.pvalid >> 2, items4 = pp.cb * q;
+    const uint32_t mul = pp.mul_pv4();
+    for (int it = pp.tid; it < items4; it += pp.nthreads) {
+      const int c = fdiv(it, mul), p = (it - c * q) << 2;
+      const OutRq o = orq[c];
+      int4* ap = reinterpret_cast<int4*>(pp.acc + c * pp.pg + p);
+      uint4* vp = reinterpret_cast<uint4*>(&pp.v[colB[c] * pp.pg + p]);
+      const int4 t = *ap;
+      uint4 x = *vp;
+      *ap = make_int4(0, 0, 0, 0);
+      const uint32_t t0 = (uint32_t)rq_out(t.x, o), t1 = (uint32_t)rq_out(t.y, o);
+      const uint32_t t2 = (uint32_t)rq_out(t.z, o), t3 = (uint32_t)rq_out(t.w, o);
+      x.x = kInv ? x.x - t0 : x.x + t0;
+      x.y = kInv ? x.y - t1 : x.y + t1;
+      x.z = kInv ? x.z - t2 : x.z + t2;
+      x.w = kInv ? x.w - t3 : x.w + t3;
+      *vp = x;
+    }
+    return;
+  }
   const int items = pp.cb * pp.pvalid;
   auto one = [&](int it) {
     const int c = fdiv(it, pp.mul_pv), p = it - c * pp.pvalid;
@@ -506,9 +533,10 @@ __device__ __forceinline__ void requant_input(const PixelPass& pp, const int32_t
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       y[i] = 0;
-      if (g0 + i < pp.ca) y[i] = clampi(rq_exact(pp.v[cols[g0 + i] * pp.pg + p], m0, s), -128, 127);
+      if (g0 + i < pp.ca) y[i] = rq_exact(pp.v[cols[g0 + i] * pp.pg + p], m0, s);
     }
-    *reinterpret_cast<uint32_t*>(pp.xa + (size_t)p * pp.cpad + g0) = pack4(y[0], y[1], y[2], y[3]);
+    // the clip to -128..127 is the pack's saturation
+    *reinterpret_cast<uint32_t*>(pp.xa + (size_t)p * pp.cpad + g0) = pack4_sat(y[0], y[1], y[2], y[3]);
   }
 }
 
