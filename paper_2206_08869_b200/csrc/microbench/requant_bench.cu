@@ -1,11 +1,13 @@
 // Microbenchmark behind the epilogue's design: how many hidden activations per clock one SM can
 // requantise (y = clip(hi32(acc * m0 + 2^(30+s)) >> (s-1), 0, 127), Eq. "quant_conv" of Sec. 4.1 in
 // the library's fixed-point form), for a few instruction sequences, with the accumulators in
-// registers and read from tensor memory, at 1 to 8 warps per scheduler. Not part of the library.
+// registers and read from tensor memory, at 1 to 8 warps per scheduler, and for a form that goes
+// through the fp64 pipe. Not part of the library.
 //
 //   nvcc -O3 -std=c++17 -gencode arch=compute_100a,code=sm_100a -o requant_bench requant_bench.cu && ./requant_bench
 #include <cstdio>
 #include <cstdint>
+#include <cmath>
 #include <cuda_runtime.h>
 
 #include "../ptx.cuh"
@@ -193,6 +195,91 @@ void run_tmem(const char* name, const int* dm0, unsigned long long* dclk, uint32
   }
 }
 
+// ---- the same requantisation through the fp64 pipe ---------------------------------------------------
+// y = floor((acc * m0 + 2^(31+sh)) / 2^(32+sh)) in double precision, exact while |acc * m0| + 2^(31+sh)
+// < 2^53: acc becomes a double by the exponent trick (2^52 + 2^31 + acc as the low word of 0x43300000),
+// one fused multiply-add with ms = m0 * 2^-(32+sh) and c = 0.5 - (2^52 + 2^31) * ms gives
+// (acc * m0 + 2^(31+sh)) / 2^(32+sh) without rounding, and a round-down add of 1.5 * 2^52 leaves its
+// floor in the low word. Is the otherwise idle fp64 pipe a second lane for the epilogue?
+__device__ __forceinline__ int rq_f64(int acc, double ms, double c) {
+  const double d = __hiloint2double(0x43300000, acc ^ 0x80000000);
+  return __double2loint(__dadd_rd(fma(d, ms, c), 6755399441055744.0));
+}
+
+// kF of every 16 columns go through the fp64 form (0: none, 16: all)
+template <int kF>
+__global__ void bench_f64(const int* __restrict__ gm0, int iters, int sh, unsigned long long* out_clk, uint32_t* out_sum) {
+  __shared__ __align__(16) int sm0[256];
+  __shared__ __align__(16) double2 smc[256];
+  __shared__ __align__(16) uint4 sout[1024];
+  for (int i = threadIdx.x; i < 256; i += blockDim.x) {
+    sm0[i] = gm0[i];
+    const double ms = ldexp((double)gm0[i], -(32 + sh));
+    smc[i] = make_double2(ms, 0.5 - 4503601774854144.0 * ms);
+  }
+  __syncthreads();
+  const long long rnd64 = 1ll << (31 + sh);
+  int acc[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) acc[i] = ((threadIdx.x * 977 + i * 131071) ^ 0x5a5a) & 0x1FFFFF;
+  uint32_t sum = 0;
+  const unsigned long long t0 = clock64();
+  for (int it = 0; it < iters; ++it) {
+    const int ch0 = (it * 16) & 255;
+    int y[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const bool f = (i * kF) / 16 != ((i + 1) * kF) / 16;
+      if (f) { const double2 k = smc[ch0 + i]; y[i] = rq_f64(acc[i] - (1 << 20), k.x, k.y); }
+      else y[i] = rq1w(acc[i] - (1 << 20), sm0[ch0 + i], sh, rnd64);
+    }
+    uint32_t wd[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) wd[q] = relu4(pack4_sat(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]));
+    sout[threadIdx.x & 1023] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = (acc[i] + 0x10101 * (it + 1)) & 0x1FFFFF;     // |acc - 2^20| stays below 2^21
+    sum += wd[0] + wd[3] * 3u + wd[1] * 5u + wd[2] * 7u;
+  }
+  const unsigned long long t1 = clock64();
+  if (threadIdx.x == 0) out_clk[blockIdx.x] = t1 - t0;
+  out_sum[blockIdx.x * blockDim.x + threadIdx.x] = sum;      // a function of the requantised values alone
+}
+
+// both forms on every accumulator in [-2^21, 2^21) for a few multipliers and shifts; the constants of
+// the fp64 form come from the host
+struct F64Case { int m0, sh; double ms, c; };
+__global__ void check_f64(const F64Case* __restrict__ cases, int n, unsigned long long* bad) {
+  const int a = (int)(blockIdx.x * blockDim.x + threadIdx.x) - (1 << 21);
+  unsigned long long nb = 0;
+  for (int j = 0; j < n; ++j) {
+    const F64Case k = cases[j];
+    nb += rq1w(a, k.m0, k.sh, 1ll << (31 + k.sh)) != rq_f64(a, k.ms, k.c);
+  }
+  if (nb) atomicAdd(bad, nb);
+}
+
+template <int kF>
+void run_f64(const char* name, const int* dm0, unsigned long long* dclk, uint32_t* dsum, uint32_t* ref) {
+  const int iters = 2000;
+  for (int warps : {4, 16, 20}) {
+    bench_f64<kF><<<1, warps * 32>>>(dm0, iters, 7, dclk, dsum);
+    cudaDeviceSynchronize();
+    bench_f64<kF><<<1, warps * 32>>>(dm0, iters, 7, dclk, dsum);
+    cudaError_t e = cudaDeviceSynchronize();
+    unsigned long long clk = 0;
+    cudaMemcpy(&clk, dclk, sizeof(clk), cudaMemcpyDeviceToHost);
+    uint32_t h[1024];
+    cudaMemcpy(h, dsum, 4 * warps * 32, cudaMemcpyDeviceToHost);
+    uint32_t x = 0;
+    for (int i = 0; i < warps * 32; ++i) x = x * 31 + h[i];
+    const char* same = "";
+    if (kF == 0) ref[warps] = x; else same = ref[warps] == x ? "same results" : "DIFFERENT results";
+    printf("%-32s warps/SM %2d: %7.1f clk per chunk per warp, %6.2f activations/clk/SM  (%s) %s\n", name, warps,
+           (double)clk / iters, 16.0 * 32 * warps * iters / (double)clk, cudaGetErrorString(e), same);
+  }
+}
+
 int main() {
   int hm0[256];
   for (int i = 0; i < 256; ++i) hm0[i] = (1 << 30) + i * 3000017;
@@ -205,5 +292,29 @@ int main() {
   run_regs<3, true>("regs: float (not exact)", dm0, dclk, dsum);
   run_tmem<1>("tmem: ld16, wait, compute", dm0, dclk, dsum);
   run_tmem<3>("tmem: load of the next piece in flight", dm0, dclk, dsum);
+  // the fp64 form: exact? and does the fp64 pipe add throughput beside the integer pipes?
+  F64Case cases[12 * 13];
+  for (int i = 0; i < 12; ++i)
+    for (int sh = 0; sh <= 12; ++sh) {
+      const int m0 = i == 0 ? 1 << 30 : (i == 1 ? (1 << 30) + 1 : (i == 2 ? 0x7FFFFFFF : hm0[i]));
+      const double ms = ldexp((double)m0, -(32 + sh));
+      cases[i * 13 + sh] = F64Case{m0, sh, ms, 0.5 - 4503601774854144.0 * ms};
+    }
+  F64Case* dcases;
+  cudaMalloc(&dcases, sizeof(cases));
+  cudaMemcpy(dcases, cases, sizeof(cases), cudaMemcpyHostToDevice);
+  cudaMemset(dclk, 0, 8);
+  check_f64<<<(1 << 22) / 256, 256>>>(dcases, 12 * 13, dclk);
+  unsigned long long bad = 1;
+  cudaDeviceSynchronize();
+  cudaMemcpy(&bad, dclk, 8, cudaMemcpyDeviceToHost);
+  printf("fp64 form against the integer form, 2^22 accumulators x 12 multipliers x 13 shifts: %llu mismatches\n", bad);
+  cudaMemcpy(dm0, hm0, sizeof(hm0), cudaMemcpyHostToDevice);
+  uint32_t ref[64] = {0};
+  run_f64<0>("regs: integer form (same loop)", dm0, dclk, dsum, ref);
+  run_f64<16>("regs: fp64 form, all columns", dm0, dclk, dsum, ref);
+  run_f64<4>("regs: 4 of 16 columns fp64", dm0, dclk, dsum, ref);
+  run_f64<8>("regs: 8 of 16 columns fp64", dm0, dclk, dsum, ref);
+  run_f64<12>("regs: 12 of 16 columns fp64", dm0, dclk, dsum, ref);
   return 0;
 }
