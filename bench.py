@@ -193,6 +193,7 @@ def main():
     ap.add_argument("--impl", default="b200")
     ap.add_argument("--config", default="2")
     ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--in-flight", type=int, default=3, help="steps in flight at the same time (streams); 1 = one after the other")
     args = ap.parse_args()
     args.config = int(args.config) if args.config.isdigit() else args.config
     args.batch = args.batch or S.CONFIGS[args.config]["batch"]
@@ -234,9 +235,46 @@ def main():
     # Blocks of `steps` back-to-back encodes, each block between two events; the blocks repeat until
     # the timed region is at least 0.25 s (so that the clock sampler sees it whatever `steps` is).
     # ms_per_step is the median block; the minimum is reported beside it.
-    for i in range(args.warmup):
-        G.iodf_forward(m, xs[i % N_SETS], zs[i % N_SETS], ps[i % N_SETS])
-    G.iodf_check(m)
+    # `--in-flight F` steps run at the same time, each on a stream and a model handle of its own (the
+    # sets of a step's inputs and outputs rotate over N_SETS > F, so steps in flight never share one).
+    # A level's launch is one CTA per image; with several steps in flight the SMs that a batch of 128
+    # leaves idle, and the ends of every level, are filled by the neighbouring steps.
+    F = max(1, min(int(args.in_flight), N_SETS - 1))
+    lanes = [(m, stream)] + [(G.iodf_create(model, B, device=local_rank), torch.cuda.Stream(device=dev)) for _ in range(F - 1)]
+
+    def fork(ev):
+        for _, st in lanes[1:]:
+            st.wait_event(ev)
+
+    def join():
+        for _, st in lanes[1:]:
+            e = torch.cuda.Event()
+            e.record(st)
+            stream.wait_event(e)
+
+    def timed_blocks(nl, blocks, steps):
+        """`blocks` blocks of `steps` encodes dealt round-robin to the first nl lanes; ms of every block"""
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(blocks + 1)]
+        evs[0].record(stream)
+        n = 0
+        for b in range(blocks):
+            if nl > 1:
+                fork(evs[b])
+            for i in range(steps):
+                mk, st = lanes[n % nl]
+                G.iodf_forward(mk, xs[n % N_SETS], zs[n % N_SETS], ps[n % N_SETS], stream=st)
+                n += 1
+            if nl > 1:
+                join()
+            evs[b + 1].record(stream)
+        return evs
+
+    for i in range(max(args.warmup, F)):
+        mk, st = lanes[i % F]
+        G.iodf_forward(mk, xs[i % N_SETS], zs[i % N_SETS], ps[i % N_SETS], stream=st)
+    torch.cuda.synchronize()
+    for mk, _ in lanes:
+        G.iodf_check(mk)
     w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     w0.record(stream)
     for i in range(3):
@@ -249,21 +287,21 @@ def main():
     sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(blocks + 1)]
-    evs[0].record(stream)
-    n = 0
-    for b in range(blocks):
-        for i in range(args.steps):
-            G.iodf_forward(m, xs[n % N_SETS], zs[n % N_SETS], ps[n % N_SETS])
-            n += 1
-        evs[b + 1].record(stream)
+    evs = timed_blocks(F, blocks, args.steps)
     barrier()
     block_ms = sorted(evs[b].elapsed_time(evs[b + 1]) for b in range(blocks))
     total_ms = block_ms[len(block_ms) // 2]          # the median block of `steps` steps
     min_ms = block_ms[0]
     sampler.stop_flag = True
     sampler.join()
-    G.iodf_check(m)
+    for mk, _ in lanes:
+        G.iodf_check(mk)
+    # the same steps one after the other on one stream: the time of a step alone
+    evs = timed_blocks(1, 5, args.steps)
+    barrier()
+    one_ms = sorted(evs[b].elapsed_time(evs[b + 1]) for b in range(5))[2]
+    for mk, _ in lanes[1:]:
+        G.iodf_destroy(mk)
 
     # ---- dominant kernel, timed alone per launch with events on the same stream --------------
     lvl = np.zeros(int(lay.n_levels))
@@ -458,8 +496,36 @@ def main():
     barrier()
     e2e_s = time.perf_counter() - t0
     G.iodf_check(m)
+    # The same with four calls in flight, each on a stream, a model handle and a set of pinned host
+    # buffers of its own, so that a step's device-to-host copy runs under the next steps' uploads and
+    # kernels. Every step still uploads its inputs from pinned host memory, and its result is on the
+    # host before its buffers are reused.
+    E = 4
+    hx += [torch.from_numpy(S.config_images(cfg, batch=B, seed_offset=rank_seed_offset(rank, i))).pin_memory() for i in range(2, E)]
+    hz += [torch.empty((B, m.d), dtype=torch.int32).pin_memory() for _ in range(2, E)]
+    hp += [torch.empty((B, 2, m.d_fact), dtype=torch.int32).pin_memory() for _ in range(2, E)]
+    hlanes = [(m, stream)] + [(G.iodf_create(model, B, device=local_rank), torch.cuda.Stream(device=dev)) for _ in range(E - 1)]
+    for i in range(2 * E):
+        G.iodf_forward_host(hlanes[i % E][0], hx[i % E], hz[i % E], hp[i % E], stream=hlanes[i % E][1])
+    for _, st in hlanes:
+        st.synchronize()
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        mk, st = hlanes[i % E]
+        st.synchronize()          # step i - E of this lane is complete: its result has been read
+        G.iodf_forward_host(mk, hx[i % E], hz[i % E], hp[i % E], stream=st)
+    for _, st in hlanes:
+        st.synchronize()
+    barrier()
+    e2e2_s = time.perf_counter() - t0
+    for mk, _ in hlanes:
+        G.iodf_check(mk)
+    e2e_same = not bool(torch.equal(hz[0], hz[1]))      # the lanes had different inputs: different latents
+    for mk, _ in hlanes[1:]:
+        G.iodf_destroy(mk)
 
-    total_ms, min_ms, e2e_s, dec_ms = max_over_ranks([total_ms, min_ms, e2e_s, dec_ms], world, dev)
+    total_ms, min_ms, one_ms, e2e_s, e2e2_s, dec_ms = max_over_ranks([total_ms, min_ms, one_ms, e2e_s, e2e2_s, dec_ms], world, dev)
 
     if rank == 0:
         cores = os.cpu_count() or 1
@@ -467,12 +533,17 @@ def main():
             "metric": METRIC, "value": job_throughput(B, world, args.steps, total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
             "ms_per_step_min": min_ms / args.steps, "timed_blocks": blocks,
-            "timing": "median over %d blocks of %d steps, each block between CUDA events" % (blocks, args.steps),
+            "timing": "median over %d blocks of %d steps, each block between CUDA events; %d steps in flight (a stream "
+                      "and a model handle each)" % (blocks, args.steps, F),
+            "steps_in_flight": F,
+            "one_step_at_a_time": {"ms_per_step": one_ms / args.steps, "value": job_throughput(B, world, args.steps, one_ms * 1e-3)},
             "ms_per_sample": total_ms / args.steps / B,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-            "config": workload(args), "clocks": sampler.summary(), "roofline": roofline,
-            "e2e": {"value": job_throughput(B, world, e2e_steps, e2e_s), "unit": UNIT, "h2d_bytes_per_step": B * m.d,
-                    "d2h_bytes_per_step": B * m.d * 4 + B * 2 * m.d_fact * 4, "steps": e2e_steps},
+            "config": dict(workload(args), steps_in_flight=F), "clocks": sampler.summary(), "roofline": roofline,
+            "e2e": {"value": job_throughput(B, world, e2e_steps, e2e2_s), "unit": UNIT, "h2d_bytes_per_step": B * m.d,
+                    "d2h_bytes_per_step": B * m.d * 4 + B * 2 * m.d_fact * 4, "steps": e2e_steps,
+                    "how": "iodf_forward_host, pinned host buffers, four calls in flight (a model handle and a stream each)",
+                    "one_call_at_a_time": job_throughput(B, world, e2e_steps, e2e_s), "lanes_distinct": e2e_same},
             "gpu_launches": G.iodf_launches_per_call(m) * args.steps,
             "gpu_launches_all_blocks": G.iodf_launches_per_call(m) * args.steps * blocks,
             "gops_per_image": 2.0 * macs / 1e9,
