@@ -193,7 +193,7 @@ def main():
     ap.add_argument("--impl", default="b200")
     ap.add_argument("--config", default="2")
     ap.add_argument("--batch", type=int, default=None)
-    ap.add_argument("--in-flight", type=int, default=3, help="steps in flight at the same time (streams); 1 = one after the other")
+    ap.add_argument("--in-flight", type=int, default=4, help="steps in flight at the same time (streams); 1 = one after the other")
     args = ap.parse_args()
     args.config = int(args.config) if args.config.isdigit() else args.config
     args.batch = args.batch or S.CONFIGS[args.config]["batch"]
@@ -240,40 +240,41 @@ def main():
     # A level's launch is one CTA per image; with several steps in flight the SMs that a batch of 128
     # leaves idle, and the ends of every level, are filled by the neighbouring steps.
     F = max(1, min(int(args.in_flight), N_SETS - 1))
-    lanes = [(m, stream)] + [(G.iodf_create(model, B, device=local_rank), torch.cuda.Stream(device=dev)) for _ in range(F - 1)]
+    # Handles of steps in flight are made with the throughput plan (fewer CTAs per launch at the deep
+    # levels); `m`, the handle of everything timed one call at a time, with the default plan.
+    lanes = [(m, stream)] if F == 1 else [(G.iodf_create(model, B, device=local_rank, plan=G.IODF_PLAN_THROUGHPUT),
+                                           torch.cuda.Stream(device=dev)) for _ in range(F)]
+    one_lane = [(m, stream)]
 
-    def fork(ev):
-        for _, st in lanes[1:]:
-            st.wait_event(ev)
-
-    def join():
-        for _, st in lanes[1:]:
-            e = torch.cuda.Event()
-            e.record(st)
-            stream.wait_event(e)
-
-    def timed_blocks(nl, blocks, steps):
-        """`blocks` blocks of `steps` encodes dealt round-robin to the first nl lanes; ms of every block"""
+    def timed_blocks(ln, blocks, steps):
+        """`blocks` blocks of `steps` encodes dealt round-robin to the lanes `ln`; the events between blocks
+        (on the main stream, which every lane's stream waits for before a block and is waited for after it)"""
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(blocks + 1)]
         evs[0].record(stream)
         n = 0
         for b in range(blocks):
-            if nl > 1:
-                fork(evs[b])
+            for _, st in ln:
+                if st is not stream:
+                    st.wait_event(evs[b])
             for i in range(steps):
-                mk, st = lanes[n % nl]
+                mk, st = ln[n % len(ln)]
                 G.iodf_forward(mk, xs[n % N_SETS], zs[n % N_SETS], ps[n % N_SETS], stream=st)
                 n += 1
-            if nl > 1:
-                join()
+            for _, st in ln:
+                if st is not stream:
+                    e = torch.cuda.Event()
+                    e.record(st)
+                    stream.wait_event(e)
             evs[b + 1].record(stream)
         return evs
 
     for i in range(max(args.warmup, F)):
         mk, st = lanes[i % F]
         G.iodf_forward(mk, xs[i % N_SETS], zs[i % N_SETS], ps[i % N_SETS], stream=st)
+    for i in range(args.warmup):
+        G.iodf_forward(m, xs[i % N_SETS], zs[i % N_SETS], ps[i % N_SETS])
     torch.cuda.synchronize()
-    for mk, _ in lanes:
+    for mk, _ in lanes + one_lane:
         G.iodf_check(mk)
     w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     w0.record(stream)
@@ -287,7 +288,7 @@ def main():
     sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
-    evs = timed_blocks(F, blocks, args.steps)
+    evs = timed_blocks(lanes, blocks, args.steps)
     barrier()
     block_ms = sorted(evs[b].elapsed_time(evs[b + 1]) for b in range(blocks))
     total_ms = block_ms[len(block_ms) // 2]          # the median block of `steps` steps
@@ -297,11 +298,12 @@ def main():
     for mk, _ in lanes:
         G.iodf_check(mk)
     # the same steps one after the other on one stream: the time of a step alone
-    evs = timed_blocks(1, 5, args.steps)
+    evs = timed_blocks(one_lane, 5, args.steps)
     barrier()
     one_ms = sorted(evs[b].elapsed_time(evs[b + 1]) for b in range(5))[2]
-    for mk, _ in lanes[1:]:
-        G.iodf_destroy(mk)
+    for mk, _ in lanes:
+        if mk is not m:
+            G.iodf_destroy(mk)
 
     # ---- dominant kernel, timed alone per launch with events on the same stream --------------
     lvl = np.zeros(int(lay.n_levels))
@@ -504,7 +506,8 @@ def main():
     hx += [torch.from_numpy(S.config_images(cfg, batch=B, seed_offset=rank_seed_offset(rank, i))).pin_memory() for i in range(2, E)]
     hz += [torch.empty((B, m.d), dtype=torch.int32).pin_memory() for _ in range(2, E)]
     hp += [torch.empty((B, 2, m.d_fact), dtype=torch.int32).pin_memory() for _ in range(2, E)]
-    hlanes = [(m, stream)] + [(G.iodf_create(model, B, device=local_rank), torch.cuda.Stream(device=dev)) for _ in range(E - 1)]
+    hlanes = [(G.iodf_create(model, B, device=local_rank, plan=G.IODF_PLAN_THROUGHPUT), torch.cuda.Stream(device=dev))
+              for _ in range(E)]
     for i in range(2 * E):
         G.iodf_forward_host(hlanes[i % E][0], hx[i % E], hz[i % E], hp[i % E], stream=hlanes[i % E][1])
     for _, st in hlanes:
@@ -522,7 +525,7 @@ def main():
     for mk, _ in hlanes:
         G.iodf_check(mk)
     e2e_same = not bool(torch.equal(hz[0], hz[1]))      # the lanes had different inputs: different latents
-    for mk, _ in hlanes[1:]:
+    for mk, _ in hlanes:
         G.iodf_destroy(mk)
 
     total_ms, min_ms, one_ms, e2e_s, e2e2_s, dec_ms = max_over_ranks([total_ms, min_ms, one_ms, e2e_s, e2e2_s, dec_ms], world, dev)
@@ -534,7 +537,7 @@ def main():
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
             "ms_per_step_min": min_ms / args.steps, "timed_blocks": blocks,
             "timing": "median over %d blocks of %d steps, each block between CUDA events; %d steps in flight (a stream "
-                      "and a model handle each)" % (blocks, args.steps, F),
+                      "and a model handle, made with the throughput plan, each)" % (blocks, args.steps, F),
             "steps_in_flight": F,
             "one_step_at_a_time": {"ms_per_step": one_ms / args.steps, "value": job_throughput(B, world, args.steps, one_ms * 1e-3)},
             "ms_per_sample": total_ms / args.steps / B,

@@ -34,7 +34,7 @@
 extern "C" {
 #endif
 
-#define IODF_ABI_VERSION 2u
+#define IODF_ABI_VERSION 3u
 
 typedef enum {
   IODF_OK = 0,
@@ -123,12 +123,25 @@ typedef struct {
   int32_t ls_lo, ls_hi;
 } iodf_level_desc;
 
+/* How the levels whose images are smaller than a 128-pixel tile are shared out over CTAs (the
+ * results are the same bit for bit; only the launch shapes differ):
+ *   IODF_PLAN_LATENCY     as few images per CTA as keeps the SMs busy with one batch of max_batch
+ *                         images: the shortest step
+ *   IODF_PLAN_THROUGHPUT  as many images per CTA as a tile holds with the level's weights still
+ *                         resident in shared memory: fewer CTAs per launch, a step a few percent
+ *                         longer; for callers that keep several batches in flight, each on a stream
+ *                         and a model handle of its own, so that one batch's idle SMs run another's CTAs
+ */
+#define IODF_PLAN_LATENCY 0u
+#define IODF_PLAN_THROUGHPUT 1u
+
 typedef struct {
   uint32_t abi_version;                /* IODF_ABI_VERSION                                           */
   uint32_t in_c, in_h, in_w;           /* image shape; in_h, in_w divisible by 2^n_levels            */
   uint32_t n_levels;
   uint32_t max_batch;                  /* workspace is sized for this batch at create                */
   const iodf_level_desc* levels;       /* HOST                                                       */
+  uint32_t plan;                       /* IODF_PLAN_LATENCY or IODF_PLAN_THROUGHPUT (else EINVAL)    */
 } iodf_model_desc;
 
 #define IODF_MAX_LEVELS 8

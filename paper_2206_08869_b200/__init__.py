@@ -2,7 +2,8 @@
 include/iodf.h. PyTorch supplies device memory and streams; every step of the flow runs in the
 library's CUDA kernels. There is no CPU path: loading fails if the library has not been built."""
 from .binding import (IodfError, Model, iodf_create, iodf_destroy, iodf_forward, iodf_inverse,
-                      iodf_inverse_level, IODF_LEVEL_PRIOR, IODF_LEVEL_COUPLINGS, iodf_forward_patches,
+                      iodf_inverse_level, IODF_LEVEL_PRIOR, IODF_LEVEL_COUPLINGS, IODF_PLAN_LATENCY,
+                      IODF_PLAN_THROUGHPUT, iodf_forward_patches,
                       iodf_inverse_patches, Codec, iodf_codec_create, iodf_rans_encode, iodf_rans_decode_block,
                       iodf_codec_check, iodf_rans_packed_capacity, iodf_rans_pack, iodf_rans_unpack,
                       iodf_compress_host, iodf_decompress_host,
@@ -14,7 +15,8 @@ from .binding import (IodfError, Model, iodf_create, iodf_destroy, iodf_forward,
                       DECLARED_SYMBOLS)
 
 __all__ = ["IodfError", "Model", "iodf_create", "iodf_destroy", "iodf_forward", "iodf_inverse",
-           "iodf_inverse_level", "IODF_LEVEL_PRIOR", "IODF_LEVEL_COUPLINGS", "iodf_forward_patches",
+           "iodf_inverse_level", "IODF_LEVEL_PRIOR", "IODF_LEVEL_COUPLINGS", "IODF_PLAN_LATENCY",
+           "IODF_PLAN_THROUGHPUT", "iodf_forward_patches",
            "iodf_inverse_patches", "Codec", "iodf_codec_create", "iodf_rans_encode", "iodf_rans_decode_block",
            "iodf_codec_check", "iodf_rans_packed_capacity", "iodf_rans_pack", "iodf_rans_unpack",
            "iodf_compress_host", "iodf_decompress_host",

@@ -8,7 +8,8 @@ import numpy as np
 
 from . import build as _build
 
-IODF_ABI_VERSION = 2
+IODF_ABI_VERSION = 3
+IODF_PLAN_LATENCY, IODF_PLAN_THROUGHPUT = 0, 1
 IODF_MAX_LEVELS = 8
 
 DECLARED_SYMBOLS = ["iodf_create", "iodf_destroy", "iodf_get_layout", "iodf_forward", "iodf_inverse",
@@ -47,7 +48,8 @@ class LevelDesc(C.Structure):
 
 class ModelDesc(C.Structure):
     _fields_ = [("abi_version", C.c_uint32), ("in_c", C.c_uint32), ("in_h", C.c_uint32), ("in_w", C.c_uint32),
-                ("n_levels", C.c_uint32), ("max_batch", C.c_uint32), ("levels", C.POINTER(LevelDesc))]
+                ("n_levels", C.c_uint32), ("max_batch", C.c_uint32), ("levels", C.POINTER(LevelDesc)),
+                ("plan", C.c_uint32)]
 
 
 class Layout(C.Structure):
@@ -168,7 +170,7 @@ def iodf_strerror(status):
 class _Marshalled:
     """C descriptor structs for a model dict, with every referenced array kept alive."""
 
-    def __init__(self, model, max_batch):
+    def __init__(self, model, max_batch, plan=0):
         self.keep = []
         wts, par = [], []
         self.woff = self.poff = 0
@@ -216,7 +218,7 @@ class _Marshalled:
                 levels[li].ls_lo, levels[li].ls_hi = hd["ls_lo"], hd["ls_hi"]
         self.levels = levels
         self.desc = ModelDesc(IODF_ABI_VERSION, model["in_c"], model["in_h"], model["in_w"], len(model["levels"]),
-                              int(max_batch), levels)
+                              int(max_batch), levels, int(plan))
         self.wts = np.concatenate(wts) if wts else np.zeros(1, np.int8)
         self.par = np.concatenate(par) if par else np.zeros(1, np.int32)
 
@@ -234,9 +236,11 @@ class Model:
             _lib.iodf_destroy(h)
 
 
-def iodf_create(model, max_batch, device=0, marshalled=None):
+def iodf_create(model, max_batch, device=0, marshalled=None, plan=IODF_PLAN_LATENCY):
+    """plan: IODF_PLAN_LATENCY (the shortest step) or IODF_PLAN_THROUGHPUT (fewer CTAs per launch, for
+    several batches in flight on streams and handles of their own); see include/iodf.h."""
     L = load_library()
-    m = marshalled or _Marshalled(model, max_batch)
+    m = marshalled or _Marshalled(model, max_batch, plan)
     out = C.c_void_p()
     rc = L.iodf_create(C.byref(m.desc), m.wts.ctypes.data, m.wts.size, m.par.ctypes.data, m.par.size, int(device),
                        C.byref(out))

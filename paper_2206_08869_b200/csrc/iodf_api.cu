@@ -349,13 +349,15 @@ struct PipeDims {
 //   mode 3: one tile slot, weights streamed per tile in 32-byte K-slices through a small ring
 //           (the only mode for hidden widths above 256: a 512 x 512 matrix alone is 256 KB)
 bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32_t wmax[3], uint32_t n_max,
-               uint32_t limit, uint32_t max_batch, int num_sms, const PipeDims& pd) {
+               uint32_t limit, uint32_t max_batch, int num_sms, const PipeDims& pd, bool throughput) {
   int group = P.px >= kTileM ? 1 : kTileM / P.px;
   group = std::max(1, std::min<int>(group, (int)max_batch));
   // A level's time is set by the serial chain of its couplings inside one CTA, not by how many
   // rows of the 128-row tile are filled: while the CTAs of a full batch would not fill the SMs,
-  // smaller groups (more CTAs, emptier tiles) are faster.
-  while (group > 1 && ((int)max_batch + group - 1) / group < num_sms) group /= 2;
+  // smaller groups (more CTAs, emptier tiles) are faster. The throughput plan keeps the tile as
+  // full as the resident-weight modes allow instead: the step is a little longer, but a launch takes
+  // a half to a quarter of the CTAs, which leaves SMs to the other batches a caller has in flight.
+  while (!throughput && group > 1 && ((int)max_batch + group - 1) / group < num_sms) group /= 2;
   for (; group >= 1; group = (group > 1 ? group / 2 : 0)) {
     const int tiles = (group * P.px + kTileM - 1) / kTileM;
     // the role-split kernel first with im2col buffers of its own (mode -2), then sharing the slot's buffer (-1)
@@ -367,6 +369,7 @@ bool plan_smem(LevelPlan& P, uint32_t a_bytes, uint32_t meta_bytes, const uint32
       if (mode == 0 && (tiles < 2 || n_max > (uint32_t)kSlotCols)) continue;
       if (mode >= 0 && mode < 3 && n_max > 2u * kSlotCols) continue;
       if (mode == 3 && n_max <= (uint32_t)kSlotCols) continue;   // resident weights are faster when they fit
+      if (mode == 3 && throughput && group > 1) continue;        // streamed weights cost more than the fuller tile saves
       const uint32_t pg = up((uint32_t)group * P.px, 32);
       uint32_t off = 0;
       auto take = [&](uint32_t bytes) { uint32_t o = off; off = up(off + bytes, kAlign); return o; };
@@ -601,7 +604,7 @@ int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P,
 int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_model* m) {
   if (desc->abi_version != IODF_ABI_VERSION) return IODF_EVERSION;
   if (!desc->levels || desc->n_levels < 1 || desc->n_levels > IODF_MAX_LEVELS || desc->max_batch < 1 ||
-      desc->in_c < 1 || desc->in_h < 1 || desc->in_w < 1)
+      desc->in_c < 1 || desc->in_h < 1 || desc->in_w < 1 || desc->plan > IODF_PLAN_THROUGHPUT)
     return IODF_EINVAL;
   if ((desc->in_h % (1u << desc->n_levels)) || (desc->in_w % (1u << desc->n_levels))) return IODF_EINVAL;
   m->device = device;
@@ -804,7 +807,8 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
       wmax[0] = std::max(wmax[0], P.prior.w_bytes[0]);
     }
     if (hl.blob.empty()) hl.blob.resize(kAlign, 0);
-    if (!plan_smem(P, a_bytes, meta, wmax, n_max, (uint32_t)smem_limit, desc->max_batch, num_sms, pd))
+    if (!plan_smem(P, a_bytes, meta, wmax, n_max, (uint32_t)smem_limit, desc->max_batch, num_sms, pd,
+                   desc->plan == IODF_PLAN_THROUGHPUT))
       return IODF_EUNSUPPORTED;
     // the index maps divide numbers below group * c * px by at most c * px with a 32-bit magic multiplier
     if ((uint64_t)P.group * c * h * w * ((uint64_t)c * h * w) >= (1ull << 32)) return IODF_EUNSUPPORTED;

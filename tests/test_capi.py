@@ -86,6 +86,11 @@ def test_bad_descriptors_fail_on_the_host():
     with pytest.raises(G.IodfError) as e:
         G.iodf_create(_small(), 4, marshalled=mm)
     assert e.value.status == EVERSION
+    # a plan the library does not know
+    mm = binding._Marshalled(_small(), 4, plan=7)
+    with pytest.raises(G.IodfError) as e:
+        G.iodf_create(_small(), 4, marshalled=mm)
+    assert e.value.status == EINVAL
     # offsets beyond the blobs
     mm = binding._Marshalled(_small(), 4)
     mm.wts = mm.wts[:10].copy()

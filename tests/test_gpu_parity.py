@@ -21,7 +21,7 @@ def _t(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def _check_both_ways(G, model, x, max_batch=None, sample=None):
+def _check_both_ways(G, model, x, max_batch=None, sample=None, plan=0):
     """Encode x on the GPU and compare with the oracle (all images, or the `sample` indices);
     decode the oracle's z on the GPU and compare with x."""
     import torch
@@ -29,7 +29,7 @@ def _check_both_ways(G, model, x, max_batch=None, sample=None):
     pk = O.Packed(model)
     idx = np.arange(B) if sample is None else np.asarray(sample)
     z_ref, p_ref = O.forward(pk, x[idx])
-    m = G.iodf_create(model, max_batch or B)
+    m = G.iodf_create(model, max_batch or B, plan=plan)
     z, p = G.iodf_forward(m, _t(x))
     G.iodf_check(m)
     zc = z.cpu().numpy()
@@ -213,6 +213,48 @@ def test_host_buffer_entry_points(G):
 
 
 # ---- the five benchmark configurations ------------------------------------------------------------
+# ---- the throughput plan: as many images per CTA as a tile holds -----------------------------------
+@pytest.mark.parametrize("hw,splits,hidden,prune,batch", [
+    (8, [True, True], 24, (0.4, 0.7), 21),       # 16- and 4-px levels: 8 and 32 images per CTA, ragged last CTAs
+    (16, [True, True, True], 40, (0.4, 0.7), 37),# 64-, 16- and 4-px levels
+    (12, [True, False], 20, (0.4, 0.7), 50),     # 36- and 9-px levels: images that do not divide the tile
+    (16, [True, True], 320, None, 9),            # hidden width above 256: streamed weights only at one image per CTA
+])
+def test_throughput_plan_small_models_bit_exact(G, hw, splits, hidden, prune, batch):
+    model = S.make_model(300 + hw, 3, hw, hw, splits, 3, hidden, prune=prune)
+    x = S.smooth_field_images(400 + hw, batch, hw, hw, 1.5)
+    _check_both_ways(G, model, x, plan=G.IODF_PLAN_THROUGHPUT)
+
+
+def test_throughput_plan_config2_equals_the_latency_plan(G):
+    """The benchmark keeps several batches in flight on handles made with the throughput plan: same
+    latents and prior parameters as the oracle on sampled images, as the default plan on all, exact
+    round trip, and three handles running at the same time on three streams give the same again."""
+    import torch
+    x = S.config_images(2)
+    B = x.shape[0]
+    pick = sorted(set([0, 1, B // 2, B - 1] + S.Stream(6, "pick").integers(0, B, 8).tolist()))
+    model = S.config_model(2)
+    m, z = _check_both_ways(G, model, x, sample=pick, plan=G.IODF_PLAN_THROUGHPUT)
+    m0 = G.iodf_create(model, B)
+    z0, p0 = G.iodf_forward(m0, _t(x))
+    G.iodf_check(m0)
+    np.testing.assert_array_equal(z0.cpu().numpy(), z)
+    lanes = [(m, torch.cuda.Stream())] + [(G.iodf_create(model, B, plan=G.IODF_PLAN_THROUGHPUT), torch.cuda.Stream())
+                                          for _ in range(2)]
+    xs = [_t(np.ascontiguousarray(np.roll(x, k, axis=0))) for k in range(3)]
+    outs = [(torch.empty_like(z0), torch.empty_like(p0)) for _ in lanes]      # a lane's own buffers, reused
+    torch.cuda.synchronize()
+    for rep in range(4):
+        for k, (mk, st) in enumerate(lanes):
+            G.iodf_forward(mk, xs[k], outs[k][0], outs[k][1], stream=st)
+    torch.cuda.synchronize()
+    for k, (mk, _) in enumerate(lanes):
+        G.iodf_check(mk)
+        np.testing.assert_array_equal(outs[k][0].cpu().numpy(), np.roll(z, k, axis=0))
+        assert torch.equal(outs[k][1], torch.roll(p0, k, dims=0))
+
+
 def test_config0_tiny_flow(G):
     _check_both_ways(G, S.config_model(0), S.config_images(0))
 
