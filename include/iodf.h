@@ -128,9 +128,11 @@ typedef struct {
  *   IODF_PLAN_LATENCY     as few images per CTA as keeps the SMs busy with one batch of max_batch
  *                         images: the shortest step
  *   IODF_PLAN_THROUGHPUT  as many images per CTA as a tile holds with the level's weights still
- *                         resident in shared memory: fewer CTAs per launch, a step a few percent
- *                         longer; for callers that keep several batches in flight, each on a stream
- *                         and a model handle of its own, so that one batch's idle SMs run another's CTAs
+ *                         resident in shared memory (levels with residual-block couplings: as many
+ *                         padded frames (h+2)(w+2) as a tile holds): fewer CTAs per launch, a step a
+ *                         few percent longer; for callers that keep several batches in flight, each on
+ *                         a stream and a model handle of its own, so that one batch's idle SMs run
+ *                         another's CTAs
  */
 #define IODF_PLAN_LATENCY 0u
 #define IODF_PLAN_THROUGHPUT 1u

@@ -478,7 +478,8 @@ int check_residual(const iodf_coupling_desc& cp, const Blobs& B, uint32_t ca, ui
 
 // Level blob of a residual level: ResHead, coupling records, conv records, then tables and weights.
 int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P, std::vector<uint8_t>& blob,
-                        const std::vector<std::vector<int>>& cols, uint32_t smem_limit) {
+                        const std::vector<std::vector<int>>& cols, uint32_t smem_limit, uint32_t max_batch,
+                        bool throughput) {
   const int ca = P.ca, cb = P.cb, px = P.px;
   std::vector<ResCouplingRec> cps(lv.n_couplings);
   std::vector<ResConv> convs;
@@ -568,25 +569,34 @@ int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P,
   if (bands == 0) return IODF_EUNSUPPORTED;
   const int hb = P.h / bands;
   (void)px;
-  const uint32_t pg = up((uint32_t)(hb * P.w), 32);
   const int w2 = P.w + 2, guard = w2 + 1;
-  const int ntiles = (int)(up((uint32_t)((hb + 2) * w2), kTileM) / kTileM);
-  const int rows = guard + ntiles * kTileM + w2 + 1;
+  // images per CTA: one, or (throughput plan, whole images) as many frames as one tile holds and as
+  // leave the weight ring two slots
+  int group = 1;
+  if (throughput && bands == 1) group = std::max(1, std::min<int>(kTileM / ((hb + 2) * w2), (int)max_batch));
+  uint32_t pg = 0, off = 0;
+  int ntiles = 0, rows = 0;
+  for (;; --group) {
+    pg = up((uint32_t)(group * hb * P.w), 32);
+    ntiles = (int)(up((uint32_t)(group * (hb + 2) * w2), kTileM) / kTileM);
+    rows = guard + ntiles * kTileM + w2 + 1;
+    off = 0;
+    auto take = [&](uint32_t bytes) { uint32_t o = off; off = up(off + bytes, kAlign); return o; };
+    H.s_v = take((uint32_t)P.c * pg * 4);
+    H.s_xa = take((uint32_t)(H.xa_pitch / 16) * rows * 16);
+    H.s_x = take((uint32_t)(H.x_pitch / 16) * rows * 16);
+    H.s_mid = take((uint32_t)(H.mid_pitch / 16) * rows * 16);
+    H.s_rowinfo = take((uint32_t)ntiles * kTileM * 8);     // pixel and edge-row tables
+    H.s_tab = take((uint32_t)kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t)) + 256);   // + the shortcut table
+    // as deep a weight ring as fits (at least two slots)
+    H.w_slot_bytes = up((uint32_t)nmax * kmax, kAlign);
+    H.n_wslots = kResMaxWSlots;
+    while (H.n_wslots > 2 && off + (uint32_t)H.n_wslots * H.w_slot_bytes > smem_limit) --H.n_wslots;
+    H.s_wring = take((uint32_t)H.n_wslots * H.w_slot_bytes);
+    if (off <= smem_limit || group == 1) break;
+  }
   H.w2 = w2; H.guard = guard; H.rows = rows; H.ntiles = ntiles;
-  H.bands = bands; H.hb = hb;
-  uint32_t off = 0;
-  auto take = [&](uint32_t bytes) { uint32_t o = off; off = up(off + bytes, kAlign); return o; };
-  H.s_v = take((uint32_t)P.c * pg * 4);
-  H.s_xa = take((uint32_t)(H.xa_pitch / 16) * rows * 16);
-  H.s_x = take((uint32_t)(H.x_pitch / 16) * rows * 16);
-  H.s_mid = take((uint32_t)(H.mid_pitch / 16) * rows * 16);
-  H.s_rowinfo = take((uint32_t)ntiles * kTileM * 8);     // pixel and edge-row tables
-  H.s_tab = take((uint32_t)kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t)) + 256);   // + the shortcut table
-  // as deep a weight ring as fits (at least two slots)
-  H.w_slot_bytes = up((uint32_t)nmax * kmax, kAlign);
-  H.n_wslots = kResMaxWSlots;
-  while (H.n_wslots > 2 && off + (uint32_t)H.n_wslots * H.w_slot_bytes > smem_limit) --H.n_wslots;
-  H.s_wring = take((uint32_t)H.n_wslots * H.w_slot_bytes);
+  H.bands = bands; H.hb = hb; H.group = group;
   H.s_total = off;
   // one tile: every issuing warp keeps a partial accumulator of its own
   H.tmem_cols = (ntiles > 2 || ntiles == 1) ? 4 * kResMaxWidth : 2 * kResMaxWidth;
@@ -596,7 +606,7 @@ int pack_residual_level(const iodf_level_desc& lv, const Blobs& B, LevelPlan& P,
   std::memcpy(blob.data() + H.conv_off, convs.data(), sizeof(ResConv) * convs.size());
   P.residual = 1;
   P.res_bands = bands;
-  P.group = 1; P.pg = (int)pg; P.tiles = ntiles; P.rep = 1; P.nslots = 1;
+  P.group = group; P.pg = (int)pg; P.tiles = ntiles; P.rep = 1; P.nslots = 1;
   P.s_total = H.s_total;
   return IODF_OK;
 }
@@ -741,9 +751,10 @@ int build_model(const iodf_model_desc* desc, const Blobs& B, int device, iodf_mo
         cols.push_back(pi);
       }
       for (int k = 0; k < (int)c; ++k) P.col_out[k] = pi[k];
-      int rc = pack_residual_level(lv, B, P, hl.blob, cols, (uint32_t)smem_limit);
+      int rc = pack_residual_level(lv, B, P, hl.blob, cols, (uint32_t)smem_limit, desc->max_batch,
+                                   desc->plan == IODF_PLAN_THROUGHPUT);
       if (rc) return rc;
-      if ((uint64_t)c * h * w * ((uint64_t)c * h * w) >= (1ull << 32)) return IODF_EUNSUPPORTED;
+      if ((uint64_t)P.group * c * h * w * ((uint64_t)c * h * w) >= (1ull << 32)) return IODF_EUNSUPPORTED;
       if (lv.split) c = (uint32_t)ca;
       continue;
     }
@@ -860,7 +871,7 @@ void set_patch_grid(LevelArgs& a, const PatchGrid& g) {
 // The kernel that runs a level: residual couplings, the stage pipeline, or the general kernel.
 cudaError_t launch_any_level(const LevelPlan& P, const LevelArgs& a, bool inverse, int B, cudaStream_t st) {
   const int grid = (B + P.group - 1) / P.group;
-  if (P.residual) return launch_res_level(a, inverse, B, P.res_bands, P.s_total, st);
+  if (P.residual) return launch_res_level(a, inverse, grid, P.res_bands, P.s_total, st);
   if (P.pipe) return launch_level_pipe(a, inverse, grid, P.s_total, st);
   return launch_level(a, inverse, P.lean != 0, grid, P.s_total, st);
 }

@@ -134,7 +134,19 @@ struct Run {
   int bands, band;          // row bands of the image (CTAs of the cluster) and this CTA's
   int px_full;              // pixels of the whole image at this level (strides of the global layouts)
   int q0;                   // the band's first pixel
+  // several images per CTA (bands = 1): their frames follow one another in the padded layout, their
+  // pixels in the flow variable's planes (pixel index = image * px + pixel of the image)
+  int nimg, frame, ptot;    // images of this CTA, padded positions per image, pixels of all its images
+  uint32_t mul_px;          // magic multiplier of px
+  size_t prior_img_stride;  // prior parameters: elements between two images
 };
+
+// padded position (0 = first computed position) of pixel p of the CTA (image-major)
+__device__ __forceinline__ int position_of(const Run& r, int p) {
+  const int g = r.nimg > 1 ? rdiv(p, r.mul_px) : 0, q = p - g * r.g.px;
+  const int i = rdiv(q, r.g.mul_w), j = q - i * r.g.w;
+  return g * r.frame + (i + 1) * r.H->w2 + (j + 1);
+}
 
 // End of a step that wrote activations: they must be visible to the tensor core's reads (this CTA's
 // and, for edge rows, the neighbours') before the next conv is issued.
@@ -281,11 +293,10 @@ __device__ void conv_mma(Run& r, const ResConv& c, const ResConv* next, const in
     // being multiplied: its MMAs read MID, and the block's first conv has read X already.
     uint8_t* X = r.smem + r.H->s_x;
     const uint8_t* lut = r.smem + r.H->s_tab + kResMaxWidth * (sizeof(OutRq) + sizeof(int32_t));
-    const int chunks = r.H->x_pitch >> 4, px = r.g.px;
+    const int chunks = r.H->x_pitch >> 4, px = r.ptot;
     for (int it = r.tid; it < chunks * px; it += kResThreads) {
       const int ch = it / px, p = it - ch * px;
-      const int pi = rdiv(p, r.g.mul_w), pj = p - pi * r.g.w;
-      const int rr = (pi + 1) * r.H->w2 + (pj + 1);
+      const int rr = position_of(r, p);
       uint4* wp = reinterpret_cast<uint4*>(at(r, X, ch * 16, rr));
       uint4 val = *wp;
       uint32_t* wv = reinterpret_cast<uint32_t*>(&val);
@@ -393,8 +404,10 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
             *vv = io.subtract ? (*vv - (uint32_t)y) : (*vv + (uint32_t)y);
           } else {   // kResPrior: first half mu, second half the clipped log-scale index
             const int half = c.n >> 1;
-            if (col < half) io.mu[(size_t)col * r.px_full + p] = y;
-            else io.ls[(size_t)(col - half) * r.px_full + p] = clampi(y, io.ls_lo, io.ls_hi);
+            const int g = r.nimg > 1 ? rdiv(p, r.mul_px) : 0;          // image of the CTA, pixel of the image
+            const size_t at_px = (size_t)g * r.prior_img_stride + (size_t)(p - g * r.g.px);
+            if (col < half) io.mu[(size_t)col * r.px_full + at_px] = y;
+            else io.ls[(size_t)(col - half) * r.px_full + at_px] = clampi(y, io.ls_lo, io.ls_hi);
           }
         }
       }
@@ -407,10 +420,9 @@ __device__ void conv_epilogue(Run& r, const ResConv& c, const StepIo& io) {
 // image's positions of the padded layout
 __device__ void requant_input(Run& r, const int32_t* cols, int n, int32_t m0, int32_t s) {
   uint8_t* xa = r.smem + r.H->s_xa;
-  for (int it = r.tid; it < (r.warp < kResBuilderWarps ? n * r.g.px : 0); it += kResThreads) {
-    const int c = it / r.g.px, p = it - c * r.g.px;
-    const int i = rdiv(p, r.g.mul_w), j = p - i * r.g.w;
-    const int rr = (i + 1) * r.H->w2 + (j + 1);
+  for (int it = r.tid; it < (r.warp < kResBuilderWarps ? n * r.ptot : 0); it += kResThreads) {
+    const int c = it / r.ptot, p = it - c * r.ptot;
+    const int rr = position_of(r, p);
     const uint32_t byte = (uint32_t)(uint8_t)(int8_t)clampi(rq64(r.v[cols[c] * r.g.pg + p], m0, s), -128, 127);
     *at(r, xa, c, rr) = (uint8_t)byte;
     if (r.bands > 1) mirror1(r, xa, c, rr, byte);
@@ -444,10 +456,13 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
   // one CTA per image, or per band of rows of an image (the CTAs of a cluster)
   const int bands = H->bands, hb = H->hb;
   const int band = bands > 1 ? (int)cluster_rank() : 0;
-  const int b = blockIdx.x / bands;               // image
+  const int group = bands > 1 ? 1 : H->group;     // images per CTA
+  const int b = (blockIdx.x / bands) * group;     // (first) image
+  const int nimg = min(group, a.batch - b);
   const int w = P.w, pg = P.pg, c = P.c;
-  const int pxb = hb * w;                         // pixels of the band
+  const int pxb = hb * w;                         // pixels of the band (of an image)
   const int q0 = band * pxb;                      // the band's first pixel in the image
+  const int frame = (hb + 2) * H->w2;             // padded positions of an image
 
   Run r;
   r.smem = smem; r.ctl = &ctl; r.status = a.status; r.blob = a.blob; r.H = H;
@@ -465,14 +480,18 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
   r.pixel_of = pixel_of;
   r.halo_of = halo_of;
   r.bands = bands; r.band = band; r.px_full = P.px; r.q0 = q0;
+  r.nimg = nimg; r.frame = frame; r.ptot = nimg * pxb; r.mul_px = P.mul_px;
+  r.prior_img_stride = (size_t)2 * P.d_fact;
 
   const bool builder = warp < kResBuilderWarps;
-  const int per_band = builder ? c * pxb : 0;     // the issuing warps take no part in the element loops
+  const int per_band = c * pxb;                   // elements of an image's band
+  const int n_el = builder ? nimg * per_band : 0; // the issuing warps take no part in the element loops
   int32_t* v = r.v;
   for (int rr = tid; rr < (builder ? r.ntiles * kTileM : 0); rr += kResThreads) {
-    const int i = rr / H->w2, j = rr - i * H->w2;          // position (i, j) of the (hb+2) x (w+2) frame
-    const bool own = i >= 1 && i <= hb && j >= 1 && j <= w;
-    pixel_of[rr] = own ? (i - 1) * w + (j - 1) : -1;
+    const int g = rr / frame, r0 = rr - g * frame;         // image of the CTA, position in its frame
+    const int i = r0 / H->w2, j = r0 - i * H->w2;          // position (i, j) of the (hb+2) x (w+2) frame
+    const bool own = g < nimg && i >= 1 && i <= hb && j >= 1 && j <= w;
+    pixel_of[rr] = own ? g * pxb + (i - 1) * w + (j - 1) : -1;
     // the band's first row is the row below the band above's last one, and the other way round
     int hrec = 0;
     if (own && i == 1 && band > 0) hrec = ((rr + hb * H->w2) << 1) | 0;
@@ -489,27 +508,29 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
   const int px = P.px;
   if (!kInv) {
     const int w2 = 2 * w, rows2 = 2 * hb;
-    for (int e = tid; e < per_band; e += kResThreads) {
+    for (int e0 = tid; e0 < n_el; e0 += kResThreads) {
+      const int g = e0 / per_band, e = e0 - g * per_band, bi = b + g;      // image of the CTA, element of the image
       const int ci = e / (rows2 * w2), r2 = e - ci * rows2 * w2;
       const int y = r2 / w2, x = r2 - y * w2;
       const int gy = 2 * band * hb + y;                    // row of the whole pre-squeeze image
-      size_t src = ((size_t)b * (c / 4) + ci) * (size_t)(4 * px) + (size_t)gy * w2 + x;
+      size_t src = ((size_t)bi * (c / 4) + ci) * (size_t)(4 * px) + (size_t)gy * w2 + x;
       if (P.is_first && a.img_w > 0) {
-        const int by = rdiv(b, a.mul_patches_x), bx = b - by * a.patches_x;
+        const int by = rdiv(bi, a.mul_patches_x), bx = bi - by * a.patches_x;
         src = ((size_t)ci * a.img_h + (size_t)(by * 2 * P.h + gy)) * a.img_w + (size_t)(bx * w2 + x);
       }
       const int32_t val = P.is_first ? (int32_t) reinterpret_cast<const uint8_t*>(a.in)[src]
                                      : reinterpret_cast<const int32_t*>(a.in)[src];
-      v[(ci * 4 + (y & 1) * 2 + (x & 1)) * pg + (y >> 1) * w + (x >> 1)] = val;
+      v[(ci * 4 + (y & 1) * 2 + (x & 1)) * pg + g * pxb + (y >> 1) * w + (x >> 1)] = val;
     }
   } else {
-    for (int e = tid; e < per_band; e += kResThreads) {
+    for (int e0 = tid; e0 < n_el; e0 += kResThreads) {
+      const int g = e0 / per_band, e = e0 - g * per_band, bi = b + g;
       const int k = e / pxb, q = e - k * pxb;
       if (a.phase == 1 && k >= P.keep_c) continue;
       const int32_t val =
-          (k < P.keep_c) ? reinterpret_cast<const int32_t*>(a.in)[(size_t)b * (size_t)a.in_stride + (size_t)k * px + q0 + q]
-                         : a.z[(size_t)b * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q0 + q];
-      v[P.col_out[k] * pg + q] = val;
+          (k < P.keep_c) ? reinterpret_cast<const int32_t*>(a.in)[(size_t)bi * (size_t)a.in_stride + (size_t)k * px + q0 + q]
+                         : a.z[(size_t)bi * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q0 + q];
+      v[P.col_out[k] * pg + g * pxb + q] = val;
     }
   }
   // nobody writes into a neighbour's edge rows before that neighbour has cleared its buffers
@@ -549,24 +570,26 @@ __global__ void __launch_bounds__(kResAllThreads, 1) res_level_kernel(const Leve
 
   if (!kInv) {
     int32_t* keep_out = reinterpret_cast<int32_t*>(a.out);
-    for (int e = tid; e < per_band; e += kResThreads) {
+    for (int e0 = tid; e0 < n_el; e0 += kResThreads) {
+      const int g = e0 / per_band, e = e0 - g * per_band, bi = b + g;
       const int k = e / pxb, q = e - k * pxb;
-      const int32_t val = v[P.col_out[k] * pg + q];
-      if (k >= P.keep_c) a.z[(size_t)b * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q0 + q] = val;
-      else if (P.is_last) a.z[(size_t)b * P.d + P.z_final_off + (size_t)k * px + q0 + q] = val;
-      else keep_out[((size_t)b * P.keep_c + k) * (size_t)px + q0 + q] = val;
+      const int32_t val = v[P.col_out[k] * pg + g * pxb + q];
+      if (k >= P.keep_c) a.z[(size_t)bi * P.d + P.z_off + (size_t)(k - P.keep_c) * px + q0 + q] = val;
+      else if (P.is_last) a.z[(size_t)bi * P.d + P.z_final_off + (size_t)k * px + q0 + q] = val;
+      else keep_out[((size_t)bi * P.keep_c + k) * (size_t)px + q0 + q] = val;
     }
   } else if (a.phase != 1) {
     const int w2 = 2 * w, rows2 = 2 * hb;
     uint32_t bad = 0;
-    for (int e = tid; e < per_band; e += kResThreads) {
+    for (int e0 = tid; e0 < n_el; e0 += kResThreads) {
+      const int g = e0 / per_band, e = e0 - g * per_band, bi = b + g;
       const int ci = e / (rows2 * w2), r2 = e - ci * rows2 * w2;
       const int y = r2 / w2, x = r2 - y * w2;
       const int gy = 2 * band * hb + y;
-      const int32_t val = v[(ci * 4 + (y & 1) * 2 + (x & 1)) * pg + (y >> 1) * w + (x >> 1)];
-      size_t dst = ((size_t)b * (c / 4) + ci) * (size_t)(4 * px) + (size_t)gy * w2 + x;
+      const int32_t val = v[(ci * 4 + (y & 1) * 2 + (x & 1)) * pg + g * pxb + (y >> 1) * w + (x >> 1)];
+      size_t dst = ((size_t)bi * (c / 4) + ci) * (size_t)(4 * px) + (size_t)gy * w2 + x;
       if (P.is_first && a.img_w > 0) {
-        const int by = rdiv(b, a.mul_patches_x), bx = b - by * a.patches_x;
+        const int by = rdiv(bi, a.mul_patches_x), bx = bi - by * a.patches_x;
         dst = ((size_t)ci * a.img_h + (size_t)(by * 2 * P.h + gy)) * a.img_w + (size_t)(bx * w2 + x);
       }
       if (P.is_first) {

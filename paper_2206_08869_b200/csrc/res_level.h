@@ -70,7 +70,10 @@ struct ResHead {
   // the padded layout above with (hb + 2) rows; the row above and below hold the neighbouring bands'
   // edge rows, which the neighbours write through distributed shared memory after every conv.
   int32_t bands, hb;
-  int32_t pad[1];
+  // Levels whose padded frame (h + 2)(w + 2) fits a 128-position tile several times over: `group` images
+  // per CTA (throughput plan only, bands = 1), their frames one after the other in the padded layout. A
+  // real pixel's taps stay inside its own frame and every frame's border is zero, so nothing else changes.
+  int32_t group;
 };
 static_assert(sizeof(ResHead) == 128, "128-byte header");
 

@@ -22,10 +22,10 @@ def _t(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def _both_ways(G, model, x):
+def _both_ways(G, model, x, plan=0):
     import torch
     z_ref, p_ref = O.forward(O.Packed(model), x)
-    m = G.iodf_create(model, x.shape[0])
+    m = G.iodf_create(model, x.shape[0], plan=plan)
     z, p = G.iodf_forward(m, _t(x))
     G.iodf_check(m)
     np.testing.assert_array_equal(z.cpu().numpy(), z_ref)
@@ -54,6 +54,20 @@ def test_residual_models_bit_exact(G, hw, splits, couplings, hidden, blocks, pru
     model = S.make_residual_model(0xE500 + hw + hidden, 3, hw, hw, splits, couplings, hidden, blocks, prune=prune)
     x = S.smooth_field_images(0xE600 + hw, batch, hw, hw, 2.0)
     _both_ways(G, model, x)
+
+
+@pytest.mark.parametrize("hw,splits,couplings,hidden,blocks,prune,batch", [
+    (8, [True, True], 2, 24, 2, (0.4, 0.8), 11),          # 16- and 4-pixel levels: 3 and 8 images per CTA, ragged last CTAs
+    (16, [True, True, False], 1, 40, 2, (0.4, 0.7), 7),   # 64 pixels (one image per CTA), then 16 and 4 pixels
+    (8, [True], 1, 128, 8, (0.4, 0.7), 4),                # the paper's width and depth at 16 pixels: 3 + 1 images
+    (64, [True, True, True, True], 1, 16, 1, None, 5),    # row bands first (one band per CTA), grouped images at the end
+])
+def test_residual_models_throughput_plan(G, hw, splits, couplings, hidden, blocks, prune, batch):
+    """The throughput plan puts as many images' padded frames into a CTA's tile as it holds: same
+    results, in both directions, with the prior parameters and a last CTA that is not full."""
+    model = S.make_residual_model(0xEB00 + hw + hidden, 3, hw, hw, splits, couplings, hidden, blocks, prune=prune)
+    x = S.smooth_field_images(0xEC00 + hw, batch, hw, hw, 2.0)
+    _both_ways(G, model, x, plan=G.IODF_PLAN_THROUGHPUT)
 
 
 def test_first_level_of_the_imagenet64_geometry_at_the_papers_width(G):
@@ -117,6 +131,47 @@ def test_residual_and_plain_levels_in_one_model_and_stepped_decode(G):
     G.iodf_check(m)
     np.testing.assert_array_equal(prior.cpu().numpy(), p_ref)
     np.testing.assert_array_equal(xr.cpu().numpy(), x)
+
+
+def test_stepped_decode_with_several_images_per_cta(G):
+    """Throughput plan, residual couplings at 64 and 16 pixels (one and three images per CTA), decoded
+    level by level (prior head and couplings as separate launches), five images: a ragged last CTA."""
+    import torch
+    model = S.make_residual_model(0xED00, 3, 16, 16, [True, True], 2, 32, 2, prune=(0.4, 0.7))
+    x = S.smooth_field_images(0xED01, 5, 16, 16, 2.0)
+    m, z_ref, p_ref = _both_ways(G, model, x, plan=G.IODF_PLAN_THROUGHPUT)
+    lay = G.iodf_get_layout(m)
+    z = torch.full((5, int(lay.d)), 0x7A7A7A7A, dtype=torch.int32, device="cuda")
+    zf = int(lay.z_final_off)
+    z[:, zf:] = _t(z_ref[:, zf:])
+    prior = torch.full((5, 2, int(lay.d_fact)), -1, dtype=torch.int32, device="cuda")
+    xr = torch.zeros((5, 3, 16, 16), dtype=torch.uint8, device="cuda")
+    for lv in (1, 0):
+        G.iodf_inverse_level(m, lv, G.IODF_LEVEL_PRIOR, z, prior=prior)
+        zo, n = int(lay.z_off[lv]), (int(lay.level_c[lv]) // 2) * int(lay.level_h[lv]) * int(lay.level_w[lv])
+        z[:, zo:zo + n] = _t(z_ref[:, zo:zo + n])
+        G.iodf_inverse_level(m, lv, G.IODF_LEVEL_COUPLINGS, z, x_u8=xr if lv == 0 else None)
+    G.iodf_check(m)
+    np.testing.assert_array_equal(prior.cpu().numpy(), p_ref)
+    np.testing.assert_array_equal(xr.cpu().numpy(), x)
+
+
+def test_config_r32_throughput_plan_equals_the_default_plan(G):
+    """Config R32 at the benchmark's batch with the plan its steps in flight use (the 4 x 4 level takes
+    three images per CTA): the same latents and prior parameters as the default plan, exact round trip."""
+    import torch
+    model = S.config_model("R32")
+    x = _t(S.config_images("R32"))
+    m0 = G.iodf_create(model, x.shape[0])
+    m1 = G.iodf_create(model, x.shape[0], plan=G.IODF_PLAN_THROUGHPUT)
+    z0, p0 = G.iodf_forward(m0, x)
+    z1, p1 = G.iodf_forward(m1, x)
+    G.iodf_check(m0)
+    G.iodf_check(m1)
+    assert torch.equal(z0, z1) and torch.equal(p0, p1)
+    xr = G.iodf_inverse(m1, z1)
+    G.iodf_check(m1)
+    assert torch.equal(xr, x)
 
 
 def test_config_r32_in_the_benchmarks_launch_configuration(G):
