@@ -1,7 +1,8 @@
 // One flow level whose couplings use the paper's residual-block network (Eq. 3, Sec. 4.1; scatter
 // add, Sec. 4.5; App. B.1: conv 3x3 -> L blocks of two 3x3 convs -> conv 3x3, all on `hidden`
 // channels), one CTA per image of at most 256 pixels at this level; larger images (up to 2048 pixels)
-// are cut into row bands, one CTA of a thread-block cluster each (see "Row bands" below).
+// are cut into row bands, one CTA of a thread-block cluster each (see "Row bands" below), and small
+// ones may share a CTA (ResHead::group images, their padded frames one after the other).
 //
 // Every conv here is a 3x3 conv over hidden activations, so a pixel needs its neighbours' hidden
 // values: the activations of the whole image stay in shared memory (xa: the requantised network
