@@ -114,6 +114,25 @@ def test_patch_coding_equals_the_batch_of_cut_patches(G, hw, splits, hidden, H, 
     assert torch.equal(z, z2)
 
 
+def test_patch_coding_of_residual_couplings_with_several_patches_per_cta(G):
+    """Throughput plan, residual couplings on 4 x 4 patches (2 x 2 pixels at the first level: eight
+    patches' padded frames share a CTA's tile), an image of 11 patches: the patch grid's index map,
+    the grouped frames and a ragged last CTA together."""
+    import torch
+    model = S.make_residual_model(0x9D00, 3, 4, 4, [True], 2, 24, 2, prune=(0.4, 0.7))
+    image = S.smooth_field_images(0x9D01, 1, 4, 44, 3.0)[0]
+    xb = _cut(image, 4, 4)
+    z_ref, p_ref = O.forward(O.Packed(model), xb)
+    m = G.iodf_create(model, xb.shape[0], plan=G.IODF_PLAN_THROUGHPUT)
+    z, p = G.iodf_forward_patches(m, _t(image))
+    G.iodf_check(m)
+    np.testing.assert_array_equal(z.cpu().numpy(), z_ref)
+    np.testing.assert_array_equal(p.cpu().numpy(), p_ref)
+    back = G.iodf_inverse_patches(m, z, 4, 44)
+    G.iodf_check(m)
+    np.testing.assert_array_equal(back.cpu().numpy(), image)
+
+
 def test_patch_argument_errors(G):
     model = S.make_model(0x9C00, 3, 8, 8, [True], 1, 16)
     m = G.iodf_create(model, 4)
