@@ -426,6 +426,11 @@ int iodf_int8_mma_peak(iodf_model* m, uint32_t mma_groups, void* cuda_stream, un
  * library picks one per level when the model is created. "" for a bad argument. */
 const char* iodf_level_kernel_name(const iodf_model* m, int level);
 
+/* Images that one CTA of level `level`'s launch holds under the model's plan (1 where an image takes a
+ * CTA, or a band of a cluster, of its own); a launch of B images has ceil(B / that) CTAs per band.
+ * IODF_EINVAL for a bad argument. */
+int iodf_level_images_per_cta(const iodf_model* m, int level);
+
 /* Number of kernel launches one iodf_forward / iodf_inverse call enqueues. */
 int iodf_launches_per_call(const iodf_model* m, int inverse);
 

@@ -11,6 +11,7 @@ from .binding import (IodfError, Model, iodf_create, iodf_destroy, iodf_forward,
                       iodf_get_layout, iodf_forward_static, iodf_static_scratch_bytes_per_image,
                       IODF_STATIC_SCRATCH_BYTES, iodf_check, iodf_strerror,
                       iodf_launches_per_call, iodf_selftest_timeout, iodf_int8_mma_peak, iodf_level_kernel_name,
+                      iodf_level_images_per_cta,
                       load_library,
                       DECLARED_SYMBOLS)
 
@@ -23,5 +24,6 @@ __all__ = ["IodfError", "Model", "iodf_create", "iodf_destroy", "iodf_forward", 
            "iodf_forward_host", "iodf_inverse_host", "iodf_forward_timed", "iodf_inverse_timed", "iodf_get_layout", "iodf_forward_static", "iodf_static_scratch_bytes_per_image",
            "IODF_STATIC_SCRATCH_BYTES", "iodf_check", "iodf_strerror",
            "iodf_launches_per_call", "iodf_selftest_timeout", "iodf_int8_mma_peak", "iodf_level_kernel_name",
+           "iodf_level_images_per_cta",
            "load_library",
            "DECLARED_SYMBOLS"]

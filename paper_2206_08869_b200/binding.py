@@ -20,6 +20,7 @@ DECLARED_SYMBOLS = ["iodf_create", "iodf_destroy", "iodf_get_layout", "iodf_forw
                     "iodf_forward_host", "iodf_inverse_host", "iodf_forward_timed", "iodf_inverse_timed", "iodf_forward_static",
                     "iodf_static_scratch_bytes_per_image", "iodf_check", "iodf_launches_per_call",
                     "iodf_selftest_timeout", "iodf_int8_mma_peak", "iodf_level_kernel_name",
+                    "iodf_level_images_per_cta",
                     "iodf_strerror", "iodf_last_cuda_error"]
 
 
@@ -152,6 +153,8 @@ def load_library(path=None):
     L.iodf_int8_mma_peak.argtypes = [vp, C.c_uint32, vp, C.POINTER(C.c_ulonglong)]
     L.iodf_level_kernel_name.restype = C.c_char_p
     L.iodf_level_kernel_name.argtypes = [vp, C.c_int]
+    L.iodf_level_images_per_cta.restype = C.c_int
+    L.iodf_level_images_per_cta.argtypes = [vp, C.c_int]
     L.iodf_launches_per_call.restype = C.c_int
     L.iodf_launches_per_call.argtypes = [vp, C.c_int]
     L.iodf_strerror.restype = C.c_char_p
@@ -534,3 +537,10 @@ def iodf_level_kernel_name(model, level):
 
 def iodf_launches_per_call(model, inverse=False):
     return load_library().iodf_launches_per_call(model.handle, int(inverse))
+
+
+def iodf_level_images_per_cta(model, level):
+    n = load_library().iodf_level_images_per_cta(model.handle, int(level))
+    if n < 0:
+        raise IodfError(n, "iodf_level_images_per_cta")
+    return n

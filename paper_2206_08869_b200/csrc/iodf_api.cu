@@ -1474,6 +1474,11 @@ const char* iodf_level_kernel_name(const iodf_model* m, int level) {
   return P.residual ? "res_level_kernel" : (P.pipe ? "level_pipe_kernel" : "level_kernel");
 }
 
+int iodf_level_images_per_cta(const iodf_model* m, int level) {
+  if (!m || level < 0 || level >= (int)m->levels.size()) return IODF_EINVAL;
+  return m->levels[level].plan.group;
+}
+
 int iodf_launches_per_call(const iodf_model* m, int inverse) {
   (void)inverse;
   return m ? (int)m->levels.size() : 0;

@@ -226,6 +226,22 @@ def test_throughput_plan_small_models_bit_exact(G, hw, splits, hidden, prune, ba
     _check_both_ways(G, model, x, plan=G.IODF_PLAN_THROUGHPUT)
 
 
+def test_plans_differ_in_images_per_cta_as_documented(G):
+    """Config 2 at batch 128: one image per CTA at every level under the default plan; under the
+    throughput plan two at the 64-pixel level and four at the 16-pixel level (a full tile there would
+    need streamed weights). Config R32: three 4 x 4 images' padded frames per tile."""
+    model = S.config_model(2)
+    m0, m1 = G.iodf_create(model, 128), G.iodf_create(model, 128, plan=G.IODF_PLAN_THROUGHPUT)
+    assert [G.iodf_level_images_per_cta(m0, lv) for lv in range(4)] == [1, 1, 1, 1]
+    assert [G.iodf_level_images_per_cta(m1, lv) for lv in range(4)] == [1, 1, 2, 4]
+    r = S.config_model("R32")
+    r0, r1 = G.iodf_create(r, 64), G.iodf_create(r, 64, plan=G.IODF_PLAN_THROUGHPUT)
+    assert [G.iodf_level_images_per_cta(r0, lv) for lv in range(3)] == [1, 1, 1]
+    assert [G.iodf_level_images_per_cta(r1, lv) for lv in range(3)] == [1, 1, 3]
+    with pytest.raises(G.IodfError):
+        G.iodf_level_images_per_cta(m0, 4)
+
+
 def test_throughput_plan_config2_equals_the_latency_plan(G):
     """The benchmark keeps several batches in flight on handles made with the throughput plan: same
     latents and prior parameters as the oracle on sampled images, as the default plan on all, exact
